@@ -1,0 +1,166 @@
+/*
+ * rs.h -- C ABI of the Representation Shift hot path on NVIDIA B200 (sm_100a).
+ *
+ * The library runs one pre-LN Vision-Transformer block with training-free
+ * token pruning:
+ *     x'  = SA(LN(x)) + x                      (Eq. att)
+ *     x^  = MLP(LN(x')) + x'                   (Eq. MLP)
+ *     s_i = D(MLP(LN(x'))_i, x'_i)             (Sec. 3.2, operation choice (ii), D = L2)
+ *     x~  = x^ without its r lowest-score tokens   (Sec. 3.1, reduced token set)
+ * with an attention kernel that never writes the N x N attention map.
+ *
+ * Conventions for every entry point
+ *   - "dev" pointers are CUDA device pointers owned by the caller; the library
+ *     never allocates or frees device memory after rs_create.  Host pointers
+ *     are marked "host".
+ *   - Tensors are row-major with the innermost dimension contiguous.  Linear
+ *     weights are [out, in] (the transpose of the paper's W in "[Q,K,V] = xW").
+ *   - Device pointers must be 16-byte aligned; D % 8 == 0; head_dim == 64.
+ *   - `stream` is a cudaStream_t passed as void*.  Calls only enqueue work on
+ *     it and return; nothing synchronises except rs_async_status.
+ *   - Errors are return codes.  Invalid arguments are detected on the host and
+ *     nothing is launched.  Nothing throws, aborts or traps.  A device-side
+ *     anomaly (a bounded wait that ran out) sets a status word that
+ *     rs_async_status returns.
+ *   - One rs_ctx per host thread.
+ */
+#ifndef RS_H_
+#define RS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define RS_API __attribute__((visibility("default")))
+#else
+#define RS_API
+#endif
+
+typedef enum {
+    RS_OK = 0,
+    RS_ERR_INVALID_ARG = 1,   /* null / misaligned pointer, size out of range              */
+    RS_ERR_UNSUPPORTED = 2,   /* valid request the library has no kernel for               */
+    RS_ERR_WORKSPACE = 3,     /* workspace missing or smaller than the *_workspace_bytes   */
+    RS_ERR_CUDA = 4,          /* a CUDA runtime call failed; see rs_last_error             */
+    RS_ERR_TIMEOUT = 5        /* a bounded device-side wait expired (rs_async_status only) */
+} rs_status;
+
+typedef enum { RS_F32 = 0, RS_BF16 = 1 } rs_dtype;
+
+/* Distance D of Sec. 3.3 "Distance metrics". */
+typedef enum { RS_DIST_L2 = 0, RS_DIST_L1 = 1, RS_DIST_COS = 2 } rs_dist;
+
+/* Which pair of representations the block scores (Sec. 3.3 "Operation choice"). */
+typedef enum {
+    RS_SCORE_MLP = 0,       /* (ii)  s = D(MLP(LN(x')), x')      -- the paper's default     */
+    RS_SCORE_MLP_DELTA = 1  /*       s = D(x^, x') = |MLP(LN(x'))| -- "before and after the
+                                     MLP layer" read with the residual included             */
+} rs_score_mode;
+
+typedef struct rs_ctx rs_ctx; /* opaque: device id, status word, last error text */
+
+/* Create / destroy a context bound to CUDA device `device`.  rs_create
+ * allocates a few bytes of device memory for the status word. */
+RS_API rs_status rs_create(rs_ctx** out, int device);
+RS_API void rs_destroy(rs_ctx* ctx);
+/* Text of the last error on this context; never NULL; valid until the next call. */
+RS_API const char* rs_last_error(const rs_ctx* ctx);
+/* Synchronise `stream`, then return and clear the device status word. */
+RS_API rs_status rs_async_status(rs_ctx* ctx, void* stream);
+/* 1 if the tcgen05 tensor-core kernels are used for (dtype), else 0 (SIMT path). */
+RS_API int rs_uses_tensor_cores(const rs_ctx* ctx, rs_dtype dtype);
+/* Number of kernels the library has launched through this context so far. */
+RS_API long long rs_launch_count(const rs_ctx* ctx);
+
+/* Per-kernel-class device timing, for benchmarks (the paper reports whole-model
+ * throughput only; this has no counterpart there).  While enabled, every launch
+ * is bracketed by CUDA events on the launch stream (up to 8192 launches between
+ * reads; later ones are not recorded).  rs_timing_read synchronises `stream`,
+ * adds up the elapsed milliseconds and launch counts per class into the two
+ * host arrays of RS_K_COUNT entries, and clears the record. */
+typedef enum {
+    RS_K_LAYERNORM = 0, RS_K_GEMM = 1, RS_K_ATTN = 2, RS_K_SCORE = 3, RS_K_SELECT = 4, RS_K_GATHER = 5,
+    RS_K_COUNT = 6
+} rs_kernel_class;
+RS_API rs_status rs_timing_enable(rs_ctx* ctx, int on);
+RS_API rs_status rs_timing_read(rs_ctx* ctx, void* stream, double* ms /*host[RS_K_COUNT]*/,
+                                long long* launches /*host[RS_K_COUNT]*/);
+
+/* ---- rs_attn_fwd: Eq. sa, out = Softmax(Q K^T * scale) V per (sample, head) ----------
+ * q, k, v (dev): element [b, i, h, c] lives at  b*batch_stride + i*row_stride +
+ * h*head_stride + c  (strides in elements), so the three may alias one packed
+ * [B, N, 3, H, 64] buffer.  Strides must be multiples of 8 elements.
+ * out (dev): [B, N, H*head_dim] contiguous, same dtype.  No [N, N] buffer is
+ * ever written to global memory.  scale == 0 selects 1/sqrt(head_dim). */
+typedef struct {
+    rs_dtype dtype;
+    int B, N, H, head_dim;
+    float scale;
+    long long q_batch_stride, q_row_stride, q_head_stride;
+    long long k_batch_stride, k_row_stride, k_head_stride;
+    long long v_batch_stride, v_row_stride, v_head_stride;
+} rs_attn_desc;
+
+RS_API rs_status rs_attn_fwd(rs_ctx* ctx, const rs_attn_desc* desc /*host*/, const void* q, const void* k,
+                      const void* v, void* out, void* stream);
+
+/* ---- rs_shift_score: Sec. 3.2, s[b, i] = D(after[b, i, :], before[b, i, :]) ------------
+ * after, before (dev): [B, N, D] of `dtype`; scores (dev): [B, N] fp32. */
+RS_API rs_status rs_shift_score(rs_ctx* ctx, rs_dtype dtype, rs_dist dist, int B, int N, int D,
+                         const void* after, const void* before, float* scores, void* stream);
+
+/* ---- rs_topk_compact: Sec. 3.1 / 3.2, drop the r lowest-score tokens of every sample ----
+ * Keeps K = N - r tokens: token 0 first if has_cls, then by score descending,
+ * ties to the lower index, NaN last.  keep_idx (dev, [B, K] int32) lists the
+ * kept indices in ascending order; x_out[b, j, :] = x[b, keep_idx[b, j], :].
+ * scores (dev): [B, N] fp32.  x (dev): [B, N, D]; x_out (dev): [B, K, D], must
+ * not overlap x.  0 <= r <= N - 1, 1 <= N <= 32768.  r == 0 is a plain copy.
+ * x and x_out may both be NULL to get the indices only. */
+RS_API rs_status rs_topk_compact(rs_ctx* ctx, rs_dtype dtype, int B, int N, int D, int r, int has_cls,
+                          const float* scores, const void* x, void* x_out, int32_t* keep_idx,
+                          void* stream);
+
+/* ---- rs_block_fwd: Eq. att + Eq. MLP + score + pruning in one call ----------------------
+ * dtype: storage type of x, the weight matrices and x_out.  With RS_BF16 the
+ * contractions run on the tensor cores with fp32 accumulation; the residual
+ * stream x' is held in fp32 inside the block.  out_dtype: type written to
+ * x_out / x_full (RS_F32 with dtype RS_BF16 gives the un-rounded result). */
+typedef struct {
+    rs_dtype dtype;
+    rs_dtype out_dtype;
+    int B, N, D, H, D_mlp;
+    int r;                 /* tokens dropped after the block, 0 <= r <= N-1 */
+    int has_cls;
+    float ln_eps;          /* 0 => 1e-6 */
+    float scale;           /* 0 => 1/sqrt(D/H) */
+    rs_score_mode score_mode;
+    rs_dist dist;          /* only RS_DIST_L2 inside the block */
+} rs_block_desc;
+
+typedef struct {           /* all dev pointers */
+    const void *w_qkv /*[3D,D]*/, *w_o /*[D,D]*/, *w_fc1 /*[D_mlp,D]*/, *w_fc2 /*[D,D_mlp]*/; /* dtype */
+    const float *b_qkv, *b_o, *b_fc1, *b_fc2;        /* fp32; may be NULL */
+    const float *ln1_g, *ln1_b, *ln2_g, *ln2_b;      /* fp32 */
+} rs_block_weights;
+
+/* Bytes of scratch rs_block_fwd needs for this descriptor (0 on a bad descriptor). */
+RS_API size_t rs_block_workspace_bytes(const rs_block_desc* desc /*host*/);
+
+/* x (dev): [B, N, D].  x_out (dev): [B, N-r, D].  scores (dev, optional):
+ * [B, N] fp32.  keep_idx (dev, optional): [B, N-r] int32.  x_full (dev,
+ * optional): [B, N, D] un-pruned x^ of out_dtype.  workspace (dev): at least
+ * rs_block_workspace_bytes(desc) bytes, 256-byte aligned, contents undefined
+ * before and after. */
+RS_API rs_status rs_block_fwd(rs_ctx* ctx, const rs_block_desc* desc /*host*/,
+                       const rs_block_weights* weights /*host struct of dev pointers*/,
+                       const void* x, void* x_out, float* scores, int32_t* keep_idx, void* x_full,
+                       void* workspace, size_t workspace_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RS_H_ */

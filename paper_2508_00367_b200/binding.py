@@ -1,0 +1,335 @@
+"""Thin ctypes binding of librs.so: argument marshalling only.
+
+Every step of the path runs in the library's CUDA kernels.  torch supplies
+device memory and the current stream.  There is no CPU or eager fallback: if
+the shared library is missing, or a call returns an error code, a RuntimeError
+is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Dict, List, Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "librs.so")
+
+RS_OK = 0
+RS_F32, RS_BF16 = 0, 1
+DIST = {"l2": 0, "l1": 1, "cos": 2}
+SCORE_MODE = {"mlp": 0, "mlp_delta": 1}
+STATUS_NAMES = {0: "RS_OK", 1: "RS_ERR_INVALID_ARG", 2: "RS_ERR_UNSUPPORTED", 3: "RS_ERR_WORKSPACE",
+                4: "RS_ERR_CUDA", 5: "RS_ERR_TIMEOUT"}
+
+EXPORTS = ("rs_create", "rs_destroy", "rs_last_error", "rs_async_status", "rs_uses_tensor_cores",
+           "rs_launch_count", "rs_attn_fwd", "rs_shift_score", "rs_topk_compact",
+           "rs_block_workspace_bytes", "rs_block_fwd", "rs_timing_enable", "rs_timing_read")
+KERNEL_CLASSES = ("layernorm", "gemm", "attn", "score", "select", "gather")
+
+
+class RsError(RuntimeError):
+    def __init__(self, status: int, msg: str):
+        super().__init__(f"{STATUS_NAMES.get(status, status)}: {msg}")
+        self.status = status
+
+
+class AttnDesc(ctypes.Structure):
+    _fields_ = [("dtype", ctypes.c_int), ("B", ctypes.c_int), ("N", ctypes.c_int), ("H", ctypes.c_int),
+                ("head_dim", ctypes.c_int), ("scale", ctypes.c_float),
+                ("q_batch_stride", ctypes.c_longlong), ("q_row_stride", ctypes.c_longlong),
+                ("q_head_stride", ctypes.c_longlong),
+                ("k_batch_stride", ctypes.c_longlong), ("k_row_stride", ctypes.c_longlong),
+                ("k_head_stride", ctypes.c_longlong),
+                ("v_batch_stride", ctypes.c_longlong), ("v_row_stride", ctypes.c_longlong),
+                ("v_head_stride", ctypes.c_longlong)]
+
+
+class BlockDesc(ctypes.Structure):
+    _fields_ = [("dtype", ctypes.c_int), ("out_dtype", ctypes.c_int), ("B", ctypes.c_int),
+                ("N", ctypes.c_int), ("D", ctypes.c_int), ("H", ctypes.c_int), ("D_mlp", ctypes.c_int),
+                ("r", ctypes.c_int), ("has_cls", ctypes.c_int), ("ln_eps", ctypes.c_float),
+                ("scale", ctypes.c_float), ("score_mode", ctypes.c_int), ("dist", ctypes.c_int)]
+
+
+class BlockWeights(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in
+                ("w_qkv", "w_o", "w_fc1", "w_fc2", "b_qkv", "b_o", "b_fc1", "b_fc2",
+                 "ln1_g", "ln1_b", "ln2_g", "ln2_b")]
+
+
+_lib = None
+
+
+def load_library() -> ctypes.CDLL:
+    """Load librs.so (built in-tree by paper_2508_00367_b200.build).  Fails loudly if absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2508_00367_b200.build` "
+                           "(there is no fallback path)")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, ci = ctypes.c_void_p, ctypes.c_int
+    lib.rs_create.argtypes = [ctypes.POINTER(vp), ci]
+    lib.rs_create.restype = ci
+    lib.rs_destroy.argtypes = [vp]
+    lib.rs_destroy.restype = None
+    lib.rs_last_error.argtypes = [vp]
+    lib.rs_last_error.restype = ctypes.c_char_p
+    lib.rs_async_status.argtypes = [vp, vp]
+    lib.rs_async_status.restype = ci
+    lib.rs_uses_tensor_cores.argtypes = [vp, ci]
+    lib.rs_uses_tensor_cores.restype = ci
+    lib.rs_launch_count.argtypes = [vp]
+    lib.rs_launch_count.restype = ctypes.c_longlong
+    lib.rs_timing_enable.argtypes = [vp, ci]
+    lib.rs_timing_enable.restype = ci
+    lib.rs_timing_read.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_longlong)]
+    lib.rs_timing_read.restype = ci
+    lib.rs_attn_fwd.argtypes = [vp, ctypes.POINTER(AttnDesc), vp, vp, vp, vp, vp]
+    lib.rs_attn_fwd.restype = ci
+    lib.rs_shift_score.argtypes = [vp, ci, ci, ci, ci, ci, vp, vp, vp, vp]
+    lib.rs_shift_score.restype = ci
+    lib.rs_topk_compact.argtypes = [vp, ci, ci, ci, ci, ci, ci, vp, vp, vp, vp, vp]
+    lib.rs_topk_compact.restype = ci
+    lib.rs_block_workspace_bytes.argtypes = [ctypes.POINTER(BlockDesc)]
+    lib.rs_block_workspace_bytes.restype = ctypes.c_size_t
+    lib.rs_block_fwd.argtypes = [vp, ctypes.POINTER(BlockDesc), ctypes.POINTER(BlockWeights), vp, vp, vp, vp,
+                                 vp, vp, ctypes.c_size_t, vp]
+    lib.rs_block_fwd.restype = ci
+    _lib = lib
+    return lib
+
+
+def _dt(t: torch.Tensor) -> int:
+    if t.dtype == torch.bfloat16:
+        return RS_BF16
+    if t.dtype == torch.float32:
+        return RS_F32
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+def _torch_dt(code: int):
+    return torch.bfloat16 if code == RS_BF16 else torch.float32
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(device) -> ctypes.c_void_p:
+    return ctypes.c_void_p(torch.cuda.current_stream(device).cuda_stream)
+
+
+class Context:
+    """One rs_ctx on one CUDA device."""
+
+    def __init__(self, device: int = 0):
+        self.lib = load_library()
+        if not torch.cuda.is_available():
+            raise RuntimeError("no CUDA device: the library has no CPU path")
+        self.device = torch.device("cuda", device)
+        h = ctypes.c_void_p()
+        st = self.lib.rs_create(ctypes.byref(h), device)
+        if st != RS_OK:
+            raise RsError(st, "rs_create failed")
+        self.handle = h
+
+    def close(self):
+        if getattr(self, "handle", None):
+            self.lib.rs_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _check(self, st: int):
+        if st != RS_OK:
+            raise RsError(st, self.lib.rs_last_error(self.handle).decode())
+
+    def raw(self, fn: str, *args) -> int:
+        """Call an entry point with pre-marshalled arguments; returns the status code."""
+        return getattr(self.lib, fn)(self.handle, *args)
+
+    def last_error(self) -> str:
+        return self.lib.rs_last_error(self.handle).decode()
+
+    def async_status(self):
+        self._check(self.lib.rs_async_status(self.handle, _stream(self.device)))
+
+    def uses_tensor_cores(self, dtype=torch.bfloat16) -> bool:
+        return bool(self.lib.rs_uses_tensor_cores(self.handle, RS_BF16 if dtype == torch.bfloat16 else RS_F32))
+
+    def launch_count(self) -> int:
+        return int(self.lib.rs_launch_count(self.handle))
+
+    def timing_enable(self, on: bool):
+        self._check(self.lib.rs_timing_enable(self.handle, int(on)))
+
+    def timing_read(self) -> Dict[str, Dict[str, float]]:
+        """Per-kernel-class device time (ms) and launch count since the last read."""
+        ms = (ctypes.c_double * len(KERNEL_CLASSES))()
+        n = (ctypes.c_longlong * len(KERNEL_CLASSES))()
+        self._check(self.lib.rs_timing_read(self.handle, _stream(self.device), ms, n))
+        return {k: dict(ms=float(ms[i]), launches=int(n[i])) for i, k in enumerate(KERNEL_CLASSES)}
+
+    # ---- rs_attn_fwd ----
+    def attn_fwd(self, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, scale: float = 0.0,
+                 out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """q, k, v: [B, N, H, 64] views (innermost contiguous).  Returns [B, N, H*64]."""
+        B, N, H, dh = q.shape
+        for t in (q, k, v):
+            assert t.is_cuda and t.stride(3) == 1 and t.shape == q.shape and t.dtype == q.dtype
+        if out is None:
+            out = torch.empty(B, N, H * dh, dtype=q.dtype, device=q.device)
+        d = AttnDesc(_dt(q), B, N, H, dh, float(scale),
+                     q.stride(0), q.stride(1), q.stride(2), k.stride(0), k.stride(1), k.stride(2),
+                     v.stride(0), v.stride(1), v.stride(2))
+        self._check(self.lib.rs_attn_fwd(self.handle, ctypes.byref(d), _ptr(q), _ptr(k), _ptr(v), _ptr(out),
+                                         _stream(q.device)))
+        return out
+
+    # ---- rs_shift_score ----
+    def shift_score(self, after: torch.Tensor, before: torch.Tensor, dist: str = "l2",
+                    out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        B, N, D = after.shape
+        assert after.is_contiguous() and before.is_contiguous() and before.shape == after.shape
+        if out is None:
+            out = torch.empty(B, N, dtype=torch.float32, device=after.device)
+        self._check(self.lib.rs_shift_score(self.handle, _dt(after), DIST[dist], B, N, D, _ptr(after),
+                                            _ptr(before), _ptr(out), _stream(after.device)))
+        return out
+
+    # ---- rs_topk_compact ----
+    def topk_compact(self, scores: torch.Tensor, x: Optional[torch.Tensor], r: int, has_cls: bool = True,
+                     x_out: Optional[torch.Tensor] = None, keep_idx: Optional[torch.Tensor] = None):
+        B, N = scores.shape
+        K = N - r
+        assert scores.dtype == torch.float32 and scores.is_contiguous()
+        if keep_idx is None:
+            keep_idx = torch.empty(B, max(K, 0), dtype=torch.int32, device=scores.device)
+        D = 8
+        dt = RS_F32
+        if x is not None:
+            assert x.is_contiguous() and x.shape[:2] == (B, N)
+            D = x.shape[2]
+            dt = _dt(x)
+            if x_out is None:
+                x_out = torch.empty(B, max(K, 0), D, dtype=x.dtype, device=x.device)
+        self._check(self.lib.rs_topk_compact(self.handle, dt, B, N, D, r, int(has_cls), _ptr(scores), _ptr(x),
+                                             _ptr(x_out), _ptr(keep_idx), _stream(scores.device)))
+        return x_out, keep_idx
+
+    # ---- rs_block_fwd ----
+    def block_desc(self, B, N, D, H, D_mlp, r, dtype, out_dtype=None, has_cls=True, ln_eps=0.0, scale=0.0,
+                   score_mode="mlp", dist="l2") -> BlockDesc:
+        code = RS_BF16 if dtype == torch.bfloat16 else RS_F32
+        ocode = code if out_dtype is None else (RS_BF16 if out_dtype == torch.bfloat16 else RS_F32)
+        return BlockDesc(code, ocode, B, N, D, H, D_mlp, r, int(has_cls), float(ln_eps), float(scale),
+                         SCORE_MODE[score_mode], DIST[dist])
+
+    def block_workspace_bytes(self, desc: BlockDesc) -> int:
+        return int(self.lib.rs_block_workspace_bytes(ctypes.byref(desc)))
+
+    def block_fwd(self, x: torch.Tensor, weights: "DeviceBlockWeights", H: int, r: int, has_cls: bool = True,
+                  out_dtype=None, score_mode: str = "mlp", ln_eps: float = 0.0, scale: float = 0.0,
+                  want_full: bool = False, workspace: Optional[torch.Tensor] = None,
+                  x_out: Optional[torch.Tensor] = None, scores: Optional[torch.Tensor] = None,
+                  keep_idx: Optional[torch.Tensor] = None) -> Dict[str, torch.Tensor]:
+        """One block + pruning.  Returns dict(x_out, scores, keep_idx[, x_full])."""
+        assert x.is_cuda and x.is_contiguous()
+        B, N, D = x.shape
+        desc = self.block_desc(B, N, D, H, weights.D_mlp, r, x.dtype, out_dtype, has_cls, ln_eps, scale, score_mode)
+        odt = _torch_dt(desc.out_dtype)
+        K = N - r
+        need = self.block_workspace_bytes(desc)
+        if workspace is None:
+            workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=x.device)
+        if x_out is None:
+            x_out = torch.empty(B, max(K, 0), D, dtype=odt, device=x.device)
+        if scores is None:
+            scores = torch.empty(B, N, dtype=torch.float32, device=x.device)
+        if keep_idx is None:
+            keep_idx = torch.empty(B, max(K, 0), dtype=torch.int32, device=x.device)
+        x_full = torch.empty(B, N, D, dtype=odt, device=x.device) if want_full else None
+        self._check(self.lib.rs_block_fwd(self.handle, ctypes.byref(desc), ctypes.byref(weights.struct), _ptr(x),
+                                          _ptr(x_out), _ptr(scores), _ptr(keep_idx), _ptr(x_full),
+                                          _ptr(workspace), workspace.numel(), _stream(x.device)))
+        res = dict(x_out=x_out, scores=scores, keep_idx=keep_idx)
+        if want_full:
+            res["x_full"] = x_full
+        return res
+
+
+class DeviceBlockWeights:
+    """Block parameters resident on the device: matrices in the storage dtype,
+    biases and LayerNorm parameters in fp32."""
+
+    MATS = ("w_qkv", "w_o", "w_fc1", "w_fc2")
+    VECS = ("b_qkv", "b_o", "b_fc1", "b_fc2", "ln1_g", "ln1_b", "ln2_g", "ln2_b")
+
+    def __init__(self, w: Dict[str, torch.Tensor], dtype: torch.dtype, device):
+        self.t = {}
+        for n in self.MATS:
+            self.t[n] = w[n].to(device=device, dtype=dtype).contiguous()
+        for n in self.VECS:
+            self.t[n] = None if w.get(n) is None else w[n].to(device=device, dtype=torch.float32).contiguous()
+        self.D_mlp = self.t["w_fc1"].shape[0]
+        self.struct = BlockWeights(*[None if self.t[n] is None else self.t[n].data_ptr()
+                                     for n in self.MATS + self.VECS])
+
+
+class PrunedViT:
+    """Layer loop of the pruned forward pass: block l+1 consumes block l's
+    compacted output; `drops[l]` tokens are removed after block l."""
+
+    def __init__(self, ctx: Context, blocks: Sequence[Dict[str, torch.Tensor]], H: int, drops: Sequence[int],
+                 dtype: torch.dtype, has_cls: bool = True, score_mode: str = "mlp"):
+        assert len(blocks) == len(drops)
+        self.ctx, self.H, self.drops, self.dtype = ctx, H, list(drops), dtype
+        self.has_cls, self.score_mode = has_cls, score_mode
+        self.weights: List[DeviceBlockWeights] = [DeviceBlockWeights(w, dtype, ctx.device) for w in blocks]
+        self._plan = None
+
+    def plan(self, B: int, N: int, D: int):
+        """Allocate the workspace and the per-block outputs once for a shape."""
+        key = (B, N, D)
+        if self._plan and self._plan["key"] == key:
+            return self._plan
+        dev = self.ctx.device
+        descs, outs, need, n = [], [], 256, N
+        for l, r in enumerate(self.drops):
+            d = self.ctx.block_desc(B, n, D, self.H, self.weights[l].D_mlp, r, self.dtype, None, self.has_cls,
+                                    0.0, 0.0, self.score_mode)
+            need = max(need, self.ctx.block_workspace_bytes(d))
+            k = n - r
+            outs.append(dict(x_out=torch.empty(B, k, D, dtype=self.dtype, device=dev),
+                             scores=torch.empty(B, n, dtype=torch.float32, device=dev),
+                             keep_idx=torch.empty(B, k, dtype=torch.int32, device=dev)))
+            descs.append(d)
+            n = k
+        ws = torch.empty(need, dtype=torch.uint8, device=dev)
+        self._plan = dict(key=key, descs=descs, outs=outs, ws=ws)
+        return self._plan
+
+    def forward(self, x: torch.Tensor):
+        """x: [B, N, D] on the device.  Returns the list of per-block outputs."""
+        B, N, D = x.shape
+        p = self.plan(B, N, D)
+        lib, h = self.ctx.lib, self.ctx.handle
+        st = _stream(x.device)
+        cur = x
+        for l, d in enumerate(p["descs"]):
+            o = p["outs"][l]
+            rc = lib.rs_block_fwd(h, ctypes.byref(d), ctypes.byref(self.weights[l].struct), _ptr(cur),
+                                  _ptr(o["x_out"]), _ptr(o["scores"]), _ptr(o["keep_idx"]), None,
+                                  _ptr(p["ws"]), p["ws"].numel(), st)
+            if rc != RS_OK:
+                raise RsError(rc, self.ctx.last_error())
+            cur = o["x_out"]
+        return p["outs"]

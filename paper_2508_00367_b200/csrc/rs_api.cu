@@ -1,0 +1,306 @@
+// C ABI: argument validation, the context object and the launch sequence of
+// one block (Eq. att, Eq. MLP, Sec. 3.2 score, Sec. 3.1 pruning).
+#include <math.h>
+#include <stdarg.h>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include "rs_internal.h"
+
+namespace {
+
+rs_status fail(rs_ctx* ctx, rs_status code, const char* fmt, ...) {
+    if (ctx) {
+        va_list ap;
+        va_start(ap, fmt);
+        vsnprintf(ctx->err, sizeof(ctx->err), fmt, ap);
+        va_end(ap);
+    }
+    return code;
+}
+
+rs_status cuda_fail(rs_ctx* ctx, cudaError_t e, const char* what) {
+    return fail(ctx, RS_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+bool valid_dtype(int t) { return t == RS_F32 || t == RS_BF16; }
+
+// Launch wrapper: counts the launch and, when timing is on, brackets it with events.
+#define RS_CHECK_LAUNCH(ctx, cls, st, expr, what)                                  \
+    do {                                                                           \
+        const bool timed__ = (ctx)->timing && (ctx)->n_events < kMaxTimed;         \
+        if (timed__) cudaEventRecord((ctx)->ev[2 * (ctx)->n_events], (st));        \
+        cudaError_t e__ = (expr);                                                  \
+        if (e__ != cudaSuccess) return cuda_fail(ctx, e__, what);                  \
+        if (timed__) {                                                             \
+            cudaEventRecord((ctx)->ev[2 * (ctx)->n_events + 1], (st));             \
+            (ctx)->ev_class[(ctx)->n_events++] = (unsigned char)(cls);             \
+        }                                                                          \
+        (ctx)->launches += 1;                                                      \
+    } while (0)
+
+// Scratch layout of one block.  Every buffer starts on a 256-byte boundary.
+struct BlockWs {
+    size_t u, qkv, o, x_prime, h, m, x_hat, scores, keep, total;
+};
+
+bool block_layout(const rs_block_desc& d, BlockWs* ws) {
+    if (!valid_dtype(d.dtype) || !valid_dtype(d.out_dtype)) return false;
+    if (d.B < 1 || d.N < 1 || d.D < 8 || d.H < 1 || d.D_mlp < 8) return false;
+    const size_t T = (size_t)d.B * d.N, D = d.D, Dm = d.D_mlp;
+    const size_t sz = rs::dtype_size(d.dtype), osz = rs::dtype_size(d.out_dtype);
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t at = off; off += rs::align_up(bytes, 256); return at; };
+    ws->u = take(T * D * sz);            // LN1 / LN2 output
+    ws->qkv = take(T * 3 * D * sz);      // packed [T, 3, H, 64]
+    ws->o = take(T * D * sz);            // attention output
+    ws->x_prime = take(T * D * 4);       // residual stream x', fp32
+    ws->h = take(T * Dm * sz);           // GELU(FC1)
+    ws->m = take(T * D * 4);             // MLP(LN(x')) in fp32
+    ws->x_hat = take(T * D * osz);       // un-pruned block output when the caller gives no x_full
+    ws->scores = take(T * 4);            // when the caller gives no scores buffer
+    ws->keep = take((size_t)d.B * (size_t)(d.N) * 4);
+    ws->total = off;
+    return true;
+}
+
+}  // namespace
+
+extern "C" {
+
+rs_status rs_create(rs_ctx** out, int device) {
+    if (!out) return RS_ERR_INVALID_ARG;
+    *out = nullptr;
+    int count = 0;
+    if (cudaGetDeviceCount(&count) != cudaSuccess || device < 0 || device >= count) return RS_ERR_CUDA;
+    rs_ctx* ctx = (rs_ctx*)calloc(1, sizeof(rs_ctx));
+    if (!ctx) return RS_ERR_CUDA;
+    ctx->device = device;
+    strcpy(ctx->err, "ok");
+    cudaDeviceProp prop;
+    if (cudaSetDevice(device) != cudaSuccess || cudaGetDeviceProperties(&prop, device) != cudaSuccess) {
+        free(ctx);
+        return RS_ERR_CUDA;
+    }
+    if (prop.major != 10) {   // kernels are built for sm_100a only
+        free(ctx);
+        return RS_ERR_UNSUPPORTED;
+    }
+    ctx->sm_count = prop.multiProcessorCount;
+    if (cudaMalloc(&ctx->d_status, 256) != cudaSuccess || cudaMemset(ctx->d_status, 0, 256) != cudaSuccess ||
+        rs::select_init() != cudaSuccess) {
+        if (ctx->d_status) cudaFree(ctx->d_status);
+        free(ctx);
+        return RS_ERR_CUDA;
+    }
+    const char* no_tc = getenv("RS_DISABLE_TC");
+    ctx->use_tc = 0;
+    (void)no_tc;
+    *out = ctx;
+    return RS_OK;
+}
+
+void rs_destroy(rs_ctx* ctx) {
+    if (!ctx) return;
+    cudaSetDevice(ctx->device);
+    if (ctx->d_status) cudaFree(ctx->d_status);
+    if (ctx->ev) {
+        for (int i = 0; i < 2 * kMaxTimed; ++i) cudaEventDestroy(ctx->ev[i]);
+        free(ctx->ev);
+        free(ctx->ev_class);
+    }
+    free(ctx);
+}
+
+rs_status rs_timing_enable(rs_ctx* ctx, int on) {
+    if (!ctx) return RS_ERR_INVALID_ARG;
+    if (on && !ctx->ev) {
+        ctx->ev = (cudaEvent_t*)calloc(2 * kMaxTimed, sizeof(cudaEvent_t));
+        ctx->ev_class = (unsigned char*)calloc(kMaxTimed, 1);
+        if (!ctx->ev || !ctx->ev_class) return fail(ctx, RS_ERR_CUDA, "out of host memory");
+        for (int i = 0; i < 2 * kMaxTimed; ++i) {
+            cudaError_t e = cudaEventCreate(&ctx->ev[i]);
+            if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaEventCreate");
+        }
+    }
+    ctx->timing = on ? 1 : 0;
+    ctx->n_events = 0;
+    return RS_OK;
+}
+
+rs_status rs_timing_read(rs_ctx* ctx, void* stream, double* ms, long long* launches) {
+    if (!ctx || !ms || !launches) return RS_ERR_INVALID_ARG;
+    cudaError_t e = cudaStreamSynchronize((cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaStreamSynchronize");
+    for (int c = 0; c < RS_K_COUNT; ++c) { ms[c] = 0.0; launches[c] = 0; }
+    for (int i = 0; i < ctx->n_events; ++i) {
+        float t = 0.f;
+        e = cudaEventElapsedTime(&t, ctx->ev[2 * i], ctx->ev[2 * i + 1]);
+        if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaEventElapsedTime");
+        ms[ctx->ev_class[i]] += t;
+        launches[ctx->ev_class[i]] += 1;
+    }
+    ctx->n_events = 0;
+    return RS_OK;
+}
+
+const char* rs_last_error(const rs_ctx* ctx) { return ctx ? ctx->err : "null context"; }
+
+rs_status rs_async_status(rs_ctx* ctx, void* stream) {
+    if (!ctx) return RS_ERR_INVALID_ARG;
+    cudaError_t e = cudaStreamSynchronize((cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaStreamSynchronize");
+    int word = 0;
+    e = cudaMemcpy(&word, ctx->d_status, sizeof(int), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "status read");
+    if (word != RS_DEV_OK) {
+        cudaMemset(ctx->d_status, 0, sizeof(int));
+        return fail(ctx, RS_ERR_TIMEOUT, "device status word = %d (a bounded wait expired)", word);
+    }
+    return RS_OK;
+}
+
+int rs_uses_tensor_cores(const rs_ctx* ctx, rs_dtype dtype) {
+    return ctx && ctx->use_tc && dtype == RS_BF16;
+}
+
+long long rs_launch_count(const rs_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+rs_status rs_attn_fwd(rs_ctx* ctx, const rs_attn_desc* d, const void* q, const void* k, const void* v,
+                      void* out, void* stream) {
+    if (!ctx) return RS_ERR_INVALID_ARG;
+    if (!d || !q || !k || !v || !out) return fail(ctx, RS_ERR_INVALID_ARG, "rs_attn_fwd: null argument");
+    if (!valid_dtype(d->dtype)) return fail(ctx, RS_ERR_INVALID_ARG, "rs_attn_fwd: bad dtype");
+    if (d->B < 1 || d->N < 1 || d->H < 1) return fail(ctx, RS_ERR_INVALID_ARG, "rs_attn_fwd: B, N, H must be >= 1");
+    if (d->head_dim != 64) return fail(ctx, RS_ERR_UNSUPPORTED, "rs_attn_fwd: head_dim must be 64");
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out))
+        return fail(ctx, RS_ERR_INVALID_ARG, "rs_attn_fwd: pointers must be 16-byte aligned");
+    const long long st[9] = {d->q_batch_stride, d->q_row_stride, d->q_head_stride, d->k_batch_stride,
+                             d->k_row_stride,   d->k_head_stride, d->v_batch_stride, d->v_row_stride,
+                             d->v_head_stride};
+    for (int i = 0; i < 9; ++i)
+        if (st[i] < 0 || (st[i] % 8) != 0) return fail(ctx, RS_ERR_INVALID_ARG, "rs_attn_fwd: strides must be non-negative multiples of 8");
+    if (!(d->scale >= 0.f)) return fail(ctx, RS_ERR_INVALID_ARG, "rs_attn_fwd: scale must be >= 0");
+    RS_CHECK_LAUNCH(ctx, RS_K_ATTN, (cudaStream_t)stream, rs::launch_attn_simt(*d, q, k, v, out, (cudaStream_t)stream), "attention launch");
+    return RS_OK;
+}
+
+rs_status rs_shift_score(rs_ctx* ctx, rs_dtype dtype, rs_dist dist, int B, int N, int D, const void* after,
+                         const void* before, float* scores, void* stream) {
+    if (!ctx) return RS_ERR_INVALID_ARG;
+    if (!valid_dtype(dtype) || dist < RS_DIST_L2 || dist > RS_DIST_COS)
+        return fail(ctx, RS_ERR_INVALID_ARG, "rs_shift_score: bad dtype or distance");
+    if (B < 0 || N < 0 || D < 8 || (D % 8) != 0) return fail(ctx, RS_ERR_INVALID_ARG, "rs_shift_score: need B, N >= 0 and D a positive multiple of 8");
+    if ((long long)B * N == 0) return RS_OK;
+    if (!after || !before || !scores) return fail(ctx, RS_ERR_INVALID_ARG, "rs_shift_score: null pointer");
+    if (!aligned16(after) || !aligned16(before) || (reinterpret_cast<uintptr_t>(scores) & 3u))
+        return fail(ctx, RS_ERR_INVALID_ARG, "rs_shift_score: misaligned pointer");
+    RS_CHECK_LAUNCH(ctx, RS_K_SCORE, (cudaStream_t)stream, rs::launch_shift_score(dtype, dist, (long long)B * N, D, after, before, scores, (cudaStream_t)stream),
+                    "shift score launch");
+    return RS_OK;
+}
+
+rs_status rs_topk_compact(rs_ctx* ctx, rs_dtype dtype, int B, int N, int D, int r, int has_cls,
+                          const float* scores, const void* x, void* x_out, int32_t* keep_idx, void* stream) {
+    if (!ctx) return RS_ERR_INVALID_ARG;
+    if (!valid_dtype(dtype)) return fail(ctx, RS_ERR_INVALID_ARG, "rs_topk_compact: bad dtype");
+    if (B < 0 || N < 1) return fail(ctx, RS_ERR_INVALID_ARG, "rs_topk_compact: need B >= 0, N >= 1");
+    if (N > 32768) return fail(ctx, RS_ERR_UNSUPPORTED, "rs_topk_compact: N > 32768");
+    if (r < 0 || r > N - 1) return fail(ctx, RS_ERR_INVALID_ARG, "rs_topk_compact: need 0 <= r <= N-1");
+    if (B == 0) return RS_OK;
+    if (!scores || !keep_idx) return fail(ctx, RS_ERR_INVALID_ARG, "rs_topk_compact: null scores or keep_idx");
+    if ((x == nullptr) != (x_out == nullptr)) return fail(ctx, RS_ERR_INVALID_ARG, "rs_topk_compact: x and x_out must both be given or both be NULL");
+    const int K = N - r;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (x) {
+        if (D < 8 || (D % 8) != 0) return fail(ctx, RS_ERR_INVALID_ARG, "rs_topk_compact: D must be a positive multiple of 8");
+        if (!aligned16(x) || !aligned16(x_out)) return fail(ctx, RS_ERR_INVALID_ARG, "rs_topk_compact: misaligned pointer");
+        const size_t sz = rs::dtype_size(dtype);
+        const char* xa = (const char*)x;
+        const char* xo = (const char*)x_out;
+        const size_t xbytes = (size_t)B * N * D * sz, obytes = (size_t)B * K * D * sz;
+        if (xa < xo + obytes && xo < xa + xbytes) return fail(ctx, RS_ERR_INVALID_ARG, "rs_topk_compact: x_out overlaps x");
+    }
+    RS_CHECK_LAUNCH(ctx, RS_K_SELECT, st, rs::launch_select(scores, 0, nullptr, B, N, K, has_cls ? 1 : 0, keep_idx, st), "select launch");
+    if (x) RS_CHECK_LAUNCH(ctx, RS_K_GATHER, st, rs::launch_gather(dtype, x, keep_idx, B, N, K, D, x_out, st), "gather launch");
+    return RS_OK;
+}
+
+size_t rs_block_workspace_bytes(const rs_block_desc* d) {
+    BlockWs ws;
+    if (!d || !block_layout(*d, &ws)) return 0;
+    return ws.total;
+}
+
+rs_status rs_block_fwd(rs_ctx* ctx, const rs_block_desc* d, const rs_block_weights* w, const void* x,
+                       void* x_out, float* scores, int32_t* keep_idx, void* x_full, void* workspace,
+                       size_t workspace_bytes, void* stream) {
+    if (!ctx) return RS_ERR_INVALID_ARG;
+    if (!d || !w || !x || !x_out) return fail(ctx, RS_ERR_INVALID_ARG, "rs_block_fwd: null argument");
+    BlockWs ws;
+    if (!block_layout(*d, &ws)) return fail(ctx, RS_ERR_INVALID_ARG, "rs_block_fwd: bad descriptor");
+    if (d->H * 64 != d->D) return fail(ctx, RS_ERR_UNSUPPORTED, "rs_block_fwd: D must equal 64 * H");
+    if ((d->D % 8) || (d->D_mlp % 8)) return fail(ctx, RS_ERR_INVALID_ARG, "rs_block_fwd: D and D_mlp must be multiples of 8");
+    if (d->D > 2048 && d->dtype == RS_BF16) return fail(ctx, RS_ERR_UNSUPPORTED, "rs_block_fwd: D > 2048");
+    if (d->D > 1024 && d->dtype == RS_F32) return fail(ctx, RS_ERR_UNSUPPORTED, "rs_block_fwd: D > 1024 in fp32");
+    if (d->N > 32768) return fail(ctx, RS_ERR_UNSUPPORTED, "rs_block_fwd: N > 32768");
+    if (d->r < 0 || d->r > d->N - 1) return fail(ctx, RS_ERR_INVALID_ARG, "rs_block_fwd: need 0 <= r <= N-1");
+    if (d->dist != RS_DIST_L2) return fail(ctx, RS_ERR_UNSUPPORTED, "rs_block_fwd: only the L2 distance is fused into the block");
+    if (d->score_mode != RS_SCORE_MLP && d->score_mode != RS_SCORE_MLP_DELTA)
+        return fail(ctx, RS_ERR_INVALID_ARG, "rs_block_fwd: bad score_mode");
+    if (d->dtype == RS_F32 && d->out_dtype != RS_F32)
+        return fail(ctx, RS_ERR_UNSUPPORTED, "rs_block_fwd: fp32 storage writes fp32 outputs");
+    if (!w->w_qkv || !w->w_o || !w->w_fc1 || !w->w_fc2 || !w->ln1_g || !w->ln1_b || !w->ln2_g || !w->ln2_b)
+        return fail(ctx, RS_ERR_INVALID_ARG, "rs_block_fwd: null weight");
+    const void* ptrs[] = {x, x_out, x_full, workspace, w->w_qkv, w->w_o, w->w_fc1, w->w_fc2, w->b_qkv, w->b_o,
+                          w->b_fc1, w->b_fc2, w->ln1_g, w->ln1_b, w->ln2_g, w->ln2_b};
+    for (const void* p : ptrs)
+        if (p && !aligned16(p)) return fail(ctx, RS_ERR_INVALID_ARG, "rs_block_fwd: pointers must be 16-byte aligned");
+    if (!workspace || workspace_bytes < ws.total)
+        return fail(ctx, RS_ERR_WORKSPACE, "rs_block_fwd: workspace of %zu bytes needed, %zu given", ws.total, workspace_bytes);
+    if (reinterpret_cast<uintptr_t>(workspace) & 255u)
+        return fail(ctx, RS_ERR_INVALID_ARG, "rs_block_fwd: workspace must be 256-byte aligned");
+
+    cudaStream_t st = (cudaStream_t)stream;
+    char* base = (char*)workspace;
+    const long long T = (long long)d->B * d->N;
+    const int D = d->D, Dm = d->D_mlp, K = d->N - d->r;
+    const float eps = d->ln_eps > 0.f ? d->ln_eps : 1e-6f;
+    void* u = base + ws.u;
+    void* qkv = base + ws.qkv;
+    void* o = base + ws.o;
+    float* x_prime = (float*)(base + ws.x_prime);
+    void* h = base + ws.h;
+    float* m = (float*)(base + ws.m);
+    float* s = scores ? scores : (float*)(base + ws.scores);
+    int32_t* keep = keep_idx ? keep_idx : (int32_t*)(base + ws.keep);
+    // The un-pruned output goes to x_full if given, straight to x_out when nothing is
+    // dropped, else to scratch.
+    void* x_hat = x_full ? x_full : (d->r == 0 ? x_out : (void*)(base + ws.x_hat));
+
+    // x' = SA(LN(x)) + x                                                  (Eq. att)
+    RS_CHECK_LAUNCH(ctx, RS_K_LAYERNORM, st, rs::launch_layernorm(d->dtype, d->dtype, x, w->ln1_g, w->ln1_b, eps, T, D, u, st), "LN1");
+    RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_simt(d->dtype, u, w->w_qkv, w->b_qkv, 0, nullptr, RS_F32, qkv, d->dtype, T, 3 * D, D, st), "QKV");
+    rs_attn_desc ad;
+    ad.dtype = d->dtype; ad.B = d->B; ad.N = d->N; ad.H = d->H; ad.head_dim = 64; ad.scale = d->scale;
+    ad.q_batch_stride = ad.k_batch_stride = ad.v_batch_stride = (long long)d->N * 3 * D;
+    ad.q_row_stride = ad.k_row_stride = ad.v_row_stride = 3 * D;
+    ad.q_head_stride = ad.k_head_stride = ad.v_head_stride = 64;
+    const size_t sz = rs::dtype_size(d->dtype);
+    RS_CHECK_LAUNCH(ctx, RS_K_ATTN, st, rs::launch_attn_simt(ad, qkv, (char*)qkv + (size_t)D * sz, (char*)qkv + 2 * (size_t)D * sz, o, st), "attention");
+    RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_simt(d->dtype, o, w->w_o, w->b_o, 0, x, d->dtype, x_prime, RS_F32, T, D, D, st), "proj");
+    // x^ = MLP(LN(x')) + x',  s = |MLP(LN(x')) - x'|                      (Eq. MLP, Sec. 3.2)
+    RS_CHECK_LAUNCH(ctx, RS_K_LAYERNORM, st, rs::launch_layernorm(RS_F32, d->dtype, x_prime, w->ln2_g, w->ln2_b, eps, T, D, u, st), "LN2");
+    RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_simt(d->dtype, u, w->w_fc1, w->b_fc1, 1, nullptr, RS_F32, h, d->dtype, T, Dm, D, st), "FC1");
+    RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_simt(d->dtype, h, w->w_fc2, w->b_fc2, 0, nullptr, RS_F32, m, RS_F32, T, D, Dm, st), "FC2");
+    RS_CHECK_LAUNCH(ctx, RS_K_SCORE, st, rs::launch_residual_score(m, x_prime, T, D, d->score_mode, d->out_dtype, x_hat, s, st), "residual+score");
+    // reduced token set                                                   (Sec. 3.1)
+    RS_CHECK_LAUNCH(ctx, RS_K_SELECT, st, rs::launch_select(s, 0, nullptr, d->B, d->N, K, d->has_cls ? 1 : 0, keep, st), "select");
+    if (x_hat != x_out)
+        RS_CHECK_LAUNCH(ctx, RS_K_GATHER, st, rs::launch_gather(d->out_dtype, x_hat, keep, d->B, d->N, K, D, x_out, st), "gather");
+    return RS_OK;
+}
+
+}  // extern "C"

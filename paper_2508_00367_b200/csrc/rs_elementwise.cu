@@ -1,0 +1,235 @@
+// HBM-bound row kernels: LayerNorm, the representation-shift score (Sec. 3.2)
+// and the residual-add epilogue with the score fused in.  One warp owns one
+// token row; rows move as 16-byte vectors, several in flight per lane.
+#include "rs_internal.h"
+#include "rs_device.cuh"
+
+namespace rs {
+
+namespace {
+
+constexpr int kWarpsPerCta = 8;
+
+template <typename TO, int N>
+__device__ __forceinline__ void store_n(TO* p, const float* v);
+template <> __device__ __forceinline__ void store_n<float, 4>(float* p, const float* v) {
+    *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]);
+}
+template <> __device__ __forceinline__ void store_n<float, 8>(float* p, const float* v) {
+    *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]);
+    *reinterpret_cast<float4*>(p + 4) = make_float4(v[4], v[5], v[6], v[7]);
+}
+template <> __device__ __forceinline__ void store_n<__nv_bfloat16, 4>(__nv_bfloat16* p, const float* v) {
+    __nv_bfloat162 a = __floats2bfloat162_rn(v[0], v[1]);
+    __nv_bfloat162 b = __floats2bfloat162_rn(v[2], v[3]);
+    *reinterpret_cast<uint2*>(p) = make_uint2(*reinterpret_cast<uint32_t*>(&a), *reinterpret_cast<uint32_t*>(&b));
+}
+template <> __device__ __forceinline__ void store_n<__nv_bfloat16, 8>(__nv_bfloat16* p, const float* v) {
+    uint32_t w[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+        w[i] = *reinterpret_cast<uint32_t*>(&h);
+    }
+    *reinterpret_cast<uint4*>(p) = make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+// ---------------------------------------------------------------- LayerNorm
+// LN of Eq. att / Eq. MLP: mean and biased variance over D, then affine.
+template <typename TI, typename TO, int MAXV>
+__global__ void __launch_bounds__(kWarpsPerCta * 32)
+layernorm_kernel(const TI* __restrict__ x, const float* __restrict__ gamma,
+                 const float* __restrict__ beta, float eps, long long T, int D, TO* __restrict__ out) {
+    constexpr int VN = Vec16<TI>::N;
+    const int lane = threadIdx.x & 31;
+    const long long row = (long long)blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5);
+    if (row >= T) return;
+    const int nvec = D / VN;
+    const TI* xr = x + row * D;
+    Vec16<TI> v[MAXV];
+    float sum = 0.f;
+#pragma unroll
+    for (int j = 0; j < MAXV; ++j) {
+        const int iv = j * 32 + lane;
+        if (iv < nvec) {
+            v[j].load(xr + iv * VN);
+#pragma unroll
+            for (int e = 0; e < VN; ++e) sum += v[j].v[e];
+        }
+    }
+    const float mu = warp_sum(sum) / (float)D;
+    float sq = 0.f;
+#pragma unroll
+    for (int j = 0; j < MAXV; ++j) {
+        const int iv = j * 32 + lane;
+        if (iv < nvec) {
+#pragma unroll
+            for (int e = 0; e < VN; ++e) { const float d = v[j].v[e] - mu; sq += d * d; }
+        }
+    }
+    const float rstd = rsqrtf(warp_sum(sq) / (float)D + eps);
+    TO* orow = out + row * D;
+#pragma unroll
+    for (int j = 0; j < MAXV; ++j) {
+        const int iv = j * 32 + lane;
+        if (iv < nvec) {
+            float y[VN];
+#pragma unroll
+            for (int e = 0; e < VN; e += 4) {
+                const float4 g = *reinterpret_cast<const float4*>(gamma + iv * VN + e);
+                const float4 b = *reinterpret_cast<const float4*>(beta + iv * VN + e);
+                y[e + 0] = (v[j].v[e + 0] - mu) * rstd * g.x + b.x;
+                y[e + 1] = (v[j].v[e + 1] - mu) * rstd * g.y + b.y;
+                y[e + 2] = (v[j].v[e + 2] - mu) * rstd * g.z + b.z;
+                y[e + 3] = (v[j].v[e + 3] - mu) * rstd * g.w + b.w;
+            }
+            store_n<TO, VN>(orow + iv * VN, y);
+        }
+    }
+}
+
+// ---------------------------------------------------------------- shift score
+// s = D(F(x), x) per token (Sec. 3.2); DIST 0: L2, 1: L1, 2: cosine distance.
+template <typename T, int DIST>
+__global__ void __launch_bounds__(kWarpsPerCta * 32)
+shift_score_kernel(const T* __restrict__ after, const T* __restrict__ before, long long rows, int D,
+                   float* __restrict__ scores) {
+    constexpr int VN = Vec16<T>::N;
+    constexpr int UNROLL = 4;
+    const int lane = threadIdx.x & 31;
+    const long long row = (long long)blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5);
+    if (row >= rows) return;
+    const int nvec = D / VN;
+    const T* a = after + row * D;
+    const T* b = before + row * D;
+    float acc = 0.f, aa = 0.f, bb = 0.f;
+    for (int base = 0; base < nvec; base += 32 * UNROLL) {
+        Vec16<T> va[UNROLL], vb[UNROLL];
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+            const int iv = base + u * 32 + lane;
+            if (iv < nvec) { va[u].load(a + iv * VN); vb[u].load(b + iv * VN); }
+        }
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+            const int iv = base + u * 32 + lane;
+            if (iv < nvec) {
+#pragma unroll
+                for (int e = 0; e < VN; ++e) {
+                    if (DIST == 0) { const float d = va[u].v[e] - vb[u].v[e]; acc = fmaf(d, d, acc); }
+                    else if (DIST == 1) { acc += fabsf(va[u].v[e] - vb[u].v[e]); }
+                    else {
+                        acc = fmaf(va[u].v[e], vb[u].v[e], acc);
+                        aa = fmaf(va[u].v[e], va[u].v[e], aa);
+                        bb = fmaf(vb[u].v[e], vb[u].v[e], bb);
+                    }
+                }
+            }
+        }
+    }
+    acc = warp_sum(acc);
+    float s;
+    if (DIST == 0) s = sqrtf(acc);
+    else if (DIST == 1) s = acc;
+    else {
+        aa = warp_sum(aa); bb = warp_sum(bb);
+        s = 1.f - acc / fmaxf(sqrtf(aa) * sqrtf(bb), 1e-12f);
+    }
+    if (lane == 0) scores[row] = s;
+}
+
+// ---------------------------------------------------------------- residual add + score
+// x_hat = m + x' and s = |m - x'| (or |m|): the score rides on the residual-add
+// pass, which already has both operands in registers (Eq. MLP, Sec. 3.2).
+template <typename TO, int MODE>
+__global__ void __launch_bounds__(kWarpsPerCta * 32)
+residual_score_kernel(const float* __restrict__ m, const float* __restrict__ xp, long long rows, int D,
+                      TO* __restrict__ x_hat, float* __restrict__ scores) {
+    const int lane = threadIdx.x & 31;
+    const long long row = (long long)blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5);
+    if (row >= rows) return;
+    const int nvec = D / 4;
+    float acc = 0.f;
+    for (int iv = lane; iv < nvec; iv += 32) {
+        const float4 a = *reinterpret_cast<const float4*>(m + row * D + iv * 4);
+        const float4 b = *reinterpret_cast<const float4*>(xp + row * D + iv * 4);
+        const float y[4] = {a.x + b.x, a.y + b.y, a.z + b.z, a.w + b.w};
+        if (MODE == 0) {
+            float d;
+            d = a.x - b.x; acc = fmaf(d, d, acc);
+            d = a.y - b.y; acc = fmaf(d, d, acc);
+            d = a.z - b.z; acc = fmaf(d, d, acc);
+            d = a.w - b.w; acc = fmaf(d, d, acc);
+        } else {
+            acc = fmaf(a.x, a.x, acc); acc = fmaf(a.y, a.y, acc);
+            acc = fmaf(a.z, a.z, acc); acc = fmaf(a.w, a.w, acc);
+        }
+        store_n<TO, 4>(x_hat + row * D + iv * 4, y);
+    }
+    acc = warp_sum(acc);
+    if (lane == 0 && scores) scores[row] = sqrtf(acc);
+}
+
+inline unsigned row_grid(long long rows) { return (unsigned)((rows + kWarpsPerCta - 1) / kWarpsPerCta); }
+
+template <typename TI, typename TO>
+cudaError_t ln_dispatch(const void* x, const float* g, const float* b, float eps, long long T, int D,
+                        void* out, cudaStream_t st) {
+    const int nvec = D / Vec16<TI>::N;
+    const dim3 grid(row_grid(T)), block(kWarpsPerCta * 32);
+    if (nvec <= 32 * 4)
+        layernorm_kernel<TI, TO, 4><<<grid, block, 0, st>>>((const TI*)x, g, b, eps, T, D, (TO*)out);
+    else if (nvec <= 32 * 8)
+        layernorm_kernel<TI, TO, 8><<<grid, block, 0, st>>>((const TI*)x, g, b, eps, T, D, (TO*)out);
+    else
+        return cudaErrorInvalidValue;
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_layernorm(rs_dtype in_dtype, rs_dtype out_dtype, const void* x, const float* gamma,
+                             const float* beta, float eps, long long T, int D, void* out,
+                             cudaStream_t st) {
+    if (T == 0) return cudaSuccess;
+    if (in_dtype == RS_F32 && out_dtype == RS_F32) return ln_dispatch<float, float>(x, gamma, beta, eps, T, D, out, st);
+    if (in_dtype == RS_F32 && out_dtype == RS_BF16) return ln_dispatch<float, __nv_bfloat16>(x, gamma, beta, eps, T, D, out, st);
+    if (in_dtype == RS_BF16 && out_dtype == RS_BF16) return ln_dispatch<__nv_bfloat16, __nv_bfloat16>(x, gamma, beta, eps, T, D, out, st);
+    return ln_dispatch<__nv_bfloat16, float>(x, gamma, beta, eps, T, D, out, st);
+}
+
+cudaError_t launch_shift_score(rs_dtype dtype, rs_dist dist, long long T, int D, const void* after,
+                               const void* before, float* scores, cudaStream_t st) {
+    if (T == 0) return cudaSuccess;
+    const dim3 grid(row_grid(T)), block(kWarpsPerCta * 32);
+#define RS_SCORE_CASE(TT, DD)                                                                   \
+    shift_score_kernel<TT, DD><<<grid, block, 0, st>>>((const TT*)after, (const TT*)before, T, D, scores)
+    if (dtype == RS_BF16) {
+        if (dist == RS_DIST_L2) RS_SCORE_CASE(__nv_bfloat16, 0);
+        else if (dist == RS_DIST_L1) RS_SCORE_CASE(__nv_bfloat16, 1);
+        else RS_SCORE_CASE(__nv_bfloat16, 2);
+    } else {
+        if (dist == RS_DIST_L2) RS_SCORE_CASE(float, 0);
+        else if (dist == RS_DIST_L1) RS_SCORE_CASE(float, 1);
+        else RS_SCORE_CASE(float, 2);
+    }
+#undef RS_SCORE_CASE
+    return cudaGetLastError();
+}
+
+cudaError_t launch_residual_score(const float* m, const float* x_prime, long long T, int D,
+                                  rs_score_mode mode, rs_dtype out_dtype, void* x_hat, float* scores,
+                                  cudaStream_t st) {
+    if (T == 0) return cudaSuccess;
+    const dim3 grid(row_grid(T)), block(kWarpsPerCta * 32);
+    if (out_dtype == RS_BF16) {
+        if (mode == RS_SCORE_MLP) residual_score_kernel<__nv_bfloat16, 0><<<grid, block, 0, st>>>(m, x_prime, T, D, (__nv_bfloat16*)x_hat, scores);
+        else residual_score_kernel<__nv_bfloat16, 1><<<grid, block, 0, st>>>(m, x_prime, T, D, (__nv_bfloat16*)x_hat, scores);
+    } else {
+        if (mode == RS_SCORE_MLP) residual_score_kernel<float, 0><<<grid, block, 0, st>>>(m, x_prime, T, D, (float*)x_hat, scores);
+        else residual_score_kernel<float, 1><<<grid, block, 0, st>>>(m, x_prime, T, D, (float*)x_hat, scores);
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace rs

@@ -1,0 +1,67 @@
+// Internal declarations shared by the translation units of the library: the
+// context object and the host-side launchers of every kernel.
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "rs.h"
+
+struct rs_ctx {
+    int device;
+    int sm_count;
+    int use_tc;            // tcgen05 kernels enabled for bf16
+    int* d_status;         // device status word (0 = ok)
+    long long launches;    // kernels launched through this context
+    void* encode_tiled;    // cuTensorMapEncodeTiled entry point (driver API), or null
+    int timing;            // bracket launches with events
+    int n_events;          // recorded launches since the last read
+    cudaEvent_t* ev;       // 2 * kMaxTimed events, created on first enable
+    unsigned char* ev_class;
+    char err[512];
+};
+
+enum { kMaxTimed = 8192 };
+
+// Device status word values.
+enum { RS_DEV_OK = 0, RS_DEV_TIMEOUT = 1 };
+
+namespace rs {
+
+inline size_t dtype_size(rs_dtype t) { return t == RS_BF16 ? 2 : 4; }
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// ---- memory-bound kernels (rs_elementwise.cu) ----
+// LayerNorm over the last dimension: x [T, D] (in_dtype) -> out [T, D] (out_dtype); fp32 math.
+cudaError_t launch_layernorm(rs_dtype in_dtype, rs_dtype out_dtype, const void* x, const float* gamma,
+                             const float* beta, float eps, long long T, int D, void* out,
+                             cudaStream_t st);
+// s[t] = D(after[t,:], before[t,:]).
+cudaError_t launch_shift_score(rs_dtype dtype, rs_dist dist, long long T, int D, const void* after,
+                               const void* before, float* scores, cudaStream_t st);
+// Residual-add epilogue with the score fused in: x_hat = m + x_prime (out_dtype);
+// s = |m - x_prime| (mode MLP) or |m| (mode MLP_DELTA).  m, x_prime fp32.
+cudaError_t launch_residual_score(const float* m, const float* x_prime, long long T, int D,
+                                  rs_score_mode mode, rs_dtype out_dtype, void* x_hat, float* scores,
+                                  cudaStream_t st);
+
+// ---- selection and compaction (rs_select.cu) ----
+// scores: [B, N] fp32, or if nparts > 0 partial sums of squares [B*N, nparts] whose row
+// sum's square root is the score (then also written to scores_out when non-null).
+cudaError_t launch_select(const float* scores, int nparts, float* scores_out, int B, int N, int K,
+                          int has_cls, int32_t* keep_idx, cudaStream_t st);
+cudaError_t launch_gather(rs_dtype dtype, const void* x, const int32_t* keep_idx, int B, int N, int K,
+                          int D, void* x_out, cudaStream_t st);
+size_t select_smem_bytes(int N);
+cudaError_t select_init();   // opt in to large dynamic shared memory once per process/device
+
+// ---- SIMT contraction path (rs_simt.cu): fp32 FMA, used for RS_F32 and as a cross-check ----
+// out[M, N] = act(A[M, K] * W[N, K]^T + bias) + residual.
+cudaError_t launch_gemm_simt(rs_dtype in_dtype, const void* A, const void* W, const float* bias,
+                             int gelu, const void* residual, rs_dtype res_dtype, void* out,
+                             rs_dtype out_dtype, long long M, int N, int K, cudaStream_t st);
+cudaError_t launch_attn_simt(const rs_attn_desc& d, const void* q, const void* k, const void* v,
+                             void* out, cudaStream_t st);
+
+}  // namespace rs

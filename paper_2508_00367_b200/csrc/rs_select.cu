@@ -1,0 +1,210 @@
+// Per-sample selection of the K = N - r highest-score tokens and compaction of
+// the kept rows (Sec. 3.1 reduced token set; Sec. 3.2 "dropped the tokens
+// having the lowest k scores").
+//
+// Selection is exact and order-stable.  fp32 scores are mapped to uint32 keys
+// that sort like the floats (NaN lowest).  A 4-pass, 8-bit radix select finds
+// the key of the K-th best token; tokens above it are kept, and ties at that
+// key are resolved towards the lower index by a prefix count.  A block-wide
+// scan of the keep flags then yields the ascending index list directly, with
+// no sort.  Integer work only once the keys are formed, hence bit-exact.
+#include "rs_internal.h"
+#include "rs_device.cuh"
+
+namespace rs {
+
+namespace {
+
+constexpr int kSelThreads = 512;
+
+__device__ __forceinline__ uint32_t score_key(float s) {
+    if (s != s) return 0u;                 // NaN ranks below every number
+    if (s == 0.f) s = 0.f;                 // -0 and +0 tie
+    const uint32_t b = __float_as_uint(s);
+    return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+
+// Exclusive prefix sum over the block of one int per thread; returns the
+// exclusive prefix, writes the block total to *total.  `wsum` holds >= 32 ints.
+__device__ __forceinline__ int block_exclusive_scan(int v, int* wsum, int* total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += t;
+    }
+    if (lane == 31) wsum[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+        const int nw = blockDim.x >> 5;
+        int w = lane < nw ? wsum[lane] : 0;
+        int winc = w;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, winc, o);
+            if (lane >= o) winc += t;
+        }
+        wsum[lane] = winc - w;             // exclusive prefix of warp sums
+        if (lane == 31) *total = winc;
+    }
+    __syncthreads();
+    const int res = wsum[warp] + inc - v;
+    __syncthreads();
+    return res;
+}
+
+__global__ void __launch_bounds__(kSelThreads)
+select_kernel(const float* __restrict__ scores, int nparts, float* __restrict__ scores_out, int N,
+              int K, int has_cls, int32_t* __restrict__ keep_idx) {
+    extern __shared__ uint32_t keys[];     // [N]
+    __shared__ int hist[256];
+    __shared__ int wsum[32];
+    __shared__ int sh_bin, sh_remaining, sh_total;
+
+    const int b = blockIdx.x;
+    const int tid = threadIdx.x;
+    const int first = has_cls ? 1 : 0;     // token 0 is kept unconditionally when has_cls
+    const int want = K - first;            // tokens to choose among indices >= first
+
+    for (int i = tid; i < N; i += kSelThreads) {
+        float s;
+        if (nparts > 0) {                  // fixed-order sum of the per-tile partial sums of squares
+            const float* p = scores + ((long long)b * N + i) * nparts;
+            float acc = 0.f;
+            for (int j = 0; j < nparts; ++j) acc += p[j];
+            s = sqrtf(acc);
+            if (scores_out) scores_out[(long long)b * N + i] = s;
+        } else {
+            s = scores[(long long)b * N + i];
+        }
+        keys[i] = score_key(s);
+    }
+    __syncthreads();
+
+    // ---- radix select: key of the want-th largest among [first, N) ----
+    uint32_t prefix = 0, mask = 0;
+    int remaining = want;                  // still to be taken from the candidates matching prefix
+    if (want > 0) {
+        for (int shift = 24; shift >= 0; shift -= 8) {
+            if (tid < 256) hist[tid] = 0;
+            __syncthreads();
+            for (int i = first + tid; i < N; i += kSelThreads) {
+                const uint32_t k = keys[i];
+                if ((k & mask) == prefix) atomicAdd(&hist[(k >> shift) & 255u], 1);
+            }
+            __syncthreads();
+            if (tid < 32) {                // warp 0: walk the bins from the top
+                int above = 0, bin = -1, rem_out = 0;
+                for (int base = 224; base >= 0 && bin < 0; base -= 32) {
+                    const int d = base + 31 - tid;          // lane 0 holds the highest bin
+                    const int c = hist[d];
+                    int inc = c;
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) {
+                        const int t = __shfl_up_sync(0xffffffffu, inc, o);
+                        if (tid >= o) inc += t;
+                    }
+                    const int cum = above + inc;            // tokens in bins >= d
+                    const bool hit = (cum >= remaining) && (cum - c < remaining);
+                    const unsigned m = __ballot_sync(0xffffffffu, hit);
+                    if (m) {
+                        const int src = __ffs(m) - 1;
+                        bin = __shfl_sync(0xffffffffu, d, src);
+                        rem_out = remaining - __shfl_sync(0xffffffffu, cum - c, src);
+                    }
+                    above = __shfl_sync(0xffffffffu, cum, 31);
+                }
+                if (tid == 0) { sh_bin = bin; sh_remaining = rem_out; }
+            }
+            __syncthreads();
+            prefix |= ((uint32_t)sh_bin) << shift;
+            mask |= 255u << shift;
+            remaining = sh_remaining;
+            __syncthreads();
+        }
+    }
+    const uint32_t thr = prefix;           // key of the last token that makes the cut
+    // `remaining` tokens with key == thr are kept, lowest indices first.
+
+    // ---- flags and scans over contiguous per-thread chunks ----
+    const int chunk = (N + kSelThreads - 1) / kSelThreads;
+    const int lo = min(tid * chunk, N), hi = min(lo + chunk, N);
+    int eq_cnt = 0;
+    if (want > 0)
+        for (int i = max(lo, first); i < hi; ++i) eq_cnt += (keys[i] == thr);
+    int eq_rank = block_exclusive_scan(eq_cnt, wsum, &sh_total);
+    int kept = 0;
+    for (int i = lo; i < hi; ++i) {
+        bool keep;
+        if (i < first) keep = true;
+        else if (want <= 0) keep = false;
+        else {
+            const uint32_t k = keys[i];
+            keep = k > thr;
+            if (k == thr) { keep = eq_rank < remaining; ++eq_rank; }
+        }
+        keys[i] = keep ? 1u : 0u;          // the chunk is private to this thread
+        kept += keep;
+    }
+    int pos = block_exclusive_scan(kept, wsum, &sh_total);
+    int32_t* out = keep_idx + (long long)b * K;
+    for (int i = lo; i < hi; ++i)
+        if (keys[i]) { if (pos < K) out[pos] = i; ++pos; }
+}
+
+// x_out[b, j, :] = x[b, keep_idx[b, j], :]; one warp per kept row, 16-byte vectors,
+// all loads of a row issued before the first store.
+template <int MAXV>
+__global__ void __launch_bounds__(256)
+gather_kernel(const uint4* __restrict__ x, const int32_t* __restrict__ keep_idx, long long rows, int N,
+              int K, int row_vecs, uint4* __restrict__ x_out) {
+    const int lane = threadIdx.x & 31;
+    const long long row = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (row >= rows) return;
+    const long long b = row / K;
+    const int src = keep_idx[row];
+    const uint4* s = x + (b * N + src) * row_vecs;
+    uint4* d = x_out + row * row_vecs;
+    for (int base = 0; base < row_vecs; base += 32 * MAXV) {
+        uint4 v[MAXV];
+#pragma unroll
+        for (int j = 0; j < MAXV; ++j) {
+            const int iv = base + j * 32 + lane;
+            if (iv < row_vecs) v[j] = __ldg(s + iv);
+        }
+#pragma unroll
+        for (int j = 0; j < MAXV; ++j) {
+            const int iv = base + j * 32 + lane;
+            if (iv < row_vecs) d[iv] = v[j];
+        }
+    }
+}
+
+}  // namespace
+
+size_t select_smem_bytes(int N) { return (size_t)N * sizeof(uint32_t); }
+
+cudaError_t select_init() {
+    return cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 32768 * 4);
+}
+
+cudaError_t launch_select(const float* scores, int nparts, float* scores_out, int B, int N, int K,
+                          int has_cls, int32_t* keep_idx, cudaStream_t st) {
+    if (B == 0) return cudaSuccess;
+    select_kernel<<<B, kSelThreads, select_smem_bytes(N), st>>>(scores, nparts, scores_out, N, K, has_cls,
+                                                               keep_idx);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_gather(rs_dtype dtype, const void* x, const int32_t* keep_idx, int B, int N, int K,
+                          int D, void* x_out, cudaStream_t st) {
+    const long long rows = (long long)B * K;
+    if (rows == 0) return cudaSuccess;
+    const int row_vecs = (int)((size_t)D * dtype_size(dtype) / 16);
+    const unsigned grid = (unsigned)((rows + 7) / 8);
+    gather_kernel<4><<<grid, 256, 0, st>>>((const uint4*)x, keep_idx, rows, N, K, row_vecs, (uint4*)x_out);
+    return cudaGetLastError();
+}
+
+}  // namespace rs

@@ -1,0 +1,182 @@
+"""GPU parity of the three standalone entry points (rs_shift_score,
+rs_topk_compact, rs_attn_fwd) against the CPU oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import parity
+from oracle import rs_oracle as orc
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    import paper_2508_00367_b200 as rs
+    c = rs.Context(0)
+    yield c
+    c.async_status()
+    c.close()
+
+
+def _tok(shape, dtype, seed, scale=1.0):
+    g = torch.Generator().manual_seed(seed)
+    t = torch.randn(*shape, generator=g) * scale
+    return t.to(dtype)
+
+
+DT = {"f32": torch.float32, "bf16": torch.bfloat16}
+
+
+# ------------------------------------------------------------------ rs_shift_score
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("dist", ["l2", "l1", "cos"])
+@pytest.mark.parametrize("B,N,D", [(2, 197, 384), (3, 129, 768), (1, 1, 64), (2, 17, 1024), (1, 5, 8), (1, 3, 2056)])
+def test_shift_score(ctx, dtype, dist, B, N, D):
+    a = _tok((B, N, D), DT[dtype], 1)
+    b = _tok((B, N, D), DT[dtype], 2)
+    got = ctx.shift_score(a.cuda(), b.cuda(), dist).cpu().numpy().astype(np.float64)
+    want = orc.shift_score(a.double().numpy(), b.double().numpy(), dist)
+    if dist == "cos":
+        np.testing.assert_allclose(got, want, rtol=0, atol=2e-6)
+    else:
+        np.testing.assert_allclose(got, want, rtol=2e-6, atol=0)
+
+
+def test_shift_score_identity_and_empty(ctx):
+    a = _tok((2, 33, 768), torch.bfloat16, 3).cuda()
+    assert (ctx.shift_score(a, a) == 0).all()
+    e = torch.empty(0, 7, 64, dtype=torch.float32, device="cuda")
+    assert ctx.shift_score(e, e).shape == (0, 7)
+
+
+def test_shift_score_full_size(ctx):
+    # ViT-B/16 workload, first block: B=64, N=197, D=768 bf16; oracle on sampled tokens
+    B, N, D = 64, 197, 768
+    a, b = _tok((B, N, D), torch.bfloat16, 4), _tok((B, N, D), torch.bfloat16, 5)
+    got = ctx.shift_score(a.cuda(), b.cuda()).cpu().numpy().astype(np.float64)
+    idx = np.random.default_rng(0).integers(0, B * N, size=512)
+    af, bf = a.double().numpy().reshape(-1, 1, D)[idx], b.double().numpy().reshape(-1, 1, D)[idx]
+    np.testing.assert_allclose(got.reshape(-1)[idx], orc.shift_score(af, bf)[:, 0], rtol=2e-6)
+
+
+# ------------------------------------------------------------------ rs_topk_compact
+def _scores(B, N, kind, seed):
+    rng = np.random.default_rng(seed)
+    if kind == "normal":
+        s = np.abs(rng.normal(size=(B, N)) * 5 + 20)
+    elif kind == "ties":
+        s = rng.integers(0, 5, size=(B, N)).astype(np.float64)
+    elif kind == "signed":
+        s = rng.normal(size=(B, N))
+        s[rng.random((B, N)) < 0.1] = 0.0
+        s[rng.random((B, N)) < 0.05] = -0.0
+    elif kind == "special":
+        s = rng.normal(size=(B, N))
+        m = rng.random((B, N))
+        s[m < 0.1] = np.nan
+        s[(m >= 0.1) & (m < 0.15)] = np.inf
+        s[(m >= 0.15) & (m < 0.2)] = -np.inf
+    elif kind == "equal":
+        s = np.full((B, N), 3.25)
+    return s.astype(np.float32)
+
+
+@pytest.mark.parametrize("kind", ["normal", "ties", "signed", "special", "equal"])
+@pytest.mark.parametrize("N", [1, 2, 17, 127, 128, 129, 197, 208, 257, 513, 1569, 4097])
+def test_topk_compact_bit_exact(ctx, kind, N):
+    B, D = 3, 64
+    s = _scores(B, N, kind, N)
+    x = _tok((B, N, D), torch.bfloat16, N + 1)
+    for has_cls in (True, False):
+        for r in sorted({0, 1, min(16, N - 1), max(N - 2, 0), N - 1, N // 2}):
+            if r > N - 1:
+                continue
+            xo, keep = ctx.topk_compact(torch.from_numpy(s).cuda(), x.cuda(), r, has_cls)
+            want = orc.topk(s.astype(np.float64), r, has_cls)
+            np.testing.assert_array_equal(keep.cpu().numpy(), want, err_msg=f"N={N} r={r} cls={has_cls}")
+            ref = torch.stack([x[b][torch.from_numpy(want[b]).long()] for b in range(B)])
+            assert torch.equal(xo.cpu().view(torch.int16), ref.view(torch.int16))
+
+
+@pytest.mark.parametrize("dtype,D", [("f32", 384), ("bf16", 768), ("bf16", 1024), ("f32", 8)])
+def test_topk_compact_rows(ctx, dtype, D):
+    B, N, r = 5, 197, 16
+    s = _scores(B, N, "normal", 7)
+    x = _tok((B, N, D), DT[dtype], 8)
+    xo, keep = ctx.topk_compact(torch.from_numpy(s).cuda(), x.cuda(), r, True)
+    want = orc.topk(s.astype(np.float64), r, True)
+    np.testing.assert_array_equal(keep.cpu().numpy(), want)
+    gathered = orc.gather(x.double().numpy(), want)
+    np.testing.assert_array_equal(xo.cpu().double().numpy(), gathered)
+
+
+def test_topk_compact_full_size_and_guard_bands(ctx):
+    # video workload shape: B=4, N=4097, D=1024 bf16, 25 % dropped; canaries around the outputs
+    B, N, D = 4, 4097, 1024
+    r = N // 4
+    K = N - r
+    s = _scores(B, N, "normal", 11)
+    x = _tok((B, N, D), torch.bfloat16, 12)
+    pad = 64
+    xo_buf = torch.full((B * K * D + 2 * pad,), -7.0, dtype=torch.bfloat16, device="cuda")
+    ki_buf = torch.full((B * K + 2 * pad,), -77, dtype=torch.int32, device="cuda")
+    xo = xo_buf[pad:pad + B * K * D].view(B, K, D)
+    ki = ki_buf[pad:pad + B * K].view(B, K)
+    ctx.topk_compact(torch.from_numpy(s).cuda(), x.cuda(), r, True, x_out=xo, keep_idx=ki)
+    want = orc.topk(s.astype(np.float64), r, True)
+    np.testing.assert_array_equal(ki.cpu().numpy(), want)
+    for b in (0, B - 1):
+        ref = x[b][torch.from_numpy(want[b]).long()]
+        assert torch.equal(xo[b].cpu().view(torch.int16), ref.view(torch.int16))
+    assert (xo_buf[:pad] == -7).all() and (xo_buf[-pad:] == -7).all()
+    assert (ki_buf[:pad] == -77).all() and (ki_buf[-pad:] == -77).all()
+
+
+def test_topk_indices_only_and_errors(ctx):
+    s = torch.from_numpy(_scores(2, 50, "normal", 1)).cuda()
+    _, keep = ctx.topk_compact(s, None, 10, True)
+    np.testing.assert_array_equal(keep.cpu().numpy(), orc.topk(s.cpu().double().numpy(), 10, True))
+    import paper_2508_00367_b200 as rs
+    with pytest.raises(rs.RsError):
+        ctx.topk_compact(s, None, 50, True)          # r > N-1
+    with pytest.raises(rs.RsError):
+        ctx.topk_compact(s, None, -1, True)
+    x = torch.zeros(2, 50, 12, device="cuda")        # D not a multiple of 8
+    with pytest.raises(rs.RsError):
+        ctx.topk_compact(s, x, 3, True)
+    ctx.async_status()                               # context still healthy
+
+
+# ------------------------------------------------------------------ rs_attn_fwd
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("B,N,H", [(2, 197, 6), (1, 1, 1), (1, 2, 2), (2, 17, 3), (1, 127, 2), (1, 128, 2),
+                                   (1, 129, 2), (1, 257, 2), (1, 577, 4), (1, 1099, 1)])
+def test_attn_packed_qkv(ctx, dtype, B, N, H):
+    D = H * 64
+    qkv = _tok((B, N, 3, H, 64), DT[dtype], N * 7 + H)
+    dq = qkv.cuda()
+    got = ctx.attn_fwd(dq[:, :, 0], dq[:, :, 1], dq[:, :, 2]).cpu().double().numpy()
+    f = qkv.double().numpy()
+    want = orc.attn(f[:, :, 0], f[:, :, 1], f[:, :, 2]).reshape(B, N, D)
+    parity.check_float(got, orc.round_to(want, dtype), dtype, rounded_output=True)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_attn_separate_buffers_scale_and_large_logits(ctx, dtype):
+    B, N, H = 2, 150, 2
+    q = _tok((B, N, H, 64), DT[dtype], 1, scale=3.0)
+    k = _tok((B, N, H, 64), DT[dtype], 2, scale=3.0)   # logits of order +-70: needs the max subtraction
+    v = _tok((B, N, H, 64), DT[dtype], 3)
+    got = ctx.attn_fwd(q.cuda(), k.cuda(), v.cuda(), scale=0.2).cpu().double().numpy()
+    want = orc.attn(q.double().numpy(), k.double().numpy(), v.double().numpy(), scale=0.2).reshape(B, N, H * 64)
+    parity.check_float(got, orc.round_to(want, dtype), dtype, rounded_output=True)
+
+
+def test_attn_rejects_bad_arguments(ctx):
+    import paper_2508_00367_b200 as rs
+    q = torch.zeros(1, 4, 2, 32, device="cuda")
+    with pytest.raises(rs.RsError) as e:
+        ctx.attn_fwd(q, q, q)
+    assert e.value.status == 2
+    ctx.async_status()

@@ -1,0 +1,105 @@
+"""CPU-only checks of the host side: the shared library loads and exports every
+symbol the header declares, the package's schedule tables reproduce the counts
+the paper's printed GFLOPs imply, and batch sharding across ranks (the only
+multi-GPU mode: independent samples, no exchange step) is a partition."""
+import ctypes
+import os
+import re
+import subprocess
+import sys
+
+import pytest
+import torch
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared():
+    text = open(os.path.join(ROOT, "include", "rs.h")).read()
+    return sorted(set(re.findall(r"RS_API[^;(]*?\b(rs_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_library_builds_and_exports_every_declared_symbol():
+    from paper_2508_00367_b200 import build, binding
+    lib_path = build.build()
+    lib = ctypes.CDLL(lib_path)
+    names = _declared()
+    assert len(names) >= 11
+    for n in names:
+        assert hasattr(lib, n), n
+    for n in binding.EXPORTS:
+        assert n in names
+
+
+def test_workspace_query_needs_no_gpu():
+    from paper_2508_00367_b200 import binding
+    lib = binding.load_library()
+    d = binding.BlockDesc(1, 1, 64, 197, 768, 12, 3072, 16, 1, 0.0, 0.0, 0, 0)
+    n = lib.rs_block_workspace_bytes(ctypes.byref(d))
+    T = 64 * 197
+    assert n >= T * 768 * 2 * (1 + 3 + 1) + T * 3072 * 2     # u, qkv, o, h at least
+    bad = binding.BlockDesc(7, 1, 64, 197, 768, 12, 3072, 16, 1, 0.0, 0.0, 0, 0)
+    assert lib.rs_block_workspace_bytes(ctypes.byref(bad)) == 0
+
+
+def test_workload_schedules():
+    from paper_2508_00367_b200 import synth
+    w = synth.WORKLOADS
+    assert w["vit_s_block"].tokens_per_block() == [197] and w["vit_s_block"].final_tokens() == 181
+    assert w["vit_b16"].tokens_per_block() == [197 - 16 * i for i in range(12)] and w["vit_b16"].final_tokens() == 5
+    assert w["vit_l16_384"].tokens_per_block()[-1] == 117 and w["vit_l16_384"].final_tokens() == 97
+    t = w["video_vit_b16"].tokens_per_block()
+    assert (t[0], t[3], t[6], t[9], w["video_vit_b16"].final_tokens()) == (1569, 1099, 770, 539, 539)
+    t = w["video_vit_l14"].tokens_per_block()
+    assert (t[0], t[4], t[8], t[12], t[16], t[23]) == (4097, 3073, 2305, 1729, 1297, 1297)
+
+
+def test_video_tokens_are_ar1():
+    from paper_2508_00367_b200 import synth
+    x = synth.make_tokens(4, 1 + 8 * 196, 64, "f32", frames=8, rho=0.9, seed=3)
+    fr = x[:, 1:].reshape(4, 8, 196, 64)
+    assert abs(fr.std().item() - 1.0) < 0.02
+    a, b = fr[:, :-1].flatten(), fr[:, 1:].flatten()
+    rho = torch.corrcoef(torch.stack([a, b]))[0, 1].item()
+    assert abs(rho - 0.9) < 0.01
+    # bf16 storage: values are exactly representable
+    xb = synth.make_tokens(1, 197, 64, "bf16", seed=3)
+    assert torch.equal(xb, xb.to(torch.bfloat16).float())
+
+
+def test_missing_library_fails_loudly(tmp_path, monkeypatch):
+    from paper_2508_00367_b200 import binding
+    monkeypatch.setattr(binding, "_lib", None)
+    monkeypatch.setattr(binding, "LIB_PATH", str(tmp_path / "nope.so"))
+    with pytest.raises(RuntimeError):
+        binding.load_library()
+
+
+_WORKER = r"""
+import os, sys, torch, torch.distributed as dist
+sys.path.insert(0, sys.argv[1])
+import bench
+dist.init_process_group("gloo", rank=int(os.environ["RANK"]), world_size=int(os.environ["WORLD_SIZE"]))
+rank, world = dist.get_rank(), dist.get_world_size()
+lo, hi = bench.shard_range(64, rank, world)
+mine = torch.zeros(64); mine[lo:hi] = 1
+dist.all_reduce(mine)
+assert torch.equal(mine, torch.ones(64)), mine          # every sample owned exactly once
+t = torch.tensor([10.0 + rank]); dist.all_reduce(t, op=dist.ReduceOp.MAX)
+assert t.item() == 10.0 + world - 1                      # max-over-ranks timing reduction
+val = bench.aggregate_throughput(hi - lo, t.item(), world)
+print("OK", rank, lo, hi, val)
+dist.destroy_process_group()
+"""
+
+
+def test_batch_sharding_two_ranks_gloo(tmp_path):
+    script = tmp_path / "worker.py"
+    script.write_text(_WORKER)
+    env = dict(os.environ, MASTER_ADDR="127.0.0.1", MASTER_PORT="29581", WORLD_SIZE="2")
+    procs = [subprocess.Popen([sys.executable, str(script), ROOT], env=dict(env, RANK=str(r)),
+                              stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True) for r in range(2)]
+    outs = [p.communicate(timeout=120)[0] for p in procs]
+    for p, o in zip(procs, outs):
+        assert p.returncode == 0, o
+        assert "OK" in o
