@@ -160,6 +160,40 @@ RS_API rs_status rs_block_fwd(rs_ctx* ctx, const rs_block_desc* desc /*host*/,
                        const void* x, void* x_out, float* scores, int32_t* keep_idx, void* x_full,
                        void* workspace, size_t workspace_bytes, void* stream);
 
+/* ---- rs_block_fwd_static: rs_block_fwd for callers that cannot allocate ----------------
+ * (The paper has no counterpart; this is a packaging variant of rs_block_fwd.)
+ * Some callers have no way to obtain device memory when they reach the block:
+ * code running inside a region where cudaMalloc is forbidden or would
+ * synchronise the device (a latency-critical serving loop, a plug-in that is
+ * handed only its input and output buffers, a host framework whose allocator
+ * the plug-in must not bypass).  This entry point needs no context and no
+ * workspace: its scratch is a fixed array of RS_STATIC_SCRATCH_BYTES that is
+ * part of the library image, so every GPU that loads the library holds that
+ * much memory until the process exits.  It calls no cudaMalloc / cudaFree and
+ * no allocating library routine.
+ *
+ * Arguments and results are those of rs_block_fwd (same kernels, same
+ * numbers); the caller still owns x, x_out, scores, keep_idx and x_full.
+ * err (host, optional): receives a message when the status is not RS_OK.
+ * Limits and caveats:
+ *   - rs_block_workspace_bytes(desc) must not exceed RS_STATIC_SCRATCH_BYTES,
+ *     else RS_ERR_WORKSPACE is returned and nothing is launched (a ViT-S block
+ *     of 2 x 197 tokens in fp32 needs about 7 MiB).
+ *   - The CUDA device current at the call is used.  The first call on each
+ *     device looks up the array's device address and sets a kernel attribute;
+ *     make that first call before starting any stream capture.
+ *   - All calls on a device share the one array and it keeps whatever the last
+ *     call left there.  Nothing in it has to start at zero (every call writes
+ *     what it later reads), but two calls whose kernels overlap on the GPU --
+ *     different streams, or different host threads -- race on it: serialise
+ *     them on one stream. */
+#define RS_STATIC_SCRATCH_BYTES (16u << 20)
+RS_API size_t rs_static_scratch_bytes(void);
+RS_API rs_status rs_block_fwd_static(const rs_block_desc* desc /*host*/,
+                                     const rs_block_weights* weights /*host struct of dev pointers*/,
+                                     const void* x, void* x_out, float* scores, int32_t* keep_idx,
+                                     void* x_full, void* stream, char* err /*host*/, size_t err_len);
+
 #ifdef __cplusplus
 }
 #endif

@@ -25,7 +25,8 @@ STATUS_NAMES = {0: "RS_OK", 1: "RS_ERR_INVALID_ARG", 2: "RS_ERR_UNSUPPORTED", 3:
 
 EXPORTS = ("rs_create", "rs_destroy", "rs_last_error", "rs_async_status", "rs_uses_tensor_cores",
            "rs_launch_count", "rs_attn_fwd", "rs_shift_score", "rs_topk_compact",
-           "rs_block_workspace_bytes", "rs_block_fwd", "rs_timing_enable", "rs_timing_read")
+           "rs_block_workspace_bytes", "rs_block_fwd", "rs_timing_enable", "rs_timing_read",
+           "rs_static_scratch_bytes", "rs_block_fwd_static")
 KERNEL_CLASSES = ("layernorm", "gemm", "attn", "score", "select", "gather")
 
 
@@ -99,6 +100,11 @@ def load_library() -> ctypes.CDLL:
     lib.rs_block_fwd.argtypes = [vp, ctypes.POINTER(BlockDesc), ctypes.POINTER(BlockWeights), vp, vp, vp, vp,
                                  vp, vp, ctypes.c_size_t, vp]
     lib.rs_block_fwd.restype = ci
+    lib.rs_static_scratch_bytes.argtypes = []
+    lib.rs_static_scratch_bytes.restype = ctypes.c_size_t
+    lib.rs_block_fwd_static.argtypes = [ctypes.POINTER(BlockDesc), ctypes.POINTER(BlockWeights), vp, vp, vp, vp, vp,
+                                        vp, ctypes.c_char_p, ctypes.c_size_t]
+    lib.rs_block_fwd_static.restype = ci
     _lib = lib
     return lib
 
@@ -264,6 +270,37 @@ class Context:
         if want_full:
             res["x_full"] = x_full
         return res
+
+
+def block_fwd_static(x: torch.Tensor, weights: "DeviceBlockWeights", H: int, r: int, has_cls: bool = True,
+                     out_dtype=None, score_mode: str = "mlp", want_full: bool = False):
+    """rs_block_fwd_static: the block without a context or a workspace, for callers that
+    may not allocate device memory at the point of the call.  Scratch is the library's
+    built-in array (rs_static_scratch_bytes()); larger blocks raise RsError(RS_ERR_WORKSPACE).
+    Calls sharing a device must be serialised on one stream.  The output tensors made
+    here are ordinary torch allocations -- a caller that cannot allocate passes its own
+    buffers through the C ABI directly."""
+    lib = load_library()
+    B, N, D = x.shape
+    code = _dt(x)
+    ocode = code if out_dtype is None else (RS_BF16 if out_dtype == torch.bfloat16 else RS_F32)
+    desc = BlockDesc(code, ocode, B, N, D, H, weights.D_mlp, r, int(has_cls), 0.0, 0.0, SCORE_MODE[score_mode], 0)
+    K = N - r
+    odt = _torch_dt(ocode)
+    x_out = torch.empty(B, max(K, 0), D, dtype=odt, device=x.device)
+    scores = torch.empty(B, N, dtype=torch.float32, device=x.device)
+    keep_idx = torch.empty(B, max(K, 0), dtype=torch.int32, device=x.device)
+    x_full = torch.empty(B, N, D, dtype=odt, device=x.device) if want_full else None
+    err = ctypes.create_string_buffer(512)
+    with torch.cuda.device(x.device):
+        st = lib.rs_block_fwd_static(ctypes.byref(desc), ctypes.byref(weights.struct), _ptr(x), _ptr(x_out),
+                                     _ptr(scores), _ptr(keep_idx), _ptr(x_full), _stream(x.device), err, 512)
+    if st != RS_OK:
+        raise RsError(st, err.value.decode())
+    res = dict(x_out=x_out, scores=scores, keep_idx=keep_idx)
+    if want_full:
+        res["x_full"] = x_full
+    return res
 
 
 class DeviceBlockWeights:
