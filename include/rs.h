@@ -108,6 +108,18 @@ typedef struct {
 RS_API rs_status rs_attn_fwd(rs_ctx* ctx, const rs_attn_desc* desc /*host*/, const void* q, const void* k,
                       const void* v, void* out, void* stream);
 
+/* ---- rs_linear_fwd: one projection of the block with its epilogue (Eq. sa "[Q,K,V] = xW", ----
+ * Eq. att, Eq. MLP):  out[M, N] = epilogue(A[M, K] . W[N, K]^T + bias).
+ *   RS_LIN_BIAS           out in `dtype`
+ *   RS_LIN_BIAS_GELU      exact-erf GELU, out in `dtype`
+ *   RS_LIN_BIAS_RESIDUAL  + residual[M, N] (of `dtype`), out in fp32 (the residual stream x')
+ * A, W, residual, out (dev); bias (dev, fp32, may be NULL).  With RS_BF16 and N % 128 == 0,
+ * K % 64 == 0 the tensor-core kernel runs, otherwise the fp32-FMA kernel. */
+typedef enum { RS_LIN_BIAS = 0, RS_LIN_BIAS_GELU = 1, RS_LIN_BIAS_RESIDUAL = 2 } rs_linear_epilogue;
+RS_API rs_status rs_linear_fwd(rs_ctx* ctx, rs_dtype dtype, rs_linear_epilogue epilogue, long long M, int N,
+                               int K, const void* A, const void* W, const float* bias, const void* residual,
+                               void* out, void* stream);
+
 /* ---- rs_shift_score: Sec. 3.2, s[b, i] = D(after[b, i, :], before[b, i, :]) ------------
  * after, before (dev): [B, N, D] of `dtype`; scores (dev): [B, N] fp32. */
 RS_API rs_status rs_shift_score(rs_ctx* ctx, rs_dtype dtype, rs_dist dist, int B, int N, int D,

@@ -26,7 +26,8 @@ STATUS_NAMES = {0: "RS_OK", 1: "RS_ERR_INVALID_ARG", 2: "RS_ERR_UNSUPPORTED", 3:
 EXPORTS = ("rs_create", "rs_destroy", "rs_last_error", "rs_async_status", "rs_uses_tensor_cores",
            "rs_launch_count", "rs_attn_fwd", "rs_shift_score", "rs_topk_compact",
            "rs_block_workspace_bytes", "rs_block_fwd", "rs_timing_enable", "rs_timing_read",
-           "rs_static_scratch_bytes", "rs_block_fwd_static")
+           "rs_static_scratch_bytes", "rs_block_fwd_static", "rs_linear_fwd")
+LIN_EPILOGUE = {"bias": 0, "gelu": 1, "residual": 2}
 KERNEL_CLASSES = ("layernorm", "gemm", "attn", "score", "select", "gather")
 
 
@@ -100,6 +101,8 @@ def load_library() -> ctypes.CDLL:
     lib.rs_block_fwd.argtypes = [vp, ctypes.POINTER(BlockDesc), ctypes.POINTER(BlockWeights), vp, vp, vp, vp,
                                  vp, vp, ctypes.c_size_t, vp]
     lib.rs_block_fwd.restype = ci
+    lib.rs_linear_fwd.argtypes = [vp, ci, ci, ctypes.c_longlong, ci, ci, vp, vp, vp, vp, vp, vp]
+    lib.rs_linear_fwd.restype = ci
     lib.rs_static_scratch_bytes.argtypes = []
     lib.rs_static_scratch_bytes.restype = ctypes.c_size_t
     lib.rs_block_fwd_static.argtypes = [ctypes.POINTER(BlockDesc), ctypes.POINTER(BlockWeights), vp, vp, vp, vp, vp,
@@ -198,6 +201,18 @@ class Context:
                      v.stride(0), v.stride(1), v.stride(2))
         self._check(self.lib.rs_attn_fwd(self.handle, ctypes.byref(d), _ptr(q), _ptr(k), _ptr(v), _ptr(out),
                                          _stream(q.device)))
+        return out
+
+    # ---- rs_linear_fwd ----
+    def linear_fwd(self, a: torch.Tensor, w: torch.Tensor, bias: Optional[torch.Tensor] = None,
+                   epilogue: str = "bias", residual: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """out = epilogue(a @ w.T + bias); a [M, K], w [N, K]; fp32 output for the residual epilogue."""
+        M, K = a.shape
+        N = w.shape[0]
+        assert a.is_contiguous() and w.is_contiguous() and w.shape[1] == K and w.dtype == a.dtype
+        out = torch.empty(M, N, dtype=torch.float32 if epilogue == "residual" else a.dtype, device=a.device)
+        self._check(self.lib.rs_linear_fwd(self.handle, _dt(a), LIN_EPILOGUE[epilogue], M, N, K, _ptr(a), _ptr(w),
+                                           _ptr(bias), _ptr(residual), _ptr(out), _stream(a.device)))
         return out
 
     # ---- rs_shift_score ----

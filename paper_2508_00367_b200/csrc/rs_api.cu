@@ -95,9 +95,10 @@ rs_status rs_create(rs_ctx** out, int device) {
         free(ctx);
         return RS_ERR_CUDA;
     }
+    // RS_DISABLE_TC=1 routes bf16 through the fp32-FMA kernels (cross-check of the tcgen05 path).
     const char* no_tc = getenv("RS_DISABLE_TC");
-    ctx->use_tc = 0;
-    (void)no_tc;
+    ctx->encode_tiled = rs::tc_get_encode_fn();
+    ctx->use_tc = (ctx->encode_tiled != nullptr) && !(no_tc && no_tc[0] == '1');
     *out = ctx;
     return RS_OK;
 }
@@ -184,6 +185,30 @@ rs_status rs_attn_fwd(rs_ctx* ctx, const rs_attn_desc* d, const void* q, const v
         if (st[i] < 0 || (st[i] % 8) != 0) return fail(ctx, RS_ERR_INVALID_ARG, "rs_attn_fwd: strides must be non-negative multiples of 8");
     if (!(d->scale >= 0.f)) return fail(ctx, RS_ERR_INVALID_ARG, "rs_attn_fwd: scale must be >= 0");
     RS_CHECK_LAUNCH(ctx, RS_K_ATTN, (cudaStream_t)stream, rs::launch_attn_simt(*d, q, k, v, out, (cudaStream_t)stream), "attention launch");
+    return RS_OK;
+}
+
+rs_status rs_linear_fwd(rs_ctx* ctx, rs_dtype dtype, rs_linear_epilogue epi, long long M, int N, int K,
+                        const void* A, const void* W, const float* bias, const void* residual, void* out,
+                        void* stream) {
+    if (!ctx) return RS_ERR_INVALID_ARG;
+    if (!valid_dtype(dtype) || epi < RS_LIN_BIAS || epi > RS_LIN_BIAS_RESIDUAL)
+        return fail(ctx, RS_ERR_INVALID_ARG, "rs_linear_fwd: bad dtype or epilogue");
+    if (M < 0 || N < 8 || K < 8 || (N % 8) || (K % 8) || M >= (1ll << 31))
+        return fail(ctx, RS_ERR_INVALID_ARG, "rs_linear_fwd: need M >= 0 and N, K positive multiples of 8");
+    if (M == 0) return RS_OK;
+    if (!A || !W || !out || (epi == RS_LIN_BIAS_RESIDUAL && !residual))
+        return fail(ctx, RS_ERR_INVALID_ARG, "rs_linear_fwd: null pointer");
+    if (!aligned16(A) || !aligned16(W) || !aligned16(out) || !aligned16(bias) || !aligned16(residual))
+        return fail(ctx, RS_ERR_INVALID_ARG, "rs_linear_fwd: pointers must be 16-byte aligned");
+    cudaStream_t st = (cudaStream_t)stream;
+    const rs_dtype out_dtype = epi == RS_LIN_BIAS_RESIDUAL ? RS_F32 : dtype;
+    if (ctx->use_tc && dtype == RS_BF16 && rs::gemm_tc_supported(M, N, K)) {
+        const int e = epi == RS_LIN_BIAS ? rs::RS_EPI_BIAS : epi == RS_LIN_BIAS_GELU ? rs::RS_EPI_BIAS_GELU : rs::RS_EPI_RESID;
+        RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_tc(ctx, e, A, W, bias, residual, out, out_dtype, nullptr, 0, M, N, K, st), "tensor-core GEMM");
+    } else {
+        RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_simt(dtype, A, W, bias, epi == RS_LIN_BIAS_GELU, epi == RS_LIN_BIAS_RESIDUAL ? residual : nullptr, dtype, out, out_dtype, M, N, K, st), "GEMM");
+    }
     return RS_OK;
 }
 
@@ -280,24 +305,48 @@ rs_status rs_block_fwd(rs_ctx* ctx, const rs_block_desc* d, const rs_block_weigh
     // dropped, else to scratch.
     void* x_hat = x_full ? x_full : (d->r == 0 ? x_out : (void*)(base + ws.x_hat));
 
-    // x' = SA(LN(x)) + x                                                  (Eq. att)
-    RS_CHECK_LAUNCH(ctx, RS_K_LAYERNORM, st, rs::launch_layernorm(d->dtype, d->dtype, x, w->ln1_g, w->ln1_b, eps, T, D, u, st), "LN1");
-    RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_simt(d->dtype, u, w->w_qkv, w->b_qkv, 0, nullptr, RS_F32, qkv, d->dtype, T, 3 * D, D, st), "QKV");
+    const bool tc = ctx->use_tc && d->dtype == RS_BF16 && rs::gemm_tc_supported(T, 3 * D, D) &&
+                    rs::gemm_tc_supported(T, D, D) && rs::gemm_tc_supported(T, Dm, D) &&
+                    rs::gemm_tc_supported(T, D, Dm);
+    const size_t sz = rs::dtype_size(d->dtype);
     rs_attn_desc ad;
     ad.dtype = d->dtype; ad.B = d->B; ad.N = d->N; ad.H = d->H; ad.head_dim = 64; ad.scale = d->scale;
     ad.q_batch_stride = ad.k_batch_stride = ad.v_batch_stride = (long long)d->N * 3 * D;
     ad.q_row_stride = ad.k_row_stride = ad.v_row_stride = 3 * D;
     ad.q_head_stride = ad.k_head_stride = ad.v_head_stride = 64;
-    const size_t sz = rs::dtype_size(d->dtype);
-    RS_CHECK_LAUNCH(ctx, RS_K_ATTN, st, rs::launch_attn_simt(ad, qkv, (char*)qkv + (size_t)D * sz, (char*)qkv + 2 * (size_t)D * sz, o, st), "attention");
-    RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_simt(d->dtype, o, w->w_o, w->b_o, 0, x, d->dtype, x_prime, RS_F32, T, D, D, st), "proj");
+    const void* kp = (char*)qkv + (size_t)D * sz;
+    const void* vp = (char*)qkv + 2 * (size_t)D * sz;
+    int nparts = 0;
+
+    // x' = SA(LN(x)) + x                                                  (Eq. att)
+    RS_CHECK_LAUNCH(ctx, RS_K_LAYERNORM, st, rs::launch_layernorm(d->dtype, d->dtype, x, w->ln1_g, w->ln1_b, eps, T, D, u, st), "LN1");
+    if (tc) {
+        RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_tc(ctx, rs::RS_EPI_BIAS, u, w->w_qkv, w->b_qkv, nullptr, qkv, RS_BF16, nullptr, 0, T, 3 * D, D, st), "QKV");
+        RS_CHECK_LAUNCH(ctx, RS_K_ATTN, st, rs::launch_attn_simt(ad, qkv, kp, vp, o, st), "attention");
+        RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_tc(ctx, rs::RS_EPI_RESID, o, w->w_o, w->b_o, x, x_prime, RS_F32, nullptr, 0, T, D, D, st), "proj");
+    } else {
+        RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_simt(d->dtype, u, w->w_qkv, w->b_qkv, 0, nullptr, RS_F32, qkv, d->dtype, T, 3 * D, D, st), "QKV");
+        RS_CHECK_LAUNCH(ctx, RS_K_ATTN, st, rs::launch_attn_simt(ad, qkv, kp, vp, o, st), "attention");
+        RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_simt(d->dtype, o, w->w_o, w->b_o, 0, x, d->dtype, x_prime, RS_F32, T, D, D, st), "proj");
+    }
     // x^ = MLP(LN(x')) + x',  s = |MLP(LN(x')) - x'|                      (Eq. MLP, Sec. 3.2)
     RS_CHECK_LAUNCH(ctx, RS_K_LAYERNORM, st, rs::launch_layernorm(RS_F32, d->dtype, x_prime, w->ln2_g, w->ln2_b, eps, T, D, u, st), "LN2");
-    RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_simt(d->dtype, u, w->w_fc1, w->b_fc1, 1, nullptr, RS_F32, h, d->dtype, T, Dm, D, st), "FC1");
-    RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_simt(d->dtype, h, w->w_fc2, w->b_fc2, 0, nullptr, RS_F32, m, RS_F32, T, D, Dm, st), "FC2");
-    RS_CHECK_LAUNCH(ctx, RS_K_SCORE, st, rs::launch_residual_score(m, x_prime, T, D, d->score_mode, d->out_dtype, x_hat, s, st), "residual+score");
+    if (tc) {
+        // The FC2 epilogue adds the residual and leaves per-tile partial sums of squares of the
+        // shift in `m`; the selection kernel adds them up in a fixed order.
+        nparts = rs::gemm_tc_score_parts(D);
+        RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_tc(ctx, rs::RS_EPI_BIAS_GELU, u, w->w_fc1, w->b_fc1, nullptr, h, RS_BF16, nullptr, 0, T, Dm, D, st), "FC1");
+        RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_tc(ctx, rs::RS_EPI_SCORE, h, w->w_fc2, w->b_fc2, x_prime, x_hat, d->out_dtype, m, d->score_mode == RS_SCORE_MLP_DELTA, T, D, Dm, st), "FC2+residual+score");
+    } else {
+        RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_simt(d->dtype, u, w->w_fc1, w->b_fc1, 1, nullptr, RS_F32, h, d->dtype, T, Dm, D, st), "FC1");
+        RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_simt(d->dtype, h, w->w_fc2, w->b_fc2, 0, nullptr, RS_F32, m, RS_F32, T, D, Dm, st), "FC2");
+        RS_CHECK_LAUNCH(ctx, RS_K_SCORE, st, rs::launch_residual_score(m, x_prime, T, D, d->score_mode, d->out_dtype, x_hat, s, st), "residual+score");
+    }
     // reduced token set                                                   (Sec. 3.1)
-    RS_CHECK_LAUNCH(ctx, RS_K_SELECT, st, rs::launch_select(s, 0, nullptr, d->B, d->N, K, d->has_cls ? 1 : 0, keep, st), "select");
+    if (nparts > 0)
+        RS_CHECK_LAUNCH(ctx, RS_K_SELECT, st, rs::launch_select(m, nparts, s, d->B, d->N, K, d->has_cls ? 1 : 0, keep, st), "select");
+    else
+        RS_CHECK_LAUNCH(ctx, RS_K_SELECT, st, rs::launch_select(s, 0, nullptr, d->B, d->N, K, d->has_cls ? 1 : 0, keep, st), "select");
     if (x_hat != x_out)
         RS_CHECK_LAUNCH(ctx, RS_K_GATHER, st, rs::launch_gather(d->out_dtype, x_hat, keep, d->B, d->N, K, D, x_out, st), "gather");
     return RS_OK;

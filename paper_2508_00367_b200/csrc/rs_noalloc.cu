@@ -6,6 +6,7 @@
 // cudaGetSymbolAddress, looked up once per device.
 #include <mutex>
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include "rs_internal.h"
@@ -15,11 +16,16 @@ namespace {
 // Scratch shared by every rs_block_fwd_static call on a device.  Each GPU that
 // loads the library holds these bytes until the process exits.
 static __device__ __align__(256) unsigned char rs_static_scratch[RS_STATIC_SCRATCH_BYTES];
+// Status word the tensor-core kernels write if one of their bounded waits expires.
+static __device__ __align__(256) int rs_static_status[64];
 
 constexpr int kMaxDevices = 64;
 std::mutex g_mu;
 void* g_scratch[kMaxDevices];       // device address of rs_static_scratch, per device
+int* g_status[kMaxDevices];         // device address of rs_static_status, per device
 bool g_ready[kMaxDevices];
+void* g_encode;                     // cuTensorMapEncodeTiled, looked up once (host side, no allocation)
+bool g_encode_done;
 
 void say(char* err, size_t err_len, const char* msg) {
     if (err && err_len) snprintf(err, err_len, "%s", msg);
@@ -27,15 +33,22 @@ void say(char* err, size_t err_len, const char* msg) {
 
 // First call on a device: resolve the array's device address and opt the selection
 // kernel in to its shared-memory size.  Neither call allocates.
-rs_status setup_device(int dev, void** scratch, char* err, size_t err_len) {
+rs_status setup_device(int dev, void** scratch, int** status, void** encode, char* err, size_t err_len) {
     std::lock_guard<std::mutex> lock(g_mu);
+    if (!g_encode_done) {
+        g_encode = rs::tc_get_encode_fn();
+        g_encode_done = true;
+    }
     if (!g_ready[dev]) {
         void* p = nullptr;
+        void* ps = nullptr;
         cudaError_t e = cudaGetSymbolAddress(&p, rs_static_scratch);
-        if (e != cudaSuccess || !p) {
+        if (e == cudaSuccess) e = cudaGetSymbolAddress(&ps, rs_static_status);
+        if (e != cudaSuccess || !p || !ps) {
             say(err, err_len, cudaGetErrorString(e));
             return RS_ERR_CUDA;
         }
+        g_status[dev] = (int*)ps;
         e = rs::select_init();
         if (e != cudaSuccess) {
             say(err, err_len, cudaGetErrorString(e));
@@ -45,6 +58,8 @@ rs_status setup_device(int dev, void** scratch, char* err, size_t err_len) {
         g_ready[dev] = true;
     }
     *scratch = g_scratch[dev];
+    *status = g_status[dev];
+    *encode = g_encode;
     return RS_OK;
 }
 
@@ -81,12 +96,25 @@ rs_status rs_block_fwd_static(const rs_block_desc* desc, const rs_block_weights*
         return RS_ERR_CUDA;
     }
     void* scratch = nullptr;
-    rs_status st = setup_device(dev, &scratch, err, err_len);
+    void* encode = nullptr;
+    int* status = nullptr;
+    rs_status st = setup_device(dev, &scratch, &status, &encode, err, err_len);
     if (st != RS_OK) return st;
+    int sms = 0;
+    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) {
+        say(err, err_len, cudaGetErrorString(e));
+        return RS_ERR_CUDA;
+    }
     // A context on the stack: it owns no device memory and only collects the error text.
     rs_ctx ctx;
     memset(&ctx, 0, sizeof(ctx));
     ctx.device = dev;
+    ctx.sm_count = sms;
+    ctx.d_status = status;          // same kernels as rs_block_fwd, tensor cores included
+    ctx.encode_tiled = encode;
+    const char* no_tc = getenv("RS_DISABLE_TC");
+    ctx.use_tc = (encode != nullptr) && !(no_tc && no_tc[0] == '1');
     st = rs_block_fwd(&ctx, desc, weights, x, x_out, scores, keep_idx, x_full, scratch, RS_STATIC_SCRATCH_BYTES,
                       stream);
     if (st != RS_OK) say(err, err_len, ctx.err);

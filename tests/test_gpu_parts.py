@@ -180,3 +180,29 @@ def test_attn_rejects_bad_arguments(ctx):
         ctx.attn_fwd(q, q, q)
     assert e.value.status == 2
     ctx.async_status()
+
+
+# ------------------------------------------------------------------ rs_linear_fwd
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("epilogue", ["bias", "gelu", "residual"])
+@pytest.mark.parametrize("M,N,K", [(128, 128, 64), (394, 1152, 384), (1000, 768, 3072), (64, 256, 128),
+                                   (12608, 768, 768), (77, 2304, 768), (5, 64, 64), (300, 4096, 1024)])
+def test_linear(ctx, dtype, epilogue, M, N, K):
+    if dtype == "f32" and M * N * K > 4e8:
+        pytest.skip("fp32 FMA path: small shapes only")
+    a = _tok((M, K), DT[dtype], 1)
+    w = _tok((N, K), DT[dtype], 2, scale=0.05)
+    b = _tok((N,), torch.float32, 3, scale=0.1)
+    res = _tok((M, N), DT[dtype], 4) if epilogue == "residual" else None
+    got = ctx.linear_fwd(a.cuda(), w.cuda(), b.cuda(), epilogue, None if res is None else res.cuda())
+    got = got.cpu().double().numpy()
+    rows = np.arange(M) if M <= 512 else np.unique(np.concatenate(
+        [np.arange(0, 130), np.arange(M - 130, M), np.random.default_rng(0).integers(0, M, 64)]))
+    want = orc.linear(a.double().numpy()[rows], w.double().numpy(), b.double().numpy())
+    if epilogue == "gelu":
+        want = orc.gelu(want)
+    if epilogue == "residual":
+        want = want + res.double().numpy()[rows]
+        parity.check_float(got[rows], want, dtype, rounded_output=False)
+    else:
+        parity.check_float(got[rows], orc.round_to(want, dtype), dtype, rounded_output=True)
