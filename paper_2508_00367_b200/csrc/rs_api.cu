@@ -184,7 +184,10 @@ rs_status rs_attn_fwd(rs_ctx* ctx, const rs_attn_desc* d, const void* q, const v
     for (int i = 0; i < 9; ++i)
         if (st[i] < 0 || (st[i] % 8) != 0) return fail(ctx, RS_ERR_INVALID_ARG, "rs_attn_fwd: strides must be non-negative multiples of 8");
     if (!(d->scale >= 0.f)) return fail(ctx, RS_ERR_INVALID_ARG, "rs_attn_fwd: scale must be >= 0");
-    RS_CHECK_LAUNCH(ctx, RS_K_ATTN, (cudaStream_t)stream, rs::launch_attn_simt(*d, q, k, v, out, (cudaStream_t)stream), "attention launch");
+    if (ctx->use_tc && rs::attn_tc_supported(*d))
+        RS_CHECK_LAUNCH(ctx, RS_K_ATTN, (cudaStream_t)stream, rs::launch_attn_tc(ctx, *d, q, k, v, out, (cudaStream_t)stream), "tensor-core attention launch");
+    else
+        RS_CHECK_LAUNCH(ctx, RS_K_ATTN, (cudaStream_t)stream, rs::launch_attn_simt(*d, q, k, v, out, (cudaStream_t)stream), "attention launch");
     return RS_OK;
 }
 
@@ -322,7 +325,7 @@ rs_status rs_block_fwd(rs_ctx* ctx, const rs_block_desc* d, const rs_block_weigh
     RS_CHECK_LAUNCH(ctx, RS_K_LAYERNORM, st, rs::launch_layernorm(d->dtype, d->dtype, x, w->ln1_g, w->ln1_b, eps, T, D, u, st), "LN1");
     if (tc) {
         RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_tc(ctx, rs::RS_EPI_BIAS, u, w->w_qkv, w->b_qkv, nullptr, qkv, RS_BF16, nullptr, 0, T, 3 * D, D, st), "QKV");
-        RS_CHECK_LAUNCH(ctx, RS_K_ATTN, st, rs::launch_attn_simt(ad, qkv, kp, vp, o, st), "attention");
+        RS_CHECK_LAUNCH(ctx, RS_K_ATTN, st, rs::launch_attn_tc(ctx, ad, qkv, kp, vp, o, st), "attention");
         RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_tc(ctx, rs::RS_EPI_RESID, o, w->w_o, w->b_o, x, x_prime, RS_F32, nullptr, 0, T, D, D, st), "proj");
     } else {
         RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_simt(d->dtype, u, w->w_qkv, w->b_qkv, 0, nullptr, RS_F32, qkv, d->dtype, T, 3 * D, D, st), "QKV");

@@ -151,7 +151,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         for (int tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x, ++tl) {
             const int m0 = (tile / num_n) * BM, nt = tile % num_n, n0 = nt * BN;
             const uint32_t a = tl & 1u, aph = (tl >> 1) & 1u;
-            if (!mbar_wait(&tfull[a], aph, abort_flag)) { ok = false; break; }
+            if (!__all_sync(0xffffffffu, mbar_wait(&tfull[a], aph, abort_flag))) { ok = false; break; }
             tc_fence_after();
             const int row = m0 + q * 32 + lane;
             const bool valid = row < args.M;

@@ -74,4 +74,9 @@ cudaError_t launch_gemm_tc(rs_ctx* ctx, int epi, const void* A, const void* W, c
                            const void* residual, void* out, rs_dtype out_dtype, float* partials,
                            int score_delta, long long M, int N, int K, cudaStream_t st);
 
+// ---- tcgen05 attention (rs_attn_tc.cu): bf16, head dimension 64 ----
+bool attn_tc_supported(const rs_attn_desc& d);
+cudaError_t launch_attn_tc(rs_ctx* ctx, const rs_attn_desc& d, const void* q, const void* k, const void* v,
+                           void* out, cudaStream_t st);
+
 }  // namespace rs
