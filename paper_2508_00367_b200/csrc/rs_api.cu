@@ -337,7 +337,7 @@ rs_status rs_block_fwd(rs_ctx* ctx, const rs_block_desc* d, const rs_block_weigh
     if (tc) {
         // The FC2 epilogue adds the residual and leaves per-tile partial sums of squares of the
         // shift in `m`; the selection kernel adds them up in a fixed order.
-        nparts = rs::gemm_tc_score_parts(D);
+        nparts = rs::gemm_tc_score_parts(ctx, T, D);
         RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_tc(ctx, rs::RS_EPI_BIAS_GELU, u, w->w_fc1, w->b_fc1, nullptr, h, RS_BF16, nullptr, 0, T, Dm, D, st), "FC1");
         RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_tc(ctx, rs::RS_EPI_SCORE, h, w->w_fc2, w->b_fc2, x_prime, x_hat, d->out_dtype, m, d->score_mode == RS_SCORE_MLP_DELTA, T, D, Dm, st), "FC2+residual+score");
     } else {

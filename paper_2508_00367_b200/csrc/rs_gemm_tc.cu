@@ -1,8 +1,14 @@
 // bf16 GEMM on the 5th-generation tensor cores with the block's epilogues fused in:
 //     out[M, N] = epilogue(A[M, K] . W[N, K]^T)
-// A and W are K-major; TMA (128-byte swizzle) feeds a shared-memory ring, one thread
-// issues tcgen05.mma into a double-buffered fp32 accumulator in tensor memory, and eight
-// epilogue warps drain it with tcgen05.ld while the next tile's main loop runs.
+// A and W are K-major.  Two CTAs on neighbouring SMs form a pair (a cluster of two) that owns
+// a 256 x BN output tile: each CTA loads its own 128 rows of A and BN/2 rows of W by TMA
+// (128-byte swizzle, no multicast) into a shared-memory ring, and one thread of the pair's
+// leader issues tcgen05.mma.cta_group::2, which reads both CTAs' shared memory and accumulates
+// each CTA's 128 x BN half in that CTA's tensor memory.  Per byte moved from L2 to the SMs the
+// pair tile does twice the arithmetic of a 128 x 128 tile, which is what lifts the kernel off
+// the L2 -> SM bandwidth bound.  The fp32 accumulator is double-buffered in tensor memory, so
+// the eight epilogue warps of each CTA drain tile i (tcgen05.ld -> bias / GELU / residual /
+// score -> swizzled shared memory -> TMA store) while the main loop of tile i+1 runs.
 //
 // Epilogues (Eq. att, Eq. MLP, Sec. 3.2):
 //   EPI_BIAS       out = acc + b                          -> bf16      (QKV projection)
@@ -21,31 +27,50 @@ using namespace tc;
 
 enum { EPI_BIAS = 0, EPI_BIAS_GELU = 1, EPI_RESID = 2, EPI_SCORE = 3 };
 
-constexpr int BM = 128, BK = 64;
-constexpr int kThreads = 320;                 // warp 0: TMA, warp 1: MMA, warps 2-9: epilogue
+constexpr int BM = 128;                       // rows per CTA; the pair's tile has 2 * BM rows
+constexpr int BK = 64;
+constexpr int kThreads = 320;                 // warp 0: TMA, warp 1: MMA (leader CTA), warps 2-9: epilogue
 constexpr int kEpiWarps = 8;
 constexpr int A_BYTES = BM * BK * 2;          // 16 KB
+constexpr int STG_BYTES = 128 * 128;          // one staged output block: 128 rows of 128 bytes
+constexpr int kStgBufs = 4;                   // two per column half
 
 template <int BN> struct Cfg {
-    static constexpr int B_BYTES = BN * BK * 2;
-    static constexpr int STAGES = (BN == 128) ? 6 : 4;
+    static constexpr int B_BYTES = (BN / 2) * BK * 2;              // this CTA's half of the W tile
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    static constexpr int TMEM_COLS = 2 * BN;
-    static constexpr size_t SMEM = (size_t)STAGES * STAGE_BYTES + 1024 /*align slack*/ + 256 /*barriers*/;
+    static constexpr int STAGES = (BN == 128) ? 6 : 5;
+    static constexpr int TMEM_COLS = (BN == 128) ? 256 : 512;      // two accumulators, a power of two
+    static constexpr int SPLIT = (BN == 128) ? 64 : 128;           // epilogue warps 2-5 take columns [0, SPLIT)
+    static constexpr int OFF_STG = STAGES * STAGE_BYTES;
+    static constexpr int OFF_BAR = OFF_STG + kStgBufs * STG_BYTES;
+    static constexpr size_t SMEM = (size_t)OFF_BAR + 256 /*barriers*/ + 1024 /*align slack*/;
 };
 
 struct GemmArgs {
     int M, N, K;
     const float* bias;        // [N] or null
     const void* residual;     // EPI_RESID: bf16 [M, N];  EPI_SCORE: fp32 [M, N]
-    void* out;                // [M, N]
     float* partials;          // EPI_SCORE: [M, 2 * N / BN] sums of squares
     int score_delta;          // EPI_SCORE: 1 => sum m^2 instead of (m - x')^2
     int* status;
 };
 
+// Exact-erf GELU, v * Phi(v), to fp32 accuracy (max abs error 8e-7 over all v) without erff:
+// with q(t) = -log2(Phi(-t)) for t >= 0,  Phi(v) = 2^-q(|v|) for v < 0 and 1 - 2^-q(|v|) for
+// v >= 0.  q is smooth (about t^2/2 * log2(e) plus slow terms) and a degree-5 polynomial fitted
+// on [0, 7] with weight t * Phi(-t) reproduces GELU to that accuracy; its positive leading
+// coefficient keeps 2^-q -> 0 for large |v|.  Coefficients from csrc/fit_gelu.py.
 __device__ __forceinline__ float gelu_erf(float v) {
-    return 0.5f * v * (1.f + erff(v * 0.70710678118654752f));
+    const float a = fabsf(v);
+    float q = 0.00047694556997157633f;
+    q = fmaf(q, a, -0.00711308466270566f);
+    q = fmaf(q, a, 0.05190887302160263f);
+    q = fmaf(q, a, 0.4598882496356964f);
+    q = fmaf(q, a, 1.1508461236953735f);
+    q = fmaf(q, a, 1.0000265836715698f);
+    float e;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(-q));
+    return v * (v >= 0.f ? 1.f - e : e);
 }
 
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
@@ -56,71 +81,81 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
 template <int BN, int EPI, typename OutT>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-               const GemmArgs args) {
+               const __grid_constant__ CUtensorMap tmOut, const GemmArgs args) {
     using C = Cfg<BN>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)C::STAGES * C::STAGE_BYTES);
-    uint64_t* full = bars;                       // [STAGES]
-    uint64_t* empty = bars + C::STAGES;          // [STAGES]
-    uint64_t* tfull = bars + 2 * C::STAGES;      // [2]
-    uint64_t* tempty = bars + 2 * C::STAGES + 2; // [2]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::OFF_BAR);
+    uint64_t* full = bars;                       // [STAGES] leader's: both CTAs' operands landed
+    uint64_t* empty = bars + C::STAGES;          // [STAGES] per CTA: the MMAs reading the stage retired
+    uint64_t* tfull = bars + 2 * C::STAGES;      // [2] per CTA: accumulator complete
+    uint64_t* tempty = bars + 2 * C::STAGES + 2; // [2] leader's: both CTAs' epilogues drained it
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * C::STAGES + 4);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    volatile int* half_fail = reinterpret_cast<volatile int*>(tmem_slot + 2);   // [2]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int num_m = (args.M + BM - 1) / BM, num_n = args.N / BN;
+    const uint32_t rank = cluster_ctarank();     // 0 = leader of the pair
+    const int num_m = (args.M + 2 * BM - 1) / (2 * BM), num_n = args.N / BN;
     const int tiles = num_m * num_n, kblocks = args.K / BK;
+    const int pair = (int)cluster_id_x(), npairs = (int)cluster_count_x();
 
     if (threadIdx.x == 0) {
         prefetch_tmap(&tmA);
         prefetch_tmap(&tmB);
+        prefetch_tmap(&tmOut);
         for (int s = 0; s < C::STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-        for (int a = 0; a < 2; ++a) { mbar_init(&tfull[a], 1); mbar_init(&tempty[a], kEpiWarps); }
+        for (int a = 0; a < 2; ++a) { mbar_init(&tfull[a], 1); mbar_init(&tempty[a], 2 * kEpiWarps); }
         *abort_flag = 0;
+        half_fail[0] = 0;
+        half_fail[1] = 0;
         mbar_fence_init();
     }
     if (warp == 1) {
-        tmem_alloc(tmem_slot, C::TMEM_COLS);
-        tmem_relinquish();
+        tmem_alloc_pair(tmem_slot, C::TMEM_COLS);
+        tmem_relinquish_pair();
     }
     tc_fence_before();
     __syncthreads();
+    cluster_sync();                              // the peer's barriers exist before anything signals them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
     if (warp == 0) {
-        // ---------------- TMA producer ----------------
+        // ---------------- TMA producer (both CTAs; each loads its own halves) ----------------
         if (elect_one()) {
             uint32_t it = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x) {
-                const int m0 = (tile / num_n) * BM, n0 = (tile % num_n) * BN;
+            for (int tile = pair; tile < tiles && ok; tile += npairs) {
+                const int m0 = (tile / num_n) * (2 * BM) + (int)rank * BM;
+                const int n0 = (tile % num_n) * BN + (int)rank * (BN / 2);
                 for (int kb = 0; kb < kblocks; ++kb, ++it) {
                     const int s = it % C::STAGES;
                     const uint32_t ph = (it / C::STAGES) & 1u;
                     if (!mbar_wait(&empty[s], ph ^ 1u, abort_flag)) { ok = false; break; }
                     uint8_t* sa = smem + (size_t)s * C::STAGE_BYTES;
-                    mbar_expect_tx(&full[s], C::STAGE_BYTES);
-                    tma_load_2d(sa, &tmA, &full[s], kb * BK, m0);
-                    tma_load_2d(sa + A_BYTES, &tmB, &full[s], kb * BK, n0);
+                    const uint32_t lead_full = map_to_cta(smem_u32(&full[s]), 0);
+                    if (rank == 0) mbar_expect_tx(&full[s], 2 * C::STAGE_BYTES);
+                    tma_load_2d_pair(sa, &tmA, lead_full, kb * BK, m0);
+                    tma_load_2d_pair(sa + A_BYTES, &tmB, lead_full, kb * BK, n0);
                 }
             }
-            // Copies this thread started must have landed before the CTA may exit.
+            // Every stage this thread filled must have been consumed (which implies its copies
+            // landed and the leader's commit signals reached this CTA) before the CTA may exit.
             const uint32_t issued = it;
-            for (int s = 0; s < C::STAGES; ++s) {
+            for (int s = 0; s < C::STAGES && ok; ++s) {
                 if ((uint32_t)s >= issued) break;
                 const uint32_t last = ((issued - 1 - s) / C::STAGES) * C::STAGES + s;   // last use of stage s
-                mbar_wait(&full[s], (last / C::STAGES) & 1u, abort_flag);
+                ok = mbar_wait(&empty[s], (last / C::STAGES) & 1u, abort_flag);
             }
         }
     } else if (warp == 1) {
-        // ---------------- MMA issuer ----------------
-        if (elect_one()) {
-            constexpr uint32_t idesc = idesc_bf16(BM, BN, 0, 0);
+        // ---------------- MMA issuer (leader CTA only) ----------------
+        if (rank == 0 && elect_one()) {
+            constexpr uint32_t idesc = idesc_bf16(2 * BM, BN, 0, 0);
             uint32_t it = 0, tl = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x, ++tl) {
+            for (int tile = pair; tile < tiles && ok; tile += npairs, ++tl) {
                 const uint32_t a = tl & 1u, aph = (tl >> 1) & 1u;
                 if (!mbar_wait(&tempty[a], aph ^ 1u, abort_flag)) { ok = false; break; }
                 tc_fence_after();
@@ -135,35 +170,71 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     const uint64_t db = smem_desc_sw128(sa + A_BYTES, 16, 1024);
 #pragma unroll
                     for (int k = 0; k < BK / 16; ++k)   // 32 bytes along K per MMA: +2 in the address field
-                        mma_ss(d_tmem, da + 2u * k, db + 2u * k, idesc, (kb | k) != 0);
-                    mma_commit(&empty[s]);              // frees the stage when these MMAs retire
+                        mma_ss_pair(d_tmem, da + 2u * k, db + 2u * k, idesc, (kb | k) != 0);
+                    mma_commit_pair(&empty[s], 3);      // frees the stage in both CTAs when these MMAs retire
                 }
-                if (ok) mma_commit(&tfull[a]);          // accumulator complete
+                if (ok) mma_commit_pair(&tfull[a], 3);  // accumulator complete in both CTAs
             }
         }
     } else {
-        // ---------------- epilogue ----------------
+        // ---------------- epilogue (both CTAs; each drains its own 128 x BN half) ----------------
         const int q = warp & 3;                          // TMEM lane quadrant this warp may read
-        const int half = (warp - 2) >> 2;                // which half of the tile's columns
-        constexpr int HALF_N = BN / 2;
-        uint32_t tl = 0;
-        bool ok = true;
-        for (int tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x, ++tl) {
-            const int m0 = (tile / num_n) * BM, nt = tile % num_n, n0 = nt * BN;
+        const int half = (warp - 2) >> 2;                // warps 2-5: columns [0, SPLIT), warps 6-9: the rest
+        const int c_begin = half ? C::SPLIT : 0, c_end = half ? BN : C::SPLIT;
+        constexpr int BLK_COLS = 128 / (int)sizeof(OutT);            // columns in one staged 128-byte row
+        constexpr int CHUNKS_PER_BLK = BLK_COLS / 32;                // 32-column TMEM loads per staged block
+        const int trow = q * 32 + lane;                  // row inside this CTA's half of the tile
+        const uint32_t stg_row = (uint32_t)(trow >> 3) * 1024u + (uint32_t)(trow & 7) * 128u;
+        const int r8 = trow & 7;
+        const bool storer = (q == 0 && lane == 0);       // issues this half's TMA stores
+        const uint32_t lead_tempty[2] = {map_to_cta(smem_u32(&tempty[0]), 0), map_to_cta(smem_u32(&tempty[1]), 0)};
+        uint32_t tl = 0, blk_ctr = 0;
+        constexpr int RES_VECS = EPI == EPI_RESID ? 4 : EPI == EPI_SCORE ? 8 : 1;   // 16-byte loads per 32 columns
+        for (int tile = pair; tile < tiles; tile += npairs, ++tl) {
+            const int m0 = (tile / num_n) * (2 * BM) + (int)rank * BM, nt = tile % num_n, n0 = nt * BN;
             const uint32_t a = tl & 1u, aph = (tl >> 1) & 1u;
-            if (!__all_sync(0xffffffffu, mbar_wait(&tfull[a], aph, abort_flag))) { ok = false; break; }
-            tc_fence_after();
-            const int row = m0 + q * 32 + lane;
+            const int row = m0 + trow;
             const bool valid = row < args.M;
-            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + a * BN + half * HALF_N;
+            // Residual values of 32 columns of this thread's row (zeros for rows past M).  They are
+            // fetched one chunk ahead, the first chunk before the accumulator is even complete.
+            auto load_res = [&](int c, uint4* dst) {
+                if (EPI == EPI_RESID || EPI == EPI_SCORE) {
+                    const size_t off = (size_t)row * args.N + n0 + c;
+                    const uint4* rp = EPI == EPI_RESID
+                        ? reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(args.residual) + off)
+                        : reinterpret_cast<const uint4*>(reinterpret_cast<const float*>(args.residual) + off);
+#pragma unroll
+                    for (int j = 0; j < RES_VECS; ++j) dst[j] = valid ? __ldg(rp + j) : make_uint4(0u, 0u, 0u, 0u);
+                }
+            };
+            uint4 res_next[RES_VECS];
+            load_res(c_begin, res_next);
+            // The four warps of a column half decide together whether to go on: the named
+            // barriers below have no time limit, so no warp may leave the loop alone.
+            if (!__all_sync(0xffffffffu, mbar_wait(&tfull[a], aph, abort_flag))) half_fail[half] = 1;
+            named_barrier(1 + half, 128);
+            if (half_fail[half]) break;
+            tc_fence_after();
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + a * BN;
             float sq = 0.f;
 #pragma unroll 1
-            for (int c = 0; c < HALF_N; c += 32) {
+            for (int c = c_begin; c < c_end; c += 32) {
+                const int cb = (c / 32) % CHUNKS_PER_BLK;            // chunk inside the staged block
+                uint8_t* stg = smem + C::OFF_STG + (half * 2 + (blk_ctr & 1u)) * STG_BYTES;
+                uint4 res[RES_VECS];
+#pragma unroll
+                for (int j = 0; j < RES_VECS; ++j) res[j] = res_next[j];
+                if (c + 32 < c_end) load_res(c + 32, res_next);
                 uint32_t r[32];
                 __syncwarp();                            // tcgen05.ld is warp-collective
                 tmem_ld_32x32(taddr + c, r);
                 tmem_wait_ld();
-                const int col = n0 + half * HALF_N + c;
+                if (c + 32 >= c_end) {                   // accumulator fully read by this warp
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_cluster(lead_tempty[a]);
+                }
+                const int col = n0 + c;
                 float v[32];
 #pragma unroll
                 for (int j = 0; j < 32; j += 4) {
@@ -174,39 +245,24 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     v[j + 2] = __uint_as_float(r[j + 2]) + b.z;
                     v[j + 3] = __uint_as_float(r[j + 3]) + b.w;
                 }
-                if (!valid) continue;
-                const size_t off = (size_t)row * args.N + col;
-                if (EPI == EPI_BIAS || EPI == EPI_BIAS_GELU) {
-                    if (EPI == EPI_BIAS_GELU) {
+                if (EPI == EPI_BIAS_GELU) {
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) v[j] = gelu_erf(v[j]);
-                    }
-                    uint4* o = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(args.out) + off);
-#pragma unroll
-                    for (int j = 0; j < 4; ++j)
-                        o[j] = make_uint4(pack_bf16(v[8 * j], v[8 * j + 1]), pack_bf16(v[8 * j + 2], v[8 * j + 3]),
-                                          pack_bf16(v[8 * j + 4], v[8 * j + 5]), pack_bf16(v[8 * j + 6], v[8 * j + 7]));
+                    for (int j = 0; j < 32; ++j) v[j] = gelu_erf(v[j]);
                 } else if (EPI == EPI_RESID) {
-                    const uint4* rp = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(args.residual) + off);
-                    float4* o = reinterpret_cast<float4*>(reinterpret_cast<float*>(args.out) + off);
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
-                        const uint4 x = __ldg(rp + j);
-                        const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+                        const uint32_t w[4] = {res[j].x, res[j].y, res[j].z, res[j].w};
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
                             v[8 * j + 2 * e] += __uint_as_float(w[e] << 16);
                             v[8 * j + 2 * e + 1] += __uint_as_float(w[e] & 0xffff0000u);
                         }
-                        o[2 * j] = make_float4(v[8 * j], v[8 * j + 1], v[8 * j + 2], v[8 * j + 3]);
-                        o[2 * j + 1] = make_float4(v[8 * j + 4], v[8 * j + 5], v[8 * j + 6], v[8 * j + 7]);
                     }
-                } else {   // EPI_SCORE
-                    const float4* rp = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(args.residual) + off);
+                } else if (EPI == EPI_SCORE) {
 #pragma unroll
                     for (int j = 0; j < 8; ++j) {
-                        const float4 x = __ldg(rp + j);
-                        const float xs[4] = {x.x, x.y, x.z, x.w};
+                        const float xs[4] = {__uint_as_float(res[j].x), __uint_as_float(res[j].y),
+                                             __uint_as_float(res[j].z), __uint_as_float(res[j].w)};
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
                             const float m = v[4 * j + e];
@@ -215,32 +271,50 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                             v[4 * j + e] = m + xs[e];
                         }
                     }
-                    if (sizeof(OutT) == 4) {
-                        float4* o = reinterpret_cast<float4*>(reinterpret_cast<float*>(args.out) + off);
+                }
+                // stage the 32 values of this row: 16-byte pieces, XOR-swizzled like the TMA box
+                if (sizeof(OutT) == 2) {
 #pragma unroll
-                        for (int j = 0; j < 8; ++j) o[j] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
-                    } else {
-                        uint4* o = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(args.out) + off);
-#pragma unroll
-                        for (int j = 0; j < 4; ++j)
-                            o[j] = make_uint4(pack_bf16(v[8 * j], v[8 * j + 1]), pack_bf16(v[8 * j + 2], v[8 * j + 3]),
-                                              pack_bf16(v[8 * j + 4], v[8 * j + 5]), pack_bf16(v[8 * j + 6], v[8 * j + 7]));
+                    for (int g = 0; g < 4; ++g) {
+                        const int piece = cb * 4 + g;
+                        *reinterpret_cast<uint4*>(stg + stg_row + ((piece ^ r8) << 4)) =
+                            make_uint4(pack_bf16(v[8 * g], v[8 * g + 1]), pack_bf16(v[8 * g + 2], v[8 * g + 3]),
+                                       pack_bf16(v[8 * g + 4], v[8 * g + 5]), pack_bf16(v[8 * g + 6], v[8 * g + 7]));
                     }
+                } else {
+#pragma unroll
+                    for (int g = 0; g < 8; ++g)
+                        *reinterpret_cast<float4*>(stg + stg_row + ((g ^ r8) << 4)) =
+                            make_float4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
+                }
+                if (cb == CHUNKS_PER_BLK - 1) {
+                    fence_async_smem();                  // staged data visible to the TMA engine
+                    // One barrier per block: before it the storer makes sure the previous store has
+                    // finished reading the other buffer, so after it that buffer is free for the
+                    // next block while this block's store is in flight.
+                    if (storer) tma_store_wait_read<0>();
+                    named_barrier(1 + half, 128);
+                    if (storer && m0 < args.M) {          // rows past M are dropped by the tensor map's bounds
+                        tma_store_2d(&tmOut, stg, col + 32 - BLK_COLS, m0);
+                        tma_store_commit();
+                    }
+                    ++blk_ctr;
                 }
             }
             if (EPI == EPI_SCORE && valid)
                 args.partials[(size_t)row * (2 * num_n) + 2 * nt + half] = sq;
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&tempty[a]);
         }
+        if (storer) tma_store_wait<0>();                 // all output written before the CTA exits
     }
 
+    tc_fence_before();
     __syncthreads();
     if (*abort_flag && threadIdx.x == 0) atomicExch(args.status, RS_DEV_TIMEOUT);
+    cluster_sync();                                      // neither CTA of the pair leaves while the other may signal it
     if (warp == 1) {
+        __syncwarp();
         tc_fence_after();
-        tmem_dealloc(tmem_base, C::TMEM_COLS);
+        tmem_dealloc_pair(tmem_base, C::TMEM_COLS);
     }
 }
 
@@ -248,9 +322,24 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
+// Tensor map over a row-major matrix [rows, cols] (cols contiguous) of 2- or 4-byte elements,
+// box [box_rows, 128 bytes of columns], 128-byte swizzle.
+bool make_tmap_2d(void* encode_fn, CUtensorMap* out, const void* base, int elem_bytes, uint64_t rows, uint64_t cols,
+                  uint32_t box_rows) {
+    EncodeTiledFn fn = reinterpret_cast<EncodeTiledFn>(encode_fn);
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {cols * (uint64_t)elem_bytes};
+    const cuuint32_t box[2] = {(cuuint32_t)(128 / elem_bytes), box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(out, elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
+              const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 template <int BN, int EPI, typename OutT>
-cudaError_t launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmArgs& args, int sm_count,
-                       cudaStream_t st) {
+cudaError_t launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmOut, const GemmArgs& args,
+                       int sm_count, cudaStream_t st) {
     using C = Cfg<BN>;
     static bool attr_done = false;   // per instantiation; the attribute is per function, set once
     if (!attr_done) {
@@ -259,10 +348,39 @@ cudaError_t launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, const Gem
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
-    const int tiles = ((args.M + BM - 1) / BM) * (args.N / BN);
-    const int grid = tiles < sm_count ? tiles : sm_count;
-    gemm_tc_kernel<BN, EPI, OutT><<<grid, kThreads, C::SMEM, st>>>(tmA, tmB, args);
-    return cudaGetLastError();
+    const int tiles = ((args.M + 2 * BM - 1) / (2 * BM)) * (args.N / BN);
+    const int pairs = tiles < sm_count / 2 ? tiles : sm_count / 2;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * pairs, 1, 1);
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = C::SMEM;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<BN, EPI, OutT>, tmA, tmB, tmOut, args);
+}
+
+// Tile width (256, 192 or 128 columns per pair): the one whose waves over the SM pairs cost
+// least, a wave of narrower tiles being charged a little more per column because it moves
+// more operand bytes per FLOP.
+int pick_bn(long long M, int N, int sm_count) {
+    const long long pairs = sm_count / 2, mt = (M + 2 * BM - 1) / (2 * BM);
+    const int widths[3] = {256, 192, 128};
+    const int penalty[3] = {100, 104, 112};
+    int best = 128;
+    long long best_cost = -1;
+    for (int i = 0; i < 3; ++i) {
+        if (N % widths[i]) continue;
+        const long long waves = (mt * (N / widths[i]) + pairs - 1) / pairs;
+        const long long cost = waves * widths[i] * penalty[i];
+        if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = widths[i]; }
+    }
+    return best;
 }
 
 }  // namespace
@@ -276,63 +394,42 @@ void* tc_get_encode_fn() {
     return fn;
 }
 
-// Tensor map over a row-major bf16 matrix [rows, cols] (cols contiguous), box [box_rows, 64], 128-byte swizzle.
-bool tc_make_tmap_2d(void* encode_fn, CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols,
-                     uint64_t row_stride_elems, uint32_t box_rows) {
-    EncodeTiledFn fn = reinterpret_cast<EncodeTiledFn>(encode_fn);
-    const cuuint64_t dims[2] = {cols, rows};
-    const cuuint64_t strides[1] = {row_stride_elems * 2};
-    const cuuint32_t box[2] = {64, box_rows};
-    const cuuint32_t estr[2] = {1, 1};
-    return fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 bool gemm_tc_supported(long long M, int N, int K) {
     return M >= 1 && M < (1ll << 31) && N >= 128 && (N % 128) == 0 && K >= 64 && (K % 64) == 0;
 }
 
-int gemm_tc_score_parts(int N) {   // partial sums per row written by the EPI_SCORE epilogue
-    const int bn = 128;
-    return 2 * (N / bn);
+int gemm_tc_score_parts(const rs_ctx* ctx, long long M, int N) {
+    return 2 * (N / pick_bn(M, N, ctx->sm_count));
 }
 
 cudaError_t launch_gemm_tc(rs_ctx* ctx, int epi, const void* A, const void* W, const float* bias,
                            const void* residual, void* out, rs_dtype out_dtype, float* partials, int score_delta,
                            long long M, int N, int K, cudaStream_t st) {
     if (!ctx->encode_tiled) return cudaErrorNotSupported;
-    // Tile width: the score epilogue indexes its partial sums by 128-column tiles; elsewhere pick the
-    // width with fewer, fuller waves over the SMs.
-    int bn = 128;
-    if (epi != EPI_SCORE && (N % 256) == 0) {
-        const long long mt = (M + BM - 1) / BM;
-        const long long w128 = (mt * (N / 128) + ctx->sm_count - 1) / ctx->sm_count * 128;
-        const long long w256 = (mt * (N / 256) + ctx->sm_count - 1) / ctx->sm_count * 256;
-        if (w256 <= w128) bn = 256;
-    }
-    CUtensorMap tmA, tmB;
-    if (!tc_make_tmap_2d(ctx->encode_tiled, &tmA, A, (uint64_t)M, (uint64_t)K, (uint64_t)K, BM) ||
-        !tc_make_tmap_2d(ctx->encode_tiled, &tmB, W, (uint64_t)N, (uint64_t)K, (uint64_t)K, (uint32_t)bn))
+    const int bn = pick_bn(M, N, ctx->sm_count);
+    const int out_bytes = (epi == EPI_RESID || (epi == EPI_SCORE && out_dtype == RS_F32)) ? 4 : 2;
+    CUtensorMap tmA, tmB, tmOut;
+    if (!make_tmap_2d(ctx->encode_tiled, &tmA, A, 2, (uint64_t)M, (uint64_t)K, BM) ||
+        !make_tmap_2d(ctx->encode_tiled, &tmB, W, 2, (uint64_t)N, (uint64_t)K, (uint32_t)(bn / 2)) ||
+        !make_tmap_2d(ctx->encode_tiled, &tmOut, out, out_bytes, (uint64_t)M, (uint64_t)N, BM))
         return cudaErrorInvalidValue;
     GemmArgs args;
-    args.M = (int)M; args.N = N; args.K = K; args.bias = bias; args.residual = residual; args.out = out;
+    args.M = (int)M; args.N = N; args.K = K; args.bias = bias; args.residual = residual;
     args.partials = partials; args.score_delta = score_delta; args.status = ctx->d_status;
     const int sms = ctx->sm_count;
+#define RS_GEMM_CASE(E, T)                                                                       \
+    return bn == 256   ? launch_one<256, E, T>(tmA, tmB, tmOut, args, sms, st)                  \
+           : bn == 192 ? launch_one<192, E, T>(tmA, tmB, tmOut, args, sms, st)                  \
+                       : launch_one<128, E, T>(tmA, tmB, tmOut, args, sms, st)
     switch (epi) {
-        case EPI_BIAS:
-            return bn == 256 ? launch_one<256, EPI_BIAS, __nv_bfloat16>(tmA, tmB, args, sms, st)
-                             : launch_one<128, EPI_BIAS, __nv_bfloat16>(tmA, tmB, args, sms, st);
-        case EPI_BIAS_GELU:
-            return bn == 256 ? launch_one<256, EPI_BIAS_GELU, __nv_bfloat16>(tmA, tmB, args, sms, st)
-                             : launch_one<128, EPI_BIAS_GELU, __nv_bfloat16>(tmA, tmB, args, sms, st);
-        case EPI_RESID:
-            return bn == 256 ? launch_one<256, EPI_RESID, float>(tmA, tmB, args, sms, st)
-                             : launch_one<128, EPI_RESID, float>(tmA, tmB, args, sms, st);
+        case EPI_BIAS: RS_GEMM_CASE(EPI_BIAS, __nv_bfloat16);
+        case EPI_BIAS_GELU: RS_GEMM_CASE(EPI_BIAS_GELU, __nv_bfloat16);
+        case EPI_RESID: RS_GEMM_CASE(EPI_RESID, float);
         case EPI_SCORE:
-            return out_dtype == RS_F32 ? launch_one<128, EPI_SCORE, float>(tmA, tmB, args, sms, st)
-                                       : launch_one<128, EPI_SCORE, __nv_bfloat16>(tmA, tmB, args, sms, st);
+            if (out_dtype == RS_F32) RS_GEMM_CASE(EPI_SCORE, float);
+            RS_GEMM_CASE(EPI_SCORE, __nv_bfloat16);
     }
+#undef RS_GEMM_CASE
     return cudaErrorInvalidValue;
 }
 

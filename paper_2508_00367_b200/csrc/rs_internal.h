@@ -68,7 +68,7 @@ cudaError_t launch_attn_simt(const rs_attn_desc& d, const void* q, const void* k
 enum { RS_EPI_BIAS = 0, RS_EPI_BIAS_GELU = 1, RS_EPI_RESID = 2, RS_EPI_SCORE = 3 };
 void* tc_get_encode_fn();                       // cuTensorMapEncodeTiled via the runtime, or null
 bool gemm_tc_supported(long long M, int N, int K);
-int gemm_tc_score_parts(int N);                 // partial sums per row written by RS_EPI_SCORE
+int gemm_tc_score_parts(const rs_ctx* ctx, long long M, int N);   // partial sums per row written by RS_EPI_SCORE
 // out[M, N] = epilogue(A[M, K] . W[N, K]^T); see rs_gemm_tc.cu for the epilogues.
 cudaError_t launch_gemm_tc(rs_ctx* ctx, int epi, const void* A, const void* W, const float* bias,
                            const void* residual, void* out, rs_dtype out_dtype, float* partials,
