@@ -1,14 +1,17 @@
 // Fused attention on the tensor cores (Eq. sa): out = Softmax(Q K^T * scale) V per
 // (sample, head), head dimension 64, without ever writing the N x N matrix.
 //
-// One CTA owns 128 query rows of one (sample, head) and streams the keys/values in tiles
-// of 128 through a two-stage TMA ring.  Per tile:  S = Q K^T  (tcgen05.mma, fp32 in tensor
-// memory)  ->  four softmax warps (one row per thread) keep the running max / sum, rescale
-// the O accumulator when the max moves, and write P = exp2(S*c - m*c) as bf16 into shared
-// memory in the K-major 128-byte-swizzled operand layout  ->  O += P V  (tcgen05.mma, V
-// used as an MN-major operand straight from its TMA tile).  Two CTAs share an SM so one
-// CTA's softmax overlaps the other's MMAs.  The first 64 columns of P reuse the K tile's
-// buffer, which is dead once S has been computed.
+// One CTA owns two 128-row query tiles (A and B) of one (sample, head) and streams the
+// keys/values in tiles of 128 through a TMA ring that both query tiles share.  For each
+// query tile and key tile:  S = Q K^T (tcgen05.mma, fp32 in tensor memory)  ->  one softmax
+// warpgroup (a row per thread) reads S, keeps a running maximum and sum, and writes
+// P = exp2(S*c - m*c) as bf16 back into tensor memory over S  ->  O += P V (tcgen05.mma
+// with P as the tensor-memory A operand and the V tile as an MN-major shared-memory B
+// operand).  The MMA warp alternates between the two query tiles, so the tensor pipe works
+// on one tile's P V and next Q K^T while the other tile's exponentials run.  The running
+// maximum is only raised when a tile's maximum exceeds it by more than 2^8 (P stays below
+// 256, exact softmax is recovered by the final division), so the O accumulator is rarely
+// rescaled and the softmax warps do that themselves.
 #include <math.h>
 
 #include "rs_internal.h"
@@ -22,13 +25,16 @@ using namespace tc;
 
 constexpr int BQ = 128, BKV = 128, DH = 64;
 constexpr int TILE_BYTES = 128 * DH * 2;        // 16 KB: a [128, 64] bf16 tile
-constexpr int kThreads = 192;                   // warp 0: TMA, warp 1: MMA, warps 2-5: softmax
-constexpr int kTmemCols = 256;                  // S: columns 0..127, O: columns 128..191
-constexpr int kOCol = 128;
-// shared memory: Q | K0 | K1 | V0 | V1 | P-high | barriers
-constexpr int OFF_Q = 0, OFF_K = TILE_BYTES, OFF_V = 3 * TILE_BYTES, OFF_P1 = 5 * TILE_BYTES;
-constexpr int OFF_BAR = 6 * TILE_BYTES;
-constexpr size_t kSmem = (size_t)OFF_BAR + 128 + 1024 /*alignment slack*/;
+constexpr int NS = 4;                           // K/V ring stages
+constexpr int kThreads = 384;                   // warps 0-3 / 4-7: softmax of tile A / B, warp 8: TMA, warp 9: MMA
+constexpr int kSoftmaxRegs = 224, kOtherRegs = 56;   // per-thread register budgets after the warpgroups re-split the pool
+constexpr int kTmemCols = 512;                  // S_A 0..127, S_B 128..255, O_A 256..319, O_B 320..383
+constexpr int kOCol = 256;
+constexpr float kRescaleGap = 8.f;              // log2 units the tile maximum may exceed the running one
+// shared memory: Q_A | Q_B | K[NS] | V[NS] | barriers
+constexpr int OFF_Q = 0, OFF_K = 2 * TILE_BYTES, OFF_V = (2 + NS) * TILE_BYTES;
+constexpr int OFF_BAR = (2 + 2 * NS) * TILE_BYTES;
+constexpr size_t kSmem = (size_t)OFF_BAR + 256 + 1024 /*alignment slack*/;
 
 struct AttnArgs {
     __nv_bfloat16* out;      // [B, N, H*64]
@@ -48,37 +54,39 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
     return *reinterpret_cast<uint32_t*>(&h);
 }
 
-__global__ void __launch_bounds__(kThreads, 2)
+__device__ __forceinline__ float max3(float a, float b, float c) { return fmaxf(fmaxf(a, b), c); }
+
+__global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                const __grid_constant__ CUtensorMap tmV, const AttnArgs args) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + OFF_BAR);
-    uint64_t* bar_q = bars;            // Q tile landed
-    uint64_t* kv_full = bars + 1;      // [2] K and V tile landed
-    uint64_t* kv_empty = bars + 3;     // [2] stage free again (O += P V retired)
-    uint64_t* s_full = bars + 5;       // S tile complete in tensor memory
-    uint64_t* p_ready = bars + 6;      // P written, O rescaled, S consumed (128 arrivals)
-    uint64_t* o_done = bars + 7;       // O += P V retired
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 8);
+    uint64_t* q_full = bars;                 // Q tiles landed
+    uint64_t* k_full = bars + 1;             // [NS] K tile landed
+    uint64_t* v_full = bars + 1 + NS;        // [NS] V tile landed
+    uint64_t* kv_empty = bars + 1 + 2 * NS;  // [NS] every MMA reading the stage retired
+    uint64_t* s_full = bars + 1 + 3 * NS;    // [2] S of tile A / B complete in tensor memory
+    uint64_t* p_ready = s_full + 2;          // [2] P written (one arrival per softmax warp)
+    uint64_t* o_done = s_full + 4;           // [2] O += P V retired
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(s_full + 6);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int N = args.N;
-    const int q0 = blockIdx.x * BQ, h = blockIdx.y, b = blockIdx.z;
+    const int q0 = blockIdx.x * (2 * BQ), h = blockIdx.y, b = blockIdx.z;
     const int nkv = (N + BKV - 1) / BKV;
+    const bool has_b = q0 + BQ < N;          // the second query tile has at least one row
 
     if (threadIdx.x == 0) {
         prefetch_tmap(&tmQ); prefetch_tmap(&tmK); prefetch_tmap(&tmV);
-        mbar_init(bar_q, 1);
-        for (int s = 0; s < 2; ++s) { mbar_init(&kv_full[s], 1); mbar_init(&kv_empty[s], 1); }
-        mbar_init(s_full, 1);
-        mbar_init(p_ready, 128);
-        mbar_init(o_done, 1);
+        mbar_init(q_full, 1);
+        for (int s = 0; s < NS; ++s) { mbar_init(&k_full[s], 1); mbar_init(&v_full[s], 1); mbar_init(&kv_empty[s], 1); }
+        for (int g = 0; g < 2; ++g) { mbar_init(&s_full[g], 1); mbar_init(&p_ready[g], 4); mbar_init(&o_done[g], 1); }
         *abort_flag = 0;
         mbar_fence_init();
     }
-    if (warp == 1) {
+    if (warp == 9) {
         tmem_alloc(tmem_slot, kTmemCols);
         tmem_relinquish();
     }
@@ -86,172 +94,228 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-
-    if (warp == 0) {
+    // The third warpgroup (TMA, MMA and two idle warps) hands most of its registers to the
+    // two softmax warpgroups, which hold a whole 128-column row of S per thread.
+    if (warp >= 8) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kOtherRegs));
+    if (warp == 8) {
         // ---------------- TMA producer ----------------
         if (elect_one()) {
-            mbar_expect_tx(bar_q, TILE_BYTES);
-            tma_load_4d(smem + OFF_Q, &tmQ, bar_q, 0, h, q0, b);
+            mbar_expect_tx(q_full, has_b ? 2 * TILE_BYTES : TILE_BYTES);
+            tma_load_4d(smem + OFF_Q, &tmQ, q_full, 0, h, q0, b);
+            if (has_b) tma_load_4d(smem + OFF_Q + TILE_BYTES, &tmQ, q_full, 0, h, q0 + BQ, b);
             int issued = 0;
+            bool ok = true;
             for (int j = 0; j < nkv; ++j, ++issued) {
-                const int s = j & 1;
-                if (!mbar_wait(&kv_empty[s], ((j >> 1) & 1) ^ 1, abort_flag)) break;
-                mbar_expect_tx(&kv_full[s], 2 * TILE_BYTES);
-                tma_load_4d(smem + OFF_K + s * TILE_BYTES, &tmK, &kv_full[s], 0, h, j * BKV, b);
-                tma_load_4d(smem + OFF_V + s * TILE_BYTES, &tmV, &kv_full[s], 0, h, j * BKV, b);
+                const int s = j % NS;
+                if (!mbar_wait(&kv_empty[s], ((j / NS) & 1) ^ 1, abort_flag)) { ok = false; break; }
+                mbar_expect_tx(&k_full[s], TILE_BYTES);
+                tma_load_4d(smem + OFF_K + s * TILE_BYTES, &tmK, &k_full[s], 0, h, j * BKV, b);
+                mbar_expect_tx(&v_full[s], TILE_BYTES);
+                tma_load_4d(smem + OFF_V + s * TILE_BYTES, &tmV, &v_full[s], 0, h, j * BKV, b);
             }
             // every copy started here must have landed before the CTA exits
-            mbar_wait(bar_q, 0, abort_flag);
-            for (int s = 0; s < 2 && s < issued; ++s) {
-                const int last = ((issued - 1 - s) / 2) * 2 + s;
-                mbar_wait(&kv_full[s], (last >> 1) & 1, abort_flag);
+            if (ok) ok = mbar_wait(q_full, 0, abort_flag);
+            for (int s = 0; s < NS && s < issued && ok; ++s) {
+                const int last = ((issued - 1 - s) / NS) * NS + s;
+                ok = mbar_wait(&k_full[s], (last / NS) & 1, abort_flag) && mbar_wait(&v_full[s], (last / NS) & 1, abort_flag);
             }
         }
-    } else if (warp == 1) {
+    } else if (warp == 9) {
         // ---------------- MMA issuer ----------------
         if (elect_one()) {
-            bool ok = mbar_wait(bar_q, 0, abort_flag);
+            bool ok = mbar_wait(q_full, 0, abort_flag);
             tc_fence_after();
-            const uint32_t sq = smem_u32(smem + OFF_Q);
-            for (int j = 0; j < nkv && ok; ++j) {
-                const int s = j & 1;
+            const uint32_t idesc_o = idesc_bf16(BQ, DH, 0, 1);
+            // S_g = Q_g K_j^T : both operands K-major (head dimension contiguous)
+            auto issue_s = [&](int g, int j) {
+                const int s = j % NS;
                 const int valid = min(BKV, N - j * BKV);
-                const int n_s = (valid + 15) & ~15;           // S columns actually needed
-                const int ksteps = (valid + 15) >> 4;         // 16-key slabs of P V actually needed
-                if (!mbar_wait(&kv_full[s], (j >> 1) & 1, abort_flag)) { ok = false; break; }
-                tc_fence_after();
-                const uint32_t sk = smem_u32(smem + OFF_K + s * TILE_BYTES);
-                const uint32_t sv = smem_u32(smem + OFF_V + s * TILE_BYTES);
-                // S = Q K^T : both operands K-major (head dimension contiguous)
-                const uint32_t idesc_s = idesc_bf16(BQ, n_s, 0, 0);
-                const uint64_t dq = smem_desc_sw128(sq, 16, 1024);
-                const uint64_t dk = smem_desc_sw128(sk, 16, 1024);
+                const uint32_t idesc_s = idesc_bf16(BQ, (valid + 15) & ~15, 0, 0);
+                const uint64_t dq = smem_desc_sw128(smem_u32(smem + OFF_Q + g * TILE_BYTES), 16, 1024);
+                const uint64_t dk = smem_desc_sw128(smem_u32(smem + OFF_K + s * TILE_BYTES), 16, 1024);
 #pragma unroll
-                for (int k = 0; k < DH / 16; ++k) mma_ss(tmem_base, dq + 2u * k, dk + 2u * k, idesc_s, k != 0);
-                mma_commit(s_full);
-                // O += P V : P K-major from shared memory (first 64 keys in the K buffer, rest in P-high),
-                // V MN-major (head dimension contiguous), 16 keys = 2048 bytes per slab.
-                if (!mbar_wait(p_ready, j & 1, abort_flag)) { ok = false; break; }
+                for (int k = 0; k < DH / 16; ++k)
+                    mma_ss(tmem_base + g * BKV, dq + 2u * k, dk + 2u * k, idesc_s, k != 0);
+                mma_commit(&s_full[g]);
+            };
+            // O_g += P_g V_j : P from tensor memory (bf16 pairs, 8 columns per 16 keys), V MN-major
+            // (head dimension contiguous), 16 keys = 2048 bytes per slab.
+            auto issue_pv = [&](int g, int j) {
+                const int s = j % NS;
+                const int valid = min(BKV, N - j * BKV);
+                const int ksteps = (valid + 15) >> 4;
+                const uint32_t sv = smem_u32(smem + OFF_V + s * TILE_BYTES);
+                for (int k = 0; k < ksteps; ++k)
+                    mma_ts(tmem_base + kOCol + g * DH, tmem_base + g * BKV + 8 * k,
+                           smem_desc_sw128(sv + (uint32_t)k * 2048u, 16, 1024), idesc_o, (j | k) != 0);
+                mma_commit(&o_done[g]);
+            };
+            if (ok) ok = mbar_wait(&k_full[0], 0, abort_flag);
+            if (ok) {
                 tc_fence_after();
-                const uint32_t idesc_o = idesc_bf16(BQ, DH, 0, 1);
-                const uint32_t sp1 = smem_u32(smem + OFF_P1);
-                for (int k = 0; k < ksteps; ++k) {
-                    const uint32_t pa = (k < 4 ? sk : sp1) + (uint32_t)(k & 3) * 32u;
-                    const uint64_t dp = smem_desc_sw128(pa, 16, 1024);
-                    const uint64_t dv = smem_desc_sw128(sv + (uint32_t)k * 2048u, 16, 1024);
-                    mma_ss(tmem_base + kOCol, dp, dv, idesc_o, (j | k) != 0);
+                issue_s(0, 0);
+                if (has_b) issue_s(1, 0);
+            }
+            for (int j = 0; j < nkv && ok; ++j) {
+                const int s = j % NS;
+                const bool more = j + 1 < nkv;
+                if (!mbar_wait(&v_full[s], (j / NS) & 1, abort_flag)) { ok = false; break; }
+                if (!mbar_wait(&p_ready[0], j & 1, abort_flag)) { ok = false; break; }
+                tc_fence_after();
+                issue_pv(0, j);
+                if (more) {
+                    if (!mbar_wait(&k_full[(j + 1) % NS], ((j + 1) / NS) & 1, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    issue_s(0, j + 1);
+                }
+                if (has_b) {
+                    if (!mbar_wait(&p_ready[1], j & 1, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    issue_pv(1, j);
                 }
                 mma_commit(&kv_empty[s]);
-                mma_commit(o_done);
+                if (more && has_b) issue_s(1, j + 1);
             }
         }
+    }
     } else {
-        // ---------------- softmax / correction / epilogue: one query row per thread ----------------
-        const int q = warp & 3;
-        const int row = q0 + q * 32 + lane;
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kSoftmaxRegs));
+    if (warp < 4 || has_b) {
+        // ---------------- softmax, O rescaling and output: one query row per thread ----------------
+        const int g = warp >> 2;                         // query tile of this warpgroup
+        const int q = warp & 3;                          // tensor-memory lane quadrant of this warp
+        const int row = q0 + g * BQ + q * 32 + lane;
         const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
+        const uint32_t s_addr = lane_addr + g * BKV, o_addr = lane_addr + kOCol + g * DH;
         const float sl = args.scale_log2;
-        const int r8 = (q * 32 + lane) & 7;
-        const uint32_t row_off = (uint32_t)((q * 32 + lane) >> 3) * 1024u + (uint32_t)r8 * 128u;
-        float m_run = -INFINITY, l_run = 0.f;
+        float m_l2 = 0.f, l_run = 0.f;                   // running maximum (times scale*log2 e) and sum
         bool ok = true;
         for (int j = 0; j < nkv && ok; ++j) {
-            const int s = j & 1;
             const int valid = min(BKV, N - j * BKV);
-            const int nchunks = (valid + 31) >> 5;
-            // the warp moves as one through the collective tensor-memory loads below
-            if (!__all_sync(0xffffffffu, mbar_wait(s_full, j & 1, abort_flag))) { ok = false; break; }
+            // the warp moves as one through the collective tensor-memory accesses below
+            if (!__all_sync(0xffffffffu, mbar_wait(&s_full[g], j & 1, abort_flag))) { ok = false; break; }
             tc_fence_after();
-            // pass 1: row maximum over the valid keys
-            float mx = m_run;
-            for (int c = 0; c < nchunks; ++c) {
-                uint32_t r[32];
-                __syncwarp();
-                tmem_ld_32x32(lane_addr + c * 32, r);
-                tmem_wait_ld();
-                const int lim = valid - c * 32;
+            // All 128 columns are read even on a partial key tile: columns past the keys the MMA
+            // wrote hold old values, which the masks below never let through.
+            uint32_t r[128];
 #pragma unroll
-                for (int i = 0; i < 32; ++i) mx = fmaxf(mx, i < lim ? __uint_as_float(r[i]) : -INFINITY);
+            for (int c = 0; c < 4; ++c) tmem_ld_32x32(s_addr + c * 32, r + c * 32);
+            tmem_wait_ld();
+            // row maximum over the valid keys
+            float mx = -INFINITY;
+            if (valid == BKV) {
+                float m0 = max3(__uint_as_float(r[0]), __uint_as_float(r[1]), __uint_as_float(r[2]));
+                float m1 = max3(__uint_as_float(r[3]), __uint_as_float(r[4]), __uint_as_float(r[5]));
+#pragma unroll
+                for (int i = 6; i + 3 < 128; i += 4) {
+                    m0 = max3(m0, __uint_as_float(r[i]), __uint_as_float(r[i + 1]));
+                    m1 = max3(m1, __uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
+                }
+                mx = max3(m0, m1, fmaxf(__uint_as_float(r[126]), __uint_as_float(r[127])));
+            } else {
+#pragma unroll
+                for (int i = 0; i < 128; ++i)
+                    if (i < valid) mx = fmaxf(mx, __uint_as_float(r[i]));
             }
-            const float alpha = ex2((m_run - mx) * sl);   // 0 on the first tile (m_run = -inf)
-            const float mneg = -mx * sl;
-            l_run *= alpha;
-            m_run = mx;
-            if (j > 0) {
-                // the previous O += P V must have retired before O is rescaled and P-high is overwritten
-                if (!__all_sync(0xffffffffu, mbar_wait(o_done, (j - 1) & 1, abort_flag))) { ok = false; break; }
-                tc_fence_after();
-                if (__any_sync(0xffffffffu, alpha != 1.f)) {
+            const float mx_l2 = mx * sl;
+            if (j == 0) {
+                m_l2 = mx_l2;
+            } else {
+                const bool raise = mx_l2 > m_l2 + kRescaleGap;
+                if (__any_sync(0xffffffffu, raise)) {
+                    // O += P V of the previous key tile must have retired before O is rescaled
+                    if (!__all_sync(0xffffffffu, mbar_wait(&o_done[g], (j - 1) & 1, abort_flag))) { ok = false; break; }
+                    tc_fence_after();
+                    const float alpha = raise ? ex2(m_l2 - mx_l2) : 1.f;
+                    if (raise) m_l2 = mx_l2;
+                    l_run *= alpha;
 #pragma unroll
                     for (int c = 0; c < 2; ++c) {
-                        uint32_t r[32];
-                        tmem_ld_32x32(lane_addr + kOCol + c * 32, r);
+                        uint32_t o[32];
+                        tmem_ld_32x32(o_addr + c * 32, o);
                         tmem_wait_ld();
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
-                        tmem_st_32x32(lane_addr + kOCol + c * 32, r);
+                        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                        tmem_st_32x32(o_addr + c * 32, o);
                     }
                     tmem_wait_st();
                 }
             }
-            // pass 2: P = exp2(S*c - m*c) -> bf16 -> shared memory (K-major, 128-byte swizzle)
-            uint8_t* p_lo = smem + OFF_K + s * TILE_BYTES;
-            uint8_t* p_hi = smem + OFF_P1;
-            for (int c = 0; c < nchunks; ++c) {
-                uint32_t r[32];
-                __syncwarp();
-                tmem_ld_32x32(lane_addr + c * 32, r);
-                tmem_wait_ld();
-                const int lim = valid - c * 32;
-                uint32_t pk[16];
+            // P = exp2(S*c - m*c) -> bf16 pairs -> tensor memory, over the S columns already read
+            const float mneg = -m_l2;
+            float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
+            if (valid == BKV) {
 #pragma unroll
-                for (int i = 0; i < 32; i += 2) {
-                    const float p0 = i < lim ? ex2(fmaf(__uint_as_float(r[i]), sl, mneg)) : 0.f;
-                    const float p1 = i + 1 < lim ? ex2(fmaf(__uint_as_float(r[i + 1]), sl, mneg)) : 0.f;
-                    l_run += p0 + p1;
-                    pk[i >> 1] = pack_bf16(p0, p1);
-                }
-                uint8_t* base = (c < 2 ? p_lo : p_hi) + row_off;
+                for (int c = 0; c < 8; ++c) {
+                    uint32_t pk[8];
 #pragma unroll
-                for (int g = 0; g < 4; ++g) {                 // four 16-byte groups of 8 keys
-                    const int chunk16 = (c & 1) * 4 + g;      // position inside the 128-byte row
-                    *reinterpret_cast<uint4*>(base + ((chunk16 ^ r8) << 4)) =
-                        make_uint4(pk[4 * g], pk[4 * g + 1], pk[4 * g + 2], pk[4 * g + 3]);
+                    for (int i = 0; i < 16; i += 4) {
+                        const float p0 = ex2(fmaf(__uint_as_float(r[16 * c + i]), sl, mneg));
+                        const float p1 = ex2(fmaf(__uint_as_float(r[16 * c + i + 1]), sl, mneg));
+                        const float p2 = ex2(fmaf(__uint_as_float(r[16 * c + i + 2]), sl, mneg));
+                        const float p3 = ex2(fmaf(__uint_as_float(r[16 * c + i + 3]), sl, mneg));
+                        l0 += p0; l1 += p1; l2 += p2; l3 += p3;
+                        pk[i >> 1] = pack_bf16(p0, p1);
+                        pk[(i >> 1) + 1] = pack_bf16(p2, p3);
+                    }
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) r[8 * c + i] = pk[i];
                 }
+#pragma unroll
+                for (int c = 0; c < 4; ++c) tmem_st_32x16(s_addr + c * 16, r + c * 16);
+            } else {
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    uint32_t pk[8];
+#pragma unroll
+                    for (int i = 0; i < 16; i += 2) {
+                        const int col = 16 * c + i;
+                        const float p0 = col < valid ? ex2(fmaf(__uint_as_float(r[col]), sl, mneg)) : 0.f;
+                        const float p1 = col + 1 < valid ? ex2(fmaf(__uint_as_float(r[col + 1]), sl, mneg)) : 0.f;
+                        l0 += p0; l1 += p1;
+                        pk[i >> 1] = pack_bf16(p0, p1);
+                    }
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) r[8 * c + i] = pk[i];
+                }
+#pragma unroll
+                for (int c = 0; c < 4; ++c) tmem_st_32x16(s_addr + c * 16, r + c * 16);
             }
-            fence_async_smem();
+            l_run += (l0 + l1) + (l2 + l3);
+            tmem_wait_st();
             tc_fence_before();
-            mbar_arrive(p_ready);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&p_ready[g]);
         }
         // epilogue: O / l -> bf16 -> global
-        if (ok && __all_sync(0xffffffffu, mbar_wait(o_done, (nkv - 1) & 1, abort_flag))) {
+        if (ok && __all_sync(0xffffffffu, mbar_wait(&o_done[g], (nkv - 1) & 1, abort_flag))) {
             tc_fence_after();
             const float inv = 1.f / l_run;
             __nv_bfloat16* op = args.out + ((size_t)((size_t)b * N + row) * args.H + h) * DH;
+            uint32_t o[64];
+            tmem_ld_32x32(o_addr, o);
+            tmem_ld_32x32(o_addr + 32, o + 32);
+            tmem_wait_ld();
+            if (row < N) {
 #pragma unroll
-            for (int c = 0; c < 2; ++c) {
-                uint32_t r[32];
-                __syncwarp();
-                tmem_ld_32x32(lane_addr + kOCol + c * 32, r);
-                tmem_wait_ld();
-                if (row < N) {
+                for (int g8 = 0; g8 < 8; ++g8) {
+                    uint32_t w[4];
 #pragma unroll
-                    for (int g = 0; g < 4; ++g) {
-                        uint32_t w[4];
-#pragma unroll
-                        for (int e = 0; e < 4; ++e)
-                            w[e] = pack_bf16(__uint_as_float(r[8 * g + 2 * e]) * inv, __uint_as_float(r[8 * g + 2 * e + 1]) * inv);
-                        *reinterpret_cast<uint4*>(op + c * 32 + g * 8) = make_uint4(w[0], w[1], w[2], w[3]);
-                    }
+                    for (int e = 0; e < 4; ++e)
+                        w[e] = pack_bf16(__uint_as_float(o[8 * g8 + 2 * e]) * inv, __uint_as_float(o[8 * g8 + 2 * e + 1]) * inv);
+                    *reinterpret_cast<uint4*>(op + g8 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
                 }
             }
         }
+    }
     }
 
     tc_fence_before();
     __syncthreads();
     if (*abort_flag && threadIdx.x == 0) atomicExch(args.status, RS_DEV_TIMEOUT);
-    if (warp == 1) {
+    if (warp == 9) {
+        __syncwarp();
         tc_fence_after();
         tmem_dealloc(tmem_base, kTmemCols);
     }
@@ -313,7 +377,7 @@ cudaError_t launch_attn_tc(rs_ctx* ctx, const rs_attn_desc& d, const void* q, co
     const float scale = d.scale != 0.f ? d.scale : 0.125f;
     args.scale_log2 = scale * 1.4426950408889634f;
     args.status = ctx->d_status;
-    const dim3 grid((d.N + BQ - 1) / BQ, d.H, d.B);
+    const dim3 grid((d.N + 2 * BQ - 1) / (2 * BQ), d.H, d.B);
     attn_tc_kernel<<<grid, kThreads, kSmem, st>>>(tmQ, tmK, tmV, args);
     return cudaGetLastError();
 }
