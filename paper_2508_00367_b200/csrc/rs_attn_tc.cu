@@ -4,14 +4,16 @@
 // One CTA owns two 128-row query tiles (A and B) of one (sample, head) and streams the
 // keys/values in tiles of 128 through a TMA ring that both query tiles share.  For each
 // query tile and key tile:  S = Q K^T (tcgen05.mma, fp32 in tensor memory)  ->  one softmax
-// warpgroup (a row per thread) reads S, keeps a running maximum and sum, and writes
-// P = exp2(S*c - m*c) as bf16 back into tensor memory over S  ->  O += P V (tcgen05.mma
-// with P as the tensor-memory A operand and the V tile as an MN-major shared-memory B
-// operand).  The MMA warp alternates between the two query tiles, so the tensor pipe works
-// on one tile's P V and next Q K^T while the other tile's exponentials run.  The running
-// maximum is only raised when a tile's maximum exceeds it by more than 2^8 (P stays below
-// 256, exact softmax is recovered by the final division), so the O accumulator is rarely
-// rescaled and the softmax warps do that themselves.
+// warpgroup (a row per thread) pulls the S row into registers and at once hands the S
+// columns back, so the next Q K^T is computed while this tile's exponentials run; it keeps a
+// running maximum and sum and writes P = exp2(S*c - m*c) as bf16 into its own tensor-memory
+// columns  ->  O += P V (tcgen05.mma with P as the tensor-memory A operand and the V tile as
+// an MN-major shared-memory B operand).  The exponentials (MUFU) bound this head dimension,
+// so everything else is arranged to keep them flowing: the exponent of a tile is taken
+// against the maximum known *before* the tile, in the same pass that finds the tile's own
+// maximum; only if that exceeds the running one by more than 2^8 (P would leave bf16's
+// comfortable range) is the running maximum raised, O rescaled and the pass repeated.  The
+// final division by the row sum makes the result the exact softmax either way.
 #include <math.h>
 
 #include "rs_internal.h"
@@ -28,8 +30,10 @@ constexpr int TILE_BYTES = 128 * DH * 2;        // 16 KB: a [128, 64] bf16 tile
 constexpr int NS = 4;                           // K/V ring stages
 constexpr int kThreads = 384;                   // warps 0-3 / 4-7: softmax of tile A / B, warp 8: TMA, warp 9: MMA
 constexpr int kSoftmaxRegs = 224, kOtherRegs = 56;   // per-thread register budgets after the warpgroups re-split the pool
-constexpr int kTmemCols = 512;                  // S_A 0..127, S_B 128..255, O_A 256..319, O_B 320..383
-constexpr int kOCol = 256;
+constexpr int kTmemCols = 512;                  // S_A 0..127, S_B 128..255, P_A 256..319, P_B 320..383, O_A 384..447, O_B 448..511
+constexpr int kPCol = 256, kOCol = 384;
+constexpr bool kPingPong = true;
+constexpr int kPingPongTiles = 1;
 constexpr float kRescaleGap = 8.f;              // log2 units the tile maximum may exceed the running one
 // shared memory: Q_A | Q_B | K[NS] | V[NS] | barriers
 constexpr int OFF_Q = 0, OFF_K = 2 * TILE_BYTES, OFF_V = (2 + NS) * TILE_BYTES;
@@ -53,8 +57,88 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
     __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
     return *reinterpret_cast<uint32_t*>(&h);
 }
+// bf16 pair of two non-negative floats with integer instructions only (round half up: add half
+// an ulp to the bit patterns, keep the upper halves).  The conversion instruction shares the
+// MUFU pipe with the exponentials, which is the pipe this kernel is bound by; this does not.
+// Differs from round-to-nearest-even only on exact ties.
+__device__ __forceinline__ uint32_t pack_bf16_pos(float a, float b) {
+    return __byte_perm(__float_as_uint(a) + 0x8000u, __float_as_uint(b) + 0x8000u, 0x7632);
+}
 
-__device__ __forceinline__ float max3(float a, float b, float c) { return fmaxf(fmaxf(a, b), c); }
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float r;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
+}
+
+// Packed fp32 pairs (two lanes of arithmetic per instruction on sm_100).
+__device__ __forceinline__ uint64_t pack2(float a, float b) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+    return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& a, float& b) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v));
+}
+__device__ __forceinline__ uint64_t ffma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ uint64_t fadd2(uint64_t a, uint64_t b) {
+    uint64_t r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+
+// Maximum of a row of S held in registers (valid keys only).
+template <bool MASKED>
+__device__ __forceinline__ float row_max(const uint32_t (&r)[128], int valid) {
+    float m0 = -INFINITY, m1 = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < 128; i += 4) {
+        float a = __uint_as_float(r[i]), b = __uint_as_float(r[i + 1]);
+        float c = __uint_as_float(r[i + 2]), d = __uint_as_float(r[i + 3]);
+        if (MASKED) {
+            if (i >= valid) a = -INFINITY;
+            if (i + 1 >= valid) b = -INFINITY;
+            if (i + 2 >= valid) c = -INFINITY;
+            if (i + 3 >= valid) d = -INFINITY;
+        }
+        m0 = max3(m0, a, b);
+        m1 = max3(m1, c, d);
+    }
+    return fmaxf(m0, m1);
+}
+
+// p_i = exp2(s_i * sl + mneg) for the valid keys (0 for the rest), packed to bf16 pairs in
+// place (r[0..63] on return); returns the sum of the unrounded p_i.
+template <bool MASKED>
+__device__ __forceinline__ float exp_pass(uint32_t (&r)[128], float sl, float mneg, int valid) {
+    const uint64_t sl2 = pack2(sl, sl), mneg2 = pack2(mneg, mneg);
+    uint64_t l01 = pack2(0.f, 0.f), l23 = l01;
+#pragma unroll
+    for (int i = 0; i < 128; i += 4) {
+        float x0, x1, x2, x3;
+        unpack2(ffma2(pack2(__uint_as_float(r[i]), __uint_as_float(r[i + 1])), sl2, mneg2), x0, x1);
+        unpack2(ffma2(pack2(__uint_as_float(r[i + 2]), __uint_as_float(r[i + 3])), sl2, mneg2), x2, x3);
+        if (MASKED) {
+            if (i >= valid) x0 = -INFINITY;
+            if (i + 1 >= valid) x1 = -INFINITY;
+            if (i + 2 >= valid) x2 = -INFINITY;
+            if (i + 3 >= valid) x3 = -INFINITY;
+        }
+        const float p0 = ex2(x0), p1 = ex2(x1), p2 = ex2(x2), p3 = ex2(x3);   // ex2(-inf) = 0
+        l01 = fadd2(l01, pack2(p0, p1));
+        l23 = fadd2(l23, pack2(p2, p3));
+        r[i >> 1] = pack_bf16(p0, p1);
+        r[(i >> 1) + 1] = pack_bf16(p2, p3);
+    }
+    float a, b, c, d;
+    unpack2(l01, a, b);
+    unpack2(l23, c, d);
+    return (a + b) + (c + d);
+}
 
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
@@ -69,7 +153,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     uint64_t* s_full = bars + 1 + 3 * NS;    // [2] S of tile A / B complete in tensor memory
     uint64_t* p_ready = s_full + 2;          // [2] P written (one arrival per softmax warp)
     uint64_t* o_done = s_full + 4;           // [2] O += P V retired
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(s_full + 6);
+    uint64_t* s_free = s_full + 6;           // [2] S row in registers, columns reusable (one arrival per warp)
+    uint64_t* turn = s_full + 8;             // [2][4] exponent pass of tile A / B, warp q, finished
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(s_full + 16);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -82,7 +168,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         prefetch_tmap(&tmQ); prefetch_tmap(&tmK); prefetch_tmap(&tmV);
         mbar_init(q_full, 1);
         for (int s = 0; s < NS; ++s) { mbar_init(&k_full[s], 1); mbar_init(&v_full[s], 1); mbar_init(&kv_empty[s], 1); }
-        for (int g = 0; g < 2; ++g) { mbar_init(&s_full[g], 1); mbar_init(&p_ready[g], 4); mbar_init(&o_done[g], 1); }
+        for (int g = 0; g < 2; ++g) { mbar_init(&s_full[g], 1); mbar_init(&p_ready[g], 4); mbar_init(&o_done[g], 1); mbar_init(&s_free[g], 4); }
+        for (int i = 0; i < 8; ++i) mbar_init(&turn[i], 1);
         *abort_flag = 0;
         mbar_fence_init();
     }
@@ -147,7 +234,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 const int ksteps = (valid + 15) >> 4;
                 const uint32_t sv = smem_u32(smem + OFF_V + s * TILE_BYTES);
                 for (int k = 0; k < ksteps; ++k)
-                    mma_ts(tmem_base + kOCol + g * DH, tmem_base + g * BKV + 8 * k,
+                    mma_ts(tmem_base + kOCol + g * DH, tmem_base + kPCol + g * DH + 8 * k,
                            smem_desc_sw128(sv + (uint32_t)k * 2048u, 16, 1024), idesc_o, (j | k) != 0);
                 mma_commit(&o_done[g]);
             };
@@ -159,23 +246,28 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             }
             for (int j = 0; j < nkv && ok; ++j) {
                 const int s = j % NS;
-                const bool more = j + 1 < nkv;
+                if (j + 1 < nkv) {
+                    // next S tiles as soon as the softmax warps hold the current ones in registers
+                    if (!mbar_wait(&k_full[(j + 1) % NS], ((j + 1) / NS) & 1, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(&s_free[0], j & 1, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    issue_s(0, j + 1);
+                    if (has_b) {
+                        if (!mbar_wait(&s_free[1], j & 1, abort_flag)) { ok = false; break; }
+                        tc_fence_after();
+                        issue_s(1, j + 1);
+                    }
+                }
                 if (!mbar_wait(&v_full[s], (j / NS) & 1, abort_flag)) { ok = false; break; }
                 if (!mbar_wait(&p_ready[0], j & 1, abort_flag)) { ok = false; break; }
                 tc_fence_after();
                 issue_pv(0, j);
-                if (more) {
-                    if (!mbar_wait(&k_full[(j + 1) % NS], ((j + 1) / NS) & 1, abort_flag)) { ok = false; break; }
-                    tc_fence_after();
-                    issue_s(0, j + 1);
-                }
                 if (has_b) {
                     if (!mbar_wait(&p_ready[1], j & 1, abort_flag)) { ok = false; break; }
                     tc_fence_after();
                     issue_pv(1, j);
                 }
                 mma_commit(&kv_empty[s]);
-                if (more && has_b) issue_s(1, j + 1);
             }
         }
     }
@@ -187,7 +279,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         const int q = warp & 3;                          // tensor-memory lane quadrant of this warp
         const int row = q0 + g * BQ + q * 32 + lane;
         const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
-        const uint32_t s_addr = lane_addr + g * BKV, o_addr = lane_addr + kOCol + g * DH;
+        const uint32_t s_addr = lane_addr + g * BKV, p_addr = lane_addr + kPCol + g * DH,
+                       o_addr = lane_addr + kOCol + g * DH;
         const float sl = args.scale_log2;
         float m_l2 = 0.f, l_run = 0.f;                   // running maximum (times scale*log2 e) and sum
         bool ok = true;
@@ -202,87 +295,50 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
 #pragma unroll
             for (int c = 0; c < 4; ++c) tmem_ld_32x32(s_addr + c * 32, r + c * 32);
             tmem_wait_ld();
-            // row maximum over the valid keys
-            float mx = -INFINITY;
-            if (valid == BKV) {
-                float m0 = max3(__uint_as_float(r[0]), __uint_as_float(r[1]), __uint_as_float(r[2]));
-                float m1 = max3(__uint_as_float(r[3]), __uint_as_float(r[4]), __uint_as_float(r[5]));
-#pragma unroll
-                for (int i = 6; i + 3 < 128; i += 4) {
-                    m0 = max3(m0, __uint_as_float(r[i]), __uint_as_float(r[i + 1]));
-                    m1 = max3(m1, __uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
-                }
-                mx = max3(m0, m1, fmaxf(__uint_as_float(r[126]), __uint_as_float(r[127])));
-            } else {
-#pragma unroll
-                for (int i = 0; i < 128; ++i)
-                    if (i < valid) mx = fmaxf(mx, __uint_as_float(r[i]));
-            }
-            const float mx_l2 = mx * sl;
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&s_free[g]);      // the next Q K^T may overwrite S now
+            // running maximum: raised only when the tile tops it by more than 2^kRescaleGap
+            const float mx_l2 = (valid == BKV ? row_max<false>(r, valid) : row_max<true>(r, valid)) * sl;
             if (j == 0) {
                 m_l2 = mx_l2;
-            } else {
+            } else if (__any_sync(0xffffffffu, mx_l2 > m_l2 + kRescaleGap)) {
+                // rare: rescale O and the sum; O += P V of the previous key tile must have retired
+                if (!__all_sync(0xffffffffu, mbar_wait(&o_done[g], (j - 1) & 1, abort_flag))) { ok = false; break; }
+                tc_fence_after();
                 const bool raise = mx_l2 > m_l2 + kRescaleGap;
-                if (__any_sync(0xffffffffu, raise)) {
-                    // O += P V of the previous key tile must have retired before O is rescaled
-                    if (!__all_sync(0xffffffffu, mbar_wait(&o_done[g], (j - 1) & 1, abort_flag))) { ok = false; break; }
-                    tc_fence_after();
-                    const float alpha = raise ? ex2(m_l2 - mx_l2) : 1.f;
-                    if (raise) m_l2 = mx_l2;
-                    l_run *= alpha;
+                const float alpha = raise ? ex2(m_l2 - mx_l2) : 1.f;
+                if (raise) m_l2 = mx_l2;
+                l_run *= alpha;
 #pragma unroll
-                    for (int c = 0; c < 2; ++c) {
-                        uint32_t o[32];
-                        tmem_ld_32x32(o_addr + c * 32, o);
-                        tmem_wait_ld();
+                for (int c = 0; c < 2; ++c) {
+                    uint32_t o[32];
+                    tmem_ld_32x32(o_addr + c * 32, o);
+                    tmem_wait_ld();
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-                        tmem_st_32x32(o_addr + c * 32, o);
-                    }
-                    tmem_wait_st();
+                    for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                    tmem_st_32x32(o_addr + c * 32, o);
                 }
+                tmem_wait_st();
             }
-            // P = exp2(S*c - m*c) -> bf16 pairs -> tensor memory, over the S columns already read
-            const float mneg = -m_l2;
-            float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
-            if (valid == BKV) {
-#pragma unroll
-                for (int c = 0; c < 8; ++c) {
-                    uint32_t pk[8];
-#pragma unroll
-                    for (int i = 0; i < 16; i += 4) {
-                        const float p0 = ex2(fmaf(__uint_as_float(r[16 * c + i]), sl, mneg));
-                        const float p1 = ex2(fmaf(__uint_as_float(r[16 * c + i + 1]), sl, mneg));
-                        const float p2 = ex2(fmaf(__uint_as_float(r[16 * c + i + 2]), sl, mneg));
-                        const float p3 = ex2(fmaf(__uint_as_float(r[16 * c + i + 3]), sl, mneg));
-                        l0 += p0; l1 += p1; l2 += p2; l3 += p3;
-                        pk[i >> 1] = pack_bf16(p0, p1);
-                        pk[(i >> 1) + 1] = pack_bf16(p2, p3);
-                    }
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) r[8 * c + i] = pk[i];
-                }
-#pragma unroll
-                for (int c = 0; c < 4; ++c) tmem_st_32x16(s_addr + c * 16, r + c * 16);
-            } else {
-#pragma unroll
-                for (int c = 0; c < 8; ++c) {
-                    uint32_t pk[8];
-#pragma unroll
-                    for (int i = 0; i < 16; i += 2) {
-                        const int col = 16 * c + i;
-                        const float p0 = col < valid ? ex2(fmaf(__uint_as_float(r[col]), sl, mneg)) : 0.f;
-                        const float p1 = col + 1 < valid ? ex2(fmaf(__uint_as_float(r[col + 1]), sl, mneg)) : 0.f;
-                        l0 += p0; l1 += p1;
-                        pk[i >> 1] = pack_bf16(p0, p1);
-                    }
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) r[8 * c + i] = pk[i];
-                }
-#pragma unroll
-                for (int c = 0; c < 4; ++c) tmem_st_32x16(s_addr + c * 16, r + c * 16);
+            // The two softmax warps of a scheduler (tile A's and tile B's warp q) take turns at
+            // the exponent pass: the MUFU unit is the bottleneck, and run one at a time each pass
+            // overlaps the other warp's loads, stores and waits instead of its exponentials.
+            // Order: A0 B0 A1 B1 ...
+            if (kPingPong && has_b && j < kPingPongTiles && (g == 1 || j > 0)) {
+                const uint32_t par = (g == 1 ? j : j - 1) & 1;
+                if (!__all_sync(0xffffffffu, mbar_wait(&turn[(g ^ 1) * 4 + q], par, abort_flag))) { ok = false; break; }
             }
-            l_run += (l0 + l1) + (l2 + l3);
+            const float lsum = valid == BKV ? exp_pass<false>(r, sl, -m_l2, valid) : exp_pass<true>(r, sl, -m_l2, valid);
+            if (kPingPong && has_b && lane == 0) mbar_arrive(&turn[g * 4 + q]);
+            if (j > 0) {
+                // P V of the previous key tile reads the P columns: it must have retired
+                if (!__all_sync(0xffffffffu, mbar_wait(&o_done[g], (j - 1) & 1, abort_flag))) { ok = false; break; }
+                tc_fence_after();
+            }
+            l_run += lsum;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) tmem_st_32x16(p_addr + c * 16, r + c * 16);
             tmem_wait_st();
             tc_fence_before();
             __syncwarp();
