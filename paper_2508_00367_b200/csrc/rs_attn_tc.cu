@@ -1,19 +1,20 @@
 // Fused attention on the tensor cores (Eq. sa): out = Softmax(Q K^T * scale) V per
 // (sample, head), head dimension 64, without ever writing the N x N matrix.
 //
-// One CTA owns two 128-row query tiles (A and B) of one (sample, head) and streams the
-// keys/values in tiles of 128 through a TMA ring that both query tiles share.  For each
-// query tile and key tile:  S = Q K^T (tcgen05.mma, fp32 in tensor memory)  ->  one softmax
-// warpgroup (a row per thread) pulls the S row into registers and at once hands the S
-// columns back, so the next Q K^T is computed while this tile's exponentials run; it keeps a
-// running maximum and sum and writes P = exp2(S*c - m*c) as bf16 into its own tensor-memory
-// columns  ->  O += P V (tcgen05.mma with P as the tensor-memory A operand and the V tile as
-// an MN-major shared-memory B operand).  The exponentials (MUFU) bound this head dimension,
-// so everything else is arranged to keep them flowing: the exponent of a tile is taken
-// against the maximum known *before* the tile, in the same pass that finds the tile's own
-// maximum; only if that exceeds the running one by more than 2^8 (P would leave bf16's
-// comfortable range) is the running maximum raised, O rescaled and the pass repeated.  The
-// final division by the row sum makes the result the exact softmax either way.
+// Persistent kernel, one CTA per SM, looping over work items.  An item is two 128-row query
+// tiles A and B: for N > 128 two consecutive query tiles of one (sample, head), which share
+// the key/value tiles streamed through a TMA ring; for N <= 128 the single query tile of two
+// neighbouring heads, each with its own key/value tile.  For each query tile and key tile:
+// S = Q K^T (tcgen05.mma, fp32 in tensor memory)  ->  a softmax warpgroup (a row per thread)
+// pulls the S row into registers and at once hands the S columns back, so the next Q K^T is
+// computed while this tile's exponentials run; it keeps a running maximum and sum and writes
+// P = exp2(S*c - m*c) as bf16 into P's own tensor-memory columns  ->  O += P V (tcgen05.mma
+// with P as the tensor-memory A operand and the V tile as an MN-major shared-memory B
+// operand).  The running maximum is raised only when a tile tops it by more than 2^8 (the
+// final division by the row sum gives the exact softmax either way), so O is rarely rescaled
+// and the softmax warps do that themselves.  The TMA producer, the MMA issuer and the softmax
+// warps each walk the same item list and keep their own phase counters, so loads, Q K^T of the
+// next item and the epilogue of the previous one overlap across item boundaries.
 #include <math.h>
 
 #include "rs_internal.h"
@@ -29,23 +30,53 @@ constexpr int BQ = 128, BKV = 128, DH = 64;
 constexpr int TILE_BYTES = 128 * DH * 2;        // 16 KB: a [128, 64] bf16 tile
 constexpr int NS = 4;                           // K/V ring stages
 constexpr int kThreads = 384;                   // warps 0-3 / 4-7: softmax of tile A / B, warp 8: TMA, warp 9: MMA
-constexpr int kSoftmaxRegs = 224, kOtherRegs = 56;   // per-thread register budgets after the warpgroups re-split the pool
+constexpr int kSoftmaxRegs = 208, kOtherRegs = 88;   // per-thread register budgets after the warpgroups re-split the pool
 constexpr int kTmemCols = 512;                  // S_A 0..127, S_B 128..255, P_A 256..319, P_B 320..383, O_A 384..447, O_B 448..511
 constexpr int kPCol = 256, kOCol = 384;
-constexpr bool kPingPong = true;
-constexpr int kPingPongTiles = 1;
 constexpr float kRescaleGap = 8.f;              // log2 units the tile maximum may exceed the running one
-// shared memory: Q_A | Q_B | K[NS] | V[NS] | barriers
-constexpr int OFF_Q = 0, OFF_K = 2 * TILE_BYTES, OFF_V = (2 + NS) * TILE_BYTES;
-constexpr int OFF_BAR = (2 + 2 * NS) * TILE_BYTES;
+// shared memory: Q[2 buffers][A, B] | K[NS] | V[NS] | barriers
+constexpr int OFF_Q = 0, OFF_K = 4 * TILE_BYTES, OFF_V = (4 + NS) * TILE_BYTES;
+constexpr int OFF_BAR = (4 + 2 * NS) * TILE_BYTES;
 constexpr size_t kSmem = (size_t)OFF_BAR + 256 + 1024 /*alignment slack*/;
 
 struct AttnArgs {
     __nv_bfloat16* out;      // [B, N, H*64]
     int N, H;
+    int dual;                // 1: N <= 128, an item is two heads; 0: an item is two query tiles of one head
+    int per;                 // items per (sample, head) [dual = 0] or per sample [dual = 1]
+    int n_items;
     float scale_log2;        // scale * log2(e)
     int* status;
 };
+
+// One work item, decoded the same way by every role.
+struct Item {
+    int b, h[2], q0[2];      // sample; head and first query row of tile A / B
+    int ng;                  // 1 or 2 query tiles present
+    int nkv;                 // key tiles per query tile
+    int slots;               // K/V ring stages the item consumes
+};
+__device__ __forceinline__ Item decode_item(const AttnArgs& a, int w) {
+    Item it;
+    if (a.dual) {
+        const int hp = w % a.per;
+        it.b = w / a.per;
+        it.h[0] = 2 * hp; it.h[1] = 2 * hp + 1;
+        it.q0[0] = it.q0[1] = 0;
+        it.ng = it.h[1] < a.H ? 2 : 1;
+        it.nkv = 1;
+        it.slots = it.ng;
+    } else {
+        const int qp = w % a.per, bh = w / a.per;
+        it.b = bh / a.H;
+        it.h[0] = it.h[1] = bh % a.H;
+        it.q0[0] = qp * 2 * BQ; it.q0[1] = it.q0[0] + BQ;
+        it.ng = it.q0[1] < a.N ? 2 : 1;
+        it.nkv = (a.N + BKV - 1) / BKV;
+        it.slots = it.nkv;
+    }
+    return it;
+}
 
 __device__ __forceinline__ float ex2(float x) {
     float y;
@@ -56,13 +87,6 @@ __device__ __forceinline__ float ex2(float x) {
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
     __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
     return *reinterpret_cast<uint32_t*>(&h);
-}
-// bf16 pair of two non-negative floats with integer instructions only (round half up: add half
-// an ulp to the bit patterns, keep the upper halves).  The conversion instruction shares the
-// MUFU pipe with the exponentials, which is the pipe this kernel is bound by; this does not.
-// Differs from round-to-nearest-even only on exact ties.
-__device__ __forceinline__ uint32_t pack_bf16_pos(float a, float b) {
-    return __byte_perm(__float_as_uint(a) + 0x8000u, __float_as_uint(b) + 0x8000u, 0x7632);
 }
 
 __device__ __forceinline__ float max3(float a, float b, float c) {
@@ -91,34 +115,35 @@ __device__ __forceinline__ uint64_t fadd2(uint64_t a, uint64_t b) {
     return r;
 }
 
-// Maximum of a row of S held in registers (valid keys only).
-template <bool MASKED>
+// Maximum of the first NC values of a row of S held in registers (only the first `valid` count).
+template <int NC, bool MASKED>
 __device__ __forceinline__ float row_max(const uint32_t (&r)[128], int valid) {
-    float m0 = -INFINITY, m1 = -INFINITY;
+    float m[8];
 #pragma unroll
-    for (int i = 0; i < 128; i += 4) {
-        float a = __uint_as_float(r[i]), b = __uint_as_float(r[i + 1]);
-        float c = __uint_as_float(r[i + 2]), d = __uint_as_float(r[i + 3]);
-        if (MASKED) {
-            if (i >= valid) a = -INFINITY;
-            if (i + 1 >= valid) b = -INFINITY;
-            if (i + 2 >= valid) c = -INFINITY;
-            if (i + 3 >= valid) d = -INFINITY;
+    for (int c = 0; c < 8; ++c) m[c] = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < NC; i += 16) {               // eight independent chains: latency, not count, is the cost
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            float a = __uint_as_float(r[i + 2 * c]), b = __uint_as_float(r[i + 2 * c + 1]);
+            if (MASKED) {
+                if (i + 2 * c >= valid) a = -INFINITY;
+                if (i + 2 * c + 1 >= valid) b = -INFINITY;
+            }
+            m[c] = max3(m[c], a, b);
         }
-        m0 = max3(m0, a, b);
-        m1 = max3(m1, c, d);
     }
-    return fmaxf(m0, m1);
+    return max3(max3(m[0], m[1], m[2]), max3(m[3], m[4], m[5]), fmaxf(m[6], m[7]));
 }
 
-// p_i = exp2(s_i * sl + mneg) for the valid keys (0 for the rest), packed to bf16 pairs in
-// place (r[0..63] on return); returns the sum of the unrounded p_i.
-template <bool MASKED>
+// p_i = exp2(s_i * sl + mneg) for the first `valid` of NC keys (0 for the rest), packed to bf16
+// pairs in place (r[0 .. NC/2) on return); returns the sum of the unrounded p_i.
+template <int NC, bool MASKED>
 __device__ __forceinline__ float exp_pass(uint32_t (&r)[128], float sl, float mneg, int valid) {
     const uint64_t sl2 = pack2(sl, sl), mneg2 = pack2(mneg, mneg);
     uint64_t l01 = pack2(0.f, 0.f), l23 = l01;
 #pragma unroll
-    for (int i = 0; i < 128; i += 4) {
+    for (int i = 0; i < NC; i += 4) {
         float x0, x1, x2, x3;
         unpack2(ffma2(pack2(__uint_as_float(r[i]), __uint_as_float(r[i + 1])), sl2, mneg2), x0, x1);
         unpack2(ffma2(pack2(__uint_as_float(r[i + 2]), __uint_as_float(r[i + 3])), sl2, mneg2), x2, x3);
@@ -146,30 +171,28 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + OFF_BAR);
-    uint64_t* q_full = bars;                 // Q tiles landed
-    uint64_t* k_full = bars + 1;             // [NS] K tile landed
-    uint64_t* v_full = bars + 1 + NS;        // [NS] V tile landed
-    uint64_t* kv_empty = bars + 1 + 2 * NS;  // [NS] every MMA reading the stage retired
-    uint64_t* s_full = bars + 1 + 3 * NS;    // [2] S of tile A / B complete in tensor memory
+    uint64_t* q_full = bars;                 // [2] Q tiles of the item landed in buffer 0 / 1
+    uint64_t* q_empty = bars + 2;            // [2] every Q K^T of the item in that buffer retired
+    uint64_t* k_full = bars + 4;             // [NS] K tile landed
+    uint64_t* v_full = k_full + NS;          // [NS] V tile landed
+    uint64_t* kv_empty = k_full + 2 * NS;    // [NS] every MMA reading the stage retired
+    uint64_t* s_full = k_full + 3 * NS;      // [2] S of tile A / B complete in tensor memory
     uint64_t* p_ready = s_full + 2;          // [2] P written (one arrival per softmax warp)
     uint64_t* o_done = s_full + 4;           // [2] O += P V retired
     uint64_t* s_free = s_full + 6;           // [2] S row in registers, columns reusable (one arrival per warp)
-    uint64_t* turn = s_full + 8;             // [2][4] exponent pass of tile A / B, warp q, finished
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(s_full + 16);
+    uint64_t* first_pass = s_full + 8;       // tile A's warps finished the first exponent pass of an item
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(s_full + 9);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int N = args.N;
-    const int q0 = blockIdx.x * (2 * BQ), h = blockIdx.y, b = blockIdx.z;
-    const int nkv = (N + BKV - 1) / BKV;
-    const bool has_b = q0 + BQ < N;          // the second query tile has at least one row
 
     if (threadIdx.x == 0) {
         prefetch_tmap(&tmQ); prefetch_tmap(&tmK); prefetch_tmap(&tmV);
-        mbar_init(q_full, 1);
+        for (int i = 0; i < 2; ++i) { mbar_init(&q_full[i], 1); mbar_init(&q_empty[i], 1); }
         for (int s = 0; s < NS; ++s) { mbar_init(&k_full[s], 1); mbar_init(&v_full[s], 1); mbar_init(&kv_empty[s], 1); }
         for (int g = 0; g < 2; ++g) { mbar_init(&s_full[g], 1); mbar_init(&p_ready[g], 4); mbar_init(&o_done[g], 1); mbar_init(&s_free[g], 4); }
-        for (int i = 0; i < 8; ++i) mbar_init(&turn[i], 1);
+        mbar_init(first_pass, 4);
         *abort_flag = 0;
         mbar_fence_init();
     }
@@ -188,167 +211,210 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     if (warp == 8) {
         // ---------------- TMA producer ----------------
         if (elect_one()) {
-            mbar_expect_tx(q_full, has_b ? 2 * TILE_BYTES : TILE_BYTES);
-            tma_load_4d(smem + OFF_Q, &tmQ, q_full, 0, h, q0, b);
-            if (has_b) tma_load_4d(smem + OFF_Q + TILE_BYTES, &tmQ, q_full, 0, h, q0 + BQ, b);
-            int issued = 0;
+            uint32_t kv_it = 0, item_n = 0;
             bool ok = true;
-            for (int j = 0; j < nkv; ++j, ++issued) {
-                const int s = j % NS;
-                if (!mbar_wait(&kv_empty[s], ((j / NS) & 1) ^ 1, abort_flag)) { ok = false; break; }
-                mbar_expect_tx(&k_full[s], TILE_BYTES);
-                tma_load_4d(smem + OFF_K + s * TILE_BYTES, &tmK, &k_full[s], 0, h, j * BKV, b);
-                mbar_expect_tx(&v_full[s], TILE_BYTES);
-                tma_load_4d(smem + OFF_V + s * TILE_BYTES, &tmV, &v_full[s], 0, h, j * BKV, b);
+            for (int w = blockIdx.x; w < args.n_items && ok; w += gridDim.x, ++item_n) {
+                const Item it = decode_item(args, w);
+                const uint32_t qb = item_n & 1u;
+                if (!mbar_wait(&q_empty[qb], ((item_n >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+                mbar_expect_tx(&q_full[qb], it.ng * TILE_BYTES);
+#pragma unroll
+                for (int g = 0; g < 2; ++g)
+                    if (g < it.ng) tma_load_4d(smem + OFF_Q + (qb * 2 + g) * TILE_BYTES, &tmQ, &q_full[qb], 0, it.h[g], it.q0[g], it.b);
+                for (int t = 0; t < it.slots; ++t, ++kv_it) {
+                    const int s = kv_it % NS;
+                    if (!mbar_wait(&kv_empty[s], ((kv_it / NS) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+                    const int head = (args.dual && t == 1) ? it.h[1] : it.h[0], row0 = args.dual ? 0 : t * BKV;
+                    mbar_expect_tx(&k_full[s], TILE_BYTES);
+                    tma_load_4d(smem + OFF_K + s * TILE_BYTES, &tmK, &k_full[s], 0, head, row0, it.b);
+                    mbar_expect_tx(&v_full[s], TILE_BYTES);
+                    tma_load_4d(smem + OFF_V + s * TILE_BYTES, &tmV, &v_full[s], 0, head, row0, it.b);
+                }
             }
             // every copy started here must have landed before the CTA exits
-            if (ok) ok = mbar_wait(q_full, 0, abort_flag);
-            for (int s = 0; s < NS && s < issued && ok; ++s) {
-                const int last = ((issued - 1 - s) / NS) * NS + s;
-                ok = mbar_wait(&k_full[s], (last / NS) & 1, abort_flag) && mbar_wait(&v_full[s], (last / NS) & 1, abort_flag);
-            }
+            for (uint32_t n = item_n > 2 ? item_n - 2 : 0; n < item_n && ok; ++n)
+                ok = mbar_wait(&q_full[n & 1u], (n >> 1) & 1u, abort_flag);
+            for (uint32_t t = kv_it > NS ? kv_it - NS : 0; t < kv_it && ok; ++t)
+                ok = mbar_wait(&k_full[t % NS], (t / NS) & 1u, abort_flag) && mbar_wait(&v_full[t % NS], (t / NS) & 1u, abort_flag);
         }
     } else if (warp == 9) {
         // ---------------- MMA issuer ----------------
-        if (elect_one()) {
-            bool ok = mbar_wait(q_full, 0, abort_flag);
-            tc_fence_after();
+        if (elect_one() && blockIdx.x < args.n_items) {
             const uint32_t idesc_o = idesc_bf16(BQ, DH, 0, 1);
-            // S_g = Q_g K_j^T : both operands K-major (head dimension contiguous)
-            auto issue_s = [&](int g, int j) {
-                const int s = j % NS;
-                const int valid = min(BKV, N - j * BKV);
+            uint32_t ns[2] = {0, 0}, np[2] = {0, 0};     // S tiles / P V products issued so far per query tile
+            bool ok = true;
+            // S_g = Q_g K^T : both operands K-major (head dimension contiguous).  The S columns must
+            // have been read by the softmax warps of the previous tile first.
+            auto issue_s = [&](int g, uint32_t qb, int stage, int valid) {
+                if (ns[g] > 0 && !mbar_wait(&s_free[g], (ns[g] - 1) & 1u, abort_flag)) { ok = false; return; }
+                tc_fence_after();
                 const uint32_t idesc_s = idesc_bf16(BQ, (valid + 15) & ~15, 0, 0);
-                const uint64_t dq = smem_desc_sw128(smem_u32(smem + OFF_Q + g * TILE_BYTES), 16, 1024);
-                const uint64_t dk = smem_desc_sw128(smem_u32(smem + OFF_K + s * TILE_BYTES), 16, 1024);
+                const uint64_t dq = smem_desc_sw128(smem_u32(smem + OFF_Q + (qb * 2 + g) * TILE_BYTES), 16, 1024);
+                const uint64_t dk = smem_desc_sw128(smem_u32(smem + OFF_K + stage * TILE_BYTES), 16, 1024);
 #pragma unroll
                 for (int k = 0; k < DH / 16; ++k)
                     mma_ss(tmem_base + g * BKV, dq + 2u * k, dk + 2u * k, idesc_s, k != 0);
                 mma_commit(&s_full[g]);
+                ++ns[g];
             };
-            // O_g += P_g V_j : P from tensor memory (bf16 pairs, 8 columns per 16 keys), V MN-major
+            // O_g (+)= P_g V : P from tensor memory (bf16 pairs, 8 columns per 16 keys), V MN-major
             // (head dimension contiguous), 16 keys = 2048 bytes per slab.
-            auto issue_pv = [&](int g, int j) {
-                const int s = j % NS;
-                const int valid = min(BKV, N - j * BKV);
+            auto issue_pv = [&](int g, int stage, int valid, bool first) {
+                if (!mbar_wait(&p_ready[g], np[g] & 1u, abort_flag)) { ok = false; return; }
+                tc_fence_after();
                 const int ksteps = (valid + 15) >> 4;
-                const uint32_t sv = smem_u32(smem + OFF_V + s * TILE_BYTES);
+                const uint32_t sv = smem_u32(smem + OFF_V + stage * TILE_BYTES);
                 for (int k = 0; k < ksteps; ++k)
                     mma_ts(tmem_base + kOCol + g * DH, tmem_base + kPCol + g * DH + 8 * k,
-                           smem_desc_sw128(sv + (uint32_t)k * 2048u, 16, 1024), idesc_o, (j | k) != 0);
+                           smem_desc_sw128(sv + (uint32_t)k * 2048u, 16, 1024), idesc_o, !(first && k == 0));
                 mma_commit(&o_done[g]);
+                ++np[g];
             };
-            if (ok) ok = mbar_wait(&k_full[0], 0, abort_flag);
-            if (ok) {
-                tc_fence_after();
-                issue_s(0, 0);
-                if (has_b) issue_s(1, 0);
-            }
-            for (int j = 0; j < nkv && ok; ++j) {
-                const int s = j % NS;
-                if (j + 1 < nkv) {
-                    // next S tiles as soon as the softmax warps hold the current ones in registers
-                    if (!mbar_wait(&k_full[(j + 1) % NS], ((j + 1) / NS) & 1, abort_flag)) { ok = false; break; }
-                    if (!mbar_wait(&s_free[0], j & 1, abort_flag)) { ok = false; break; }
-                    tc_fence_after();
-                    issue_s(0, j + 1);
-                    if (has_b) {
-                        if (!mbar_wait(&s_free[1], j & 1, abort_flag)) { ok = false; break; }
-                        tc_fence_after();
-                        issue_s(1, j + 1);
+            // Issues the Q K^T of step j of an item (for every query tile it has); kv0 = ring position
+            // of the item's first K/V slot.
+            auto issue_s_step = [&](const Item& it, uint32_t qb, uint32_t kv0, int j) {
+#pragma unroll
+                for (int g = 0; g < 2; ++g) {
+                    if (g >= it.ng || !ok) break;
+                    const uint32_t t = kv0 + (args.dual ? g : j);
+                    if (!mbar_wait(&k_full[t % NS], (t / NS) & 1u, abort_flag)) { ok = false; return; }
+                    issue_s(g, qb, t % NS, min(BKV, N - j * BKV));
+                }
+            };
+
+            uint32_t item_n = 0, kv0 = 0;
+            int w = blockIdx.x;
+            Item cur = decode_item(args, w);
+            ok = mbar_wait(&q_full[0], 0, abort_flag);
+            if (ok) issue_s_step(cur, 0, kv0, 0);
+            while (ok) {
+                const uint32_t qb = item_n & 1u;
+                for (int j = 0; j < cur.nkv && ok; ++j) {
+                    // look ahead: the next Q K^T (of this item, or the first of the next item) goes to
+                    // the tensor pipe before this step's P V, which still waits for the exponentials
+                    const bool last = j + 1 == cur.nkv;
+                    const int wn = w + gridDim.x;
+                    if (!last) {
+                        issue_s_step(cur, qb, kv0, j + 1);
+                    } else if (wn < args.n_items) {
+                        const Item nxt = decode_item(args, wn);
+                        const uint32_t nb = (item_n + 1) & 1u;
+                        if (!mbar_wait(&q_full[nb], ((item_n + 1) >> 1) & 1u, abort_flag)) { ok = false; break; }
+                        issue_s_step(nxt, nb, kv0 + cur.slots, 0);
+                    }
+                    if (!ok) break;
+                    const int valid = min(BKV, N - j * BKV);
+#pragma unroll
+                    for (int g = 0; g < 2; ++g) {
+                        if (g >= cur.ng || !ok) break;
+                        const uint32_t t = kv0 + (args.dual ? g : j);
+                        if (!mbar_wait(&v_full[t % NS], (t / NS) & 1u, abort_flag)) { ok = false; break; }
+                        issue_pv(g, t % NS, valid, j == 0);
+                        if (ok && (args.dual || g == cur.ng - 1)) mma_commit(&kv_empty[t % NS]);   // stage done
                     }
                 }
-                if (!mbar_wait(&v_full[s], (j / NS) & 1, abort_flag)) { ok = false; break; }
-                if (!mbar_wait(&p_ready[0], j & 1, abort_flag)) { ok = false; break; }
-                tc_fence_after();
-                issue_pv(0, j);
-                if (has_b) {
-                    if (!mbar_wait(&p_ready[1], j & 1, abort_flag)) { ok = false; break; }
-                    tc_fence_after();
-                    issue_pv(1, j);
-                }
-                mma_commit(&kv_empty[s]);
+                if (!ok) break;
+                mma_commit(&q_empty[qb]);
+                kv0 += cur.slots;
+                ++item_n;
+                w += gridDim.x;
+                if (w >= args.n_items) break;
+                cur = decode_item(args, w);
             }
         }
     }
     } else {
     asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kSoftmaxRegs));
-    if (warp < 4 || has_b) {
+    {
         // ---------------- softmax, O rescaling and output: one query row per thread ----------------
         const int g = warp >> 2;                         // query tile of this warpgroup
         const int q = warp & 3;                          // tensor-memory lane quadrant of this warp
-        const int row = q0 + g * BQ + q * 32 + lane;
         const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
         const uint32_t s_addr = lane_addr + g * BKV, p_addr = lane_addr + kPCol + g * DH,
                        o_addr = lane_addr + kOCol + g * DH;
         const float sl = args.scale_log2;
-        float m_l2 = 0.f, l_run = 0.f;                   // running maximum (times scale*log2 e) and sum
+        uint32_t cnt = 0, item_n = 0;                    // tiles / items this warpgroup has walked through
         bool ok = true;
-        for (int j = 0; j < nkv && ok; ++j) {
-            const int valid = min(BKV, N - j * BKV);
-            // the warp moves as one through the collective tensor-memory accesses below
-            if (!__all_sync(0xffffffffu, mbar_wait(&s_full[g], j & 1, abort_flag))) { ok = false; break; }
-            tc_fence_after();
-            // All 128 columns are read even on a partial key tile: columns past the keys the MMA
-            // wrote hold old values, which the masks below never let through.
-            uint32_t r[128];
-#pragma unroll
-            for (int c = 0; c < 4; ++c) tmem_ld_32x32(s_addr + c * 32, r + c * 32);
-            tmem_wait_ld();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&s_free[g]);      // the next Q K^T may overwrite S now
-            // running maximum: raised only when the tile tops it by more than 2^kRescaleGap
-            const float mx_l2 = (valid == BKV ? row_max<false>(r, valid) : row_max<true>(r, valid)) * sl;
-            if (j == 0) {
-                m_l2 = mx_l2;
-            } else if (__any_sync(0xffffffffu, mx_l2 > m_l2 + kRescaleGap)) {
-                // rare: rescale O and the sum; O += P V of the previous key tile must have retired
-                if (!__all_sync(0xffffffffu, mbar_wait(&o_done[g], (j - 1) & 1, abort_flag))) { ok = false; break; }
+        for (int w = blockIdx.x; w < args.n_items && ok; w += gridDim.x, ++item_n) {
+            const Item it = decode_item(args, w);
+            if (g >= it.ng) continue;
+            const int row = (g ? it.q0[1] : it.q0[0]) + q * 32 + lane;
+            float m_l2 = 0.f, l_run = 0.f;               // running maximum (times scale*log2 e) and sum
+            for (int j = 0; j < it.nkv && ok; ++j, ++cnt) {
+                const int valid = min(BKV, N - j * BKV);
+                // the warp moves as one through the collective tensor-memory accesses below
+                if (!__all_sync(0xffffffffu, mbar_wait(&s_full[g], cnt & 1u, abort_flag))) { ok = false; break; }
                 tc_fence_after();
-                const bool raise = mx_l2 > m_l2 + kRescaleGap;
-                const float alpha = raise ? ex2(m_l2 - mx_l2) : 1.f;
-                if (raise) m_l2 = mx_l2;
-                l_run *= alpha;
+                // Whole 32-column groups are read even on a partial key tile: columns past the keys
+                // the MMA wrote hold old values, which the masks below never let through.
+                uint32_t r[128];
+                const int ncol = valid > 64 ? 128 : valid > 32 ? 64 : 32;   // columns worth touching
+                tmem_ld_32x32(s_addr, r);
+                if (ncol > 32) tmem_ld_32x32(s_addr + 32, r + 32);
+                if (ncol > 64) {
+                    tmem_ld_32x32(s_addr + 64, r + 64);
+                    tmem_ld_32x32(s_addr + 96, r + 96);
+                }
+                tmem_wait_ld();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&s_free[g]);  // the next Q K^T may overwrite S now
+                // running maximum: raised only when the tile tops it by more than 2^kRescaleGap
+                const float mx = valid == BKV ? row_max<128, false>(r, valid)
+                                 : ncol == 128 ? row_max<128, true>(r, valid)
+                                 : ncol == 64  ? row_max<64, true>(r, valid)
+                                               : row_max<32, true>(r, valid);
+                const float mx_l2 = mx * sl;
+                if (j == 0) {
+                    m_l2 = mx_l2;
+                } else if (__any_sync(0xffffffffu, mx_l2 > m_l2 + kRescaleGap)) {
+                    // rare: rescale O and the sum; O += P V of the previous key tile must have retired
+                    if (!__all_sync(0xffffffffu, mbar_wait(&o_done[g], (cnt - 1) & 1u, abort_flag))) { ok = false; break; }
+                    tc_fence_after();
+                    const bool raise = mx_l2 > m_l2 + kRescaleGap;
+                    const float alpha = raise ? ex2(m_l2 - mx_l2) : 1.f;
+                    if (raise) m_l2 = mx_l2;
+                    l_run *= alpha;
 #pragma unroll
-                for (int c = 0; c < 2; ++c) {
-                    uint32_t o[32];
-                    tmem_ld_32x32(o_addr + c * 32, o);
-                    tmem_wait_ld();
+                    for (int c = 0; c < 2; ++c) {
+                        uint32_t o[32];
+                        tmem_ld_32x32(o_addr + c * 32, o);
+                        tmem_wait_ld();
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-                    tmem_st_32x32(o_addr + c * 32, o);
+                        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                        tmem_st_32x32(o_addr + c * 32, o);
+                    }
+                    tmem_wait_st();
+                }
+                // Tile B's first pass of an item starts when tile A's has ended: the two groups then
+                // stay out of step, and one group's loads, stores and waits hide behind the other's pass.
+                if (j == 0 && g == 1 && !__all_sync(0xffffffffu, mbar_wait(first_pass, item_n & 1u, abort_flag))) { ok = false; break; }
+                l_run += valid == BKV ? exp_pass<128, false>(r, sl, -m_l2, valid)
+                         : ncol == 128 ? exp_pass<128, true>(r, sl, -m_l2, valid)
+                         : ncol == 64  ? exp_pass<64, true>(r, sl, -m_l2, valid)
+                                       : exp_pass<32, true>(r, sl, -m_l2, valid);
+                if (j == 0 && g == 0 && lane == 0) mbar_arrive(first_pass);
+                if (cnt > 0) {
+                    // P V of the previous key tile reads the P columns: it must have retired
+                    if (!__all_sync(0xffffffffu, mbar_wait(&o_done[g], (cnt - 1) & 1u, abort_flag))) { ok = false; break; }
+                    tc_fence_after();
+                }
+                tmem_st_32x16(p_addr, r);
+                if (ncol > 32) tmem_st_32x16(p_addr + 16, r + 16);
+                if (ncol > 64) {
+                    tmem_st_32x16(p_addr + 32, r + 32);
+                    tmem_st_32x16(p_addr + 48, r + 48);
                 }
                 tmem_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&p_ready[g]);
             }
-            // The two softmax warps of a scheduler (tile A's and tile B's warp q) take turns at
-            // the exponent pass: the MUFU unit is the bottleneck, and run one at a time each pass
-            // overlaps the other warp's loads, stores and waits instead of its exponentials.
-            // Order: A0 B0 A1 B1 ...
-            if (kPingPong && has_b && j < kPingPongTiles && (g == 1 || j > 0)) {
-                const uint32_t par = (g == 1 ? j : j - 1) & 1;
-                if (!__all_sync(0xffffffffu, mbar_wait(&turn[(g ^ 1) * 4 + q], par, abort_flag))) { ok = false; break; }
-            }
-            const float lsum = valid == BKV ? exp_pass<false>(r, sl, -m_l2, valid) : exp_pass<true>(r, sl, -m_l2, valid);
-            if (kPingPong && has_b && lane == 0) mbar_arrive(&turn[g * 4 + q]);
-            if (j > 0) {
-                // P V of the previous key tile reads the P columns: it must have retired
-                if (!__all_sync(0xffffffffu, mbar_wait(&o_done[g], (j - 1) & 1, abort_flag))) { ok = false; break; }
-                tc_fence_after();
-            }
-            l_run += lsum;
-#pragma unroll
-            for (int c = 0; c < 4; ++c) tmem_st_32x16(p_addr + c * 16, r + c * 16);
-            tmem_wait_st();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&p_ready[g]);
-        }
-        // epilogue: O / l -> bf16 -> global
-        if (ok && __all_sync(0xffffffffu, mbar_wait(&o_done[g], (nkv - 1) & 1, abort_flag))) {
+            // epilogue of the item: O / l -> bf16 -> global
+            if (!ok || !__all_sync(0xffffffffu, mbar_wait(&o_done[g], (cnt - 1) & 1u, abort_flag))) { ok = false; break; }
             tc_fence_after();
             const float inv = 1.f / l_run;
-            __nv_bfloat16* op = args.out + ((size_t)((size_t)b * N + row) * args.H + h) * DH;
+            __nv_bfloat16* op = args.out + ((size_t)((size_t)it.b * N + row) * args.H + (g ? it.h[1] : it.h[0])) * DH;
             uint32_t o[64];
             tmem_ld_32x32(o_addr, o);
             tmem_ld_32x32(o_addr + 32, o + 32);
@@ -356,11 +422,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             if (row < N) {
 #pragma unroll
                 for (int g8 = 0; g8 < 8; ++g8) {
-                    uint32_t w[4];
+                    uint32_t wv[4];
 #pragma unroll
                     for (int e = 0; e < 4; ++e)
-                        w[e] = pack_bf16(__uint_as_float(o[8 * g8 + 2 * e]) * inv, __uint_as_float(o[8 * g8 + 2 * e + 1]) * inv);
-                    *reinterpret_cast<uint4*>(op + g8 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+                        wv[e] = pack_bf16(__uint_as_float(o[8 * g8 + 2 * e]) * inv, __uint_as_float(o[8 * g8 + 2 * e + 1]) * inv);
+                    *reinterpret_cast<uint4*>(op + g8 * 8) = make_uint4(wv[0], wv[1], wv[2], wv[3]);
                 }
             }
         }
@@ -430,10 +496,19 @@ cudaError_t launch_attn_tc(rs_ctx* ctx, const rs_attn_desc& d, const void* q, co
     AttnArgs args;
     args.out = (__nv_bfloat16*)out;
     args.N = d.N; args.H = d.H;
+    args.dual = d.N <= BQ ? 1 : 0;
+    args.per = args.dual ? (d.H + 1) / 2 : (d.N + 2 * BQ - 1) / (2 * BQ);
+    const long long items = (long long)args.per * (args.dual ? d.B : (long long)d.B * d.H);
+    if (items >= (1ll << 31)) return cudaErrorInvalidValue;
+    args.n_items = (int)items;
     const float scale = d.scale != 0.f ? d.scale : 0.125f;
     args.scale_log2 = scale * 1.4426950408889634f;
     args.status = ctx->d_status;
-    const dim3 grid((d.N + 2 * BQ - 1) / (2 * BQ), d.H, d.B);
+    // Short items: one resident CTA per SM walks the item list, so set-up, loads and epilogues
+    // overlap across items.  Long items (many key tiles) amortise their own set-up and gain more
+    // from the hardware handing the next item to whichever SM is free first.
+    const int nkv = (d.N + BKV - 1) / BKV;
+    const int grid = (nkv >= 16 || args.n_items < ctx->sm_count) ? args.n_items : ctx->sm_count;
     attn_tc_kernel<<<grid, kThreads, kSmem, st>>>(tmQ, tmK, tmV, args);
     return cudaGetLastError();
 }

@@ -153,6 +153,60 @@ select_kernel(const float* __restrict__ scores, int nparts, float* __restrict__ 
         if (keys[i]) { if (pos < K) out[pos] = i; ++pos; }
 }
 
+// Selection for N <= 1024: one token per thread, rank by counting.  Token i outranks token j
+// iff key_i > key_j, or the keys are equal and i < j (the same order the radix path realises),
+// so rank_i = #{j : j outranks i} and the K - first best-ranked candidates are kept.  N broadcast
+// reads of shared memory per thread replace the four histogram passes and their barriers: at
+// ViT token counts this is latency, not work.
+__global__ void __launch_bounds__(1024)
+select_small_kernel(const float* __restrict__ scores, int nparts, float* __restrict__ scores_out, int N,
+                    int K, int has_cls, int32_t* __restrict__ keep_idx) {
+    __shared__ uint32_t keys[1024];
+    __shared__ int wsum[32];
+    __shared__ int sh_total;
+    const int b = blockIdx.x, i = threadIdx.x;
+    const int first = has_cls ? 1 : 0, want = K - first;
+    uint32_t key = 0;
+    if (i < N) {
+        float s;
+        if (nparts > 0) {                  // fixed-order sum of the per-tile partial sums of squares
+            const float* p = scores + ((long long)b * N + i) * nparts;
+            float acc = 0.f;
+            for (int j = 0; j < nparts; ++j) acc += p[j];
+            s = sqrtf(acc);
+            if (scores_out) scores_out[(long long)b * N + i] = s;
+        } else {
+            s = scores[(long long)b * N + i];
+        }
+        key = score_key(s);
+        keys[i] = key;
+    }
+    __syncthreads();
+    int keep = 0;
+    if (i < N) {
+        if (i < first) {
+            keep = 1;
+        } else if (want > 0) {
+            int rank = 0;
+            int j = first;
+            for (; j + 4 <= N; j += 4) {   // keys[j] is a broadcast read: every thread reads the same word
+                const uint32_t k0 = keys[j], k1 = keys[j + 1], k2 = keys[j + 2], k3 = keys[j + 3];
+                rank += (k0 > key) || (k0 == key && j < i);
+                rank += (k1 > key) || (k1 == key && j + 1 < i);
+                rank += (k2 > key) || (k2 == key && j + 2 < i);
+                rank += (k3 > key) || (k3 == key && j + 3 < i);
+            }
+            for (; j < N; ++j) {
+                const uint32_t k0 = keys[j];
+                rank += (k0 > key) || (k0 == key && j < i);
+            }
+            keep = rank < want;
+        }
+    }
+    const int pos = block_exclusive_scan(keep, wsum, &sh_total);
+    if (keep && pos < K) keep_idx[(long long)b * K + pos] = i;
+}
+
 // x_out[b, j, :] = x[b, keep_idx[b, j], :]; one warp per kept row, 16-byte vectors,
 // all loads of a row issued before the first store.
 template <int MAXV>
@@ -192,6 +246,10 @@ cudaError_t select_init() {
 cudaError_t launch_select(const float* scores, int nparts, float* scores_out, int B, int N, int K,
                           int has_cls, int32_t* keep_idx, cudaStream_t st) {
     if (B == 0) return cudaSuccess;
+    if (N <= 1024) {
+        select_small_kernel<<<B, (N + 31) / 32 * 32, 0, st>>>(scores, nparts, scores_out, N, K, has_cls, keep_idx);
+        return cudaGetLastError();
+    }
     select_kernel<<<B, kSelThreads, select_smem_bytes(N), st>>>(scores, nparts, scores_out, N, K, has_cls,
                                                                keep_idx);
     return cudaGetLastError();

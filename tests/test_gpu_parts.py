@@ -83,7 +83,7 @@ def _scores(B, N, kind, seed):
 
 
 @pytest.mark.parametrize("kind", ["normal", "ties", "signed", "special", "equal"])
-@pytest.mark.parametrize("N", [1, 2, 17, 127, 128, 129, 197, 208, 257, 513, 1569, 4097])
+@pytest.mark.parametrize("N", [1, 2, 17, 127, 128, 129, 197, 208, 257, 513, 1024, 1025, 1569, 4097])
 def test_topk_compact_bit_exact(ctx, kind, N):
     B, D = 3, 64
     s = _scores(B, N, kind, N)
