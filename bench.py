@@ -202,14 +202,16 @@ def run_gpu(args, wl):
         barrier()
         return ms
 
+    use_graph = not args.no_graph
+
     def step_resident(i):
-        model.forward(dev_x[i % NBUF])
+        model.forward(dev_x[i % NBUF], graph=use_graph)
 
     dx = torch.empty_like(dev_x[0])
 
     def step_e2e(i):
         dx.copy_(host_x[i % NBUF], non_blocking=True)
-        outs = model.forward(dx)
+        outs = model.forward(dx, graph=use_graph)
         host_out.copy_(outs[-1]["x_out"], non_blocking=True)
 
     for i in range(max(args.warmup, 3)):
@@ -222,6 +224,8 @@ def run_gpu(args, wl):
     n0 = ctx.launch_count()
     ms = timed(step_resident, args.steps)
     launches = ctx.launch_count() - n0
+    if use_graph:      # replays do not pass through the library's counter: kernels per captured forward x steps
+        launches = model.launches_per_forward(wl.B, wl.N, wl.D) * args.steps
     clocks = sampler.stop() if rank == 0 else None
 
     for i in range(3):
@@ -232,7 +236,7 @@ def run_gpu(args, wl):
     ctx.timing_enable(True)
     tsteps = min(args.steps, 5)
     for i in range(tsteps):
-        step_resident(i)
+        model.forward(dev_x[i % NBUF])        # eager: the per-launch events are recorded by the library
     per = ctx.timing_read()
     ctx.timing_enable(False)
     ctx.async_status()
@@ -281,7 +285,7 @@ def run_gpu(args, wl):
     line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=max(args.warmup, 3),
                 ms_per_step=ms, higher_is_better=True, scaling="weak", vs_baseline=None,
                 dtype=("bf16" if wl.dtype == "bf16" else "f32"), data="synthetic",
-                config=workload_config(wl, wl.B), clocks=clocks,
+                config=dict(workload_config(wl, wl.B), launch=("CUDA graph replay, one graph per input buffer" if use_graph else "host launches")), clocks=clocks,
                 e2e=dict(value=aggregate_throughput(wl.B, ms_e2e, world), unit=UNIT,
                          h2d_bytes_per_step=host_x[0].numel() * host_x[0].element_size(),
                          d2h_bytes_per_step=host_out.numel() * host_out.element_size(), ms_per_step=ms_e2e),
@@ -296,11 +300,12 @@ def run_gpu(args, wl):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=300)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="vit_b16")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="launch every kernel from the host instead of replaying a CUDA graph")
     args = ap.parse_args()
     from paper_2508_00367_b200 import synth
     wl = synth.WORKLOADS[args.workload]

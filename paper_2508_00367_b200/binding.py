@@ -369,10 +369,42 @@ class PrunedViT:
         self._plan = dict(key=key, descs=descs, outs=outs, ws=ws)
         return self._plan
 
-    def forward(self, x: torch.Tensor):
-        """x: [B, N, D] on the device.  Returns the list of per-block outputs."""
+    def forward(self, x: torch.Tensor, graph: bool = False):
+        """x: [B, N, D] on the device.  Returns the list of per-block outputs (buffers owned by
+        the plan and overwritten by the next call).
+
+        graph=True replays the whole layer loop as one CUDA graph, captured on first use for
+        this input buffer (the graph reads x at its address: pass the same tensor again, or a
+        few fixed ones).  The first call for a shape must come outside any capture: it runs the
+        loop once eagerly so that every kernel's one-time set-up has happened."""
         B, N, D = x.shape
         p = self.plan(B, N, D)
+        if not graph:
+            self._run(x, p)
+            return p["outs"]
+        graphs = p.setdefault("graphs", {})
+        key = (x.data_ptr(), torch.cuda.current_stream(x.device).cuda_stream)
+        g = graphs.get(key)
+        if g is None:
+            if not p.get("warm"):
+                self._run(x, p)
+                torch.cuda.synchronize(x.device)
+                p["warm"] = True
+            n0 = self.ctx.launch_count()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                self._run(x, p)
+            p["launches_per_forward"] = self.ctx.launch_count() - n0
+            graphs[key] = (g, x)          # keep x alive: the graph holds its address
+            g = graphs[key]
+        g[0].replay()
+        return p["outs"]
+
+    def launches_per_forward(self, B: int, N: int, D: int) -> int:
+        """Kernels one forward pass launches (known once a graph was captured for the shape)."""
+        return int(self.plan(B, N, D).get("launches_per_forward", 0))
+
+    def _run(self, x: torch.Tensor, p):
         lib, h = self.ctx.lib, self.ctx.handle
         st = _stream(x.device)
         cur = x
@@ -384,4 +416,3 @@ class PrunedViT:
             if rc != RS_OK:
                 raise RsError(rc, self.ctx.last_error())
             cur = o["x_out"]
-        return p["outs"]
