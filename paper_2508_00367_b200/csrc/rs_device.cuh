@@ -6,12 +6,24 @@
 
 namespace rs {
 
+// 16-byte read of data that is used once: read-only path, no L1 allocation.
+__device__ __forceinline__ uint4 ld_stream(const uint4* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ float4 ld_stream(const float4* p) {
+    const uint4 v = ld_stream(reinterpret_cast<const uint4*>(p));
+    return make_float4(__uint_as_float(v.x), __uint_as_float(v.y), __uint_as_float(v.z), __uint_as_float(v.w));
+}
+
 template <typename T> struct Vec16;           // one 16-byte vector of T
 template <> struct Vec16<float> {
     static constexpr int N = 4;
     float v[4];
     __device__ __forceinline__ void load(const float* p) {
-        float4 t = *reinterpret_cast<const float4*>(p);
+        float4 t = ld_stream(reinterpret_cast<const float4*>(p));
         v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
     }
     __device__ __forceinline__ void store(float* p) const {
@@ -22,7 +34,7 @@ template <> struct Vec16<__nv_bfloat16> {
     static constexpr int N = 8;
     float v[8];
     __device__ __forceinline__ void load(const __nv_bfloat16* p) {
-        uint4 t = *reinterpret_cast<const uint4*>(p);
+        uint4 t = ld_stream(reinterpret_cast<const uint4*>(p));
         const uint32_t w[4] = {t.x, t.y, t.z, t.w};
 #pragma unroll
         for (int i = 0; i < 4; ++i) {

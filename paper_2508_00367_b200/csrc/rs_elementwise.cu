@@ -90,8 +90,24 @@ layernorm_kernel(const TI* __restrict__ x, const float* __restrict__ gamma,
 
 // ---------------------------------------------------------------- shift score
 // s = D(F(x), x) per token (Sec. 3.2); DIST 0: L2, 1: L1, 2: cosine distance.
+// One warp per token.  The 16-byte pieces stay packed in registers until they are reduced, so
+// that eight loads per lane are in flight at about 48 registers per thread and enough warps
+// fit an SM to cover the HBM latency.
+template <typename T> __device__ __forceinline__ void unpack16(const uint4& r, float (&v)[Vec16<T>::N]);
+template <> __device__ __forceinline__ void unpack16<float>(const uint4& r, float (&v)[4]) {
+    v[0] = __uint_as_float(r.x); v[1] = __uint_as_float(r.y); v[2] = __uint_as_float(r.z); v[3] = __uint_as_float(r.w);
+}
+template <> __device__ __forceinline__ void unpack16<__nv_bfloat16>(const uint4& r, float (&v)[8]) {
+    const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        v[2 * i] = __uint_as_float(w[i] << 16);
+        v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+    }
+}
+
 template <typename T, int DIST>
-__global__ void __launch_bounds__(kWarpsPerCta * 32)
+__global__ void __launch_bounds__(kWarpsPerCta * 32, 5)
 shift_score_kernel(const T* __restrict__ after, const T* __restrict__ before, long long rows, int D,
                    float* __restrict__ scores) {
     constexpr int VN = Vec16<T>::N;
@@ -100,28 +116,31 @@ shift_score_kernel(const T* __restrict__ after, const T* __restrict__ before, lo
     const long long row = (long long)blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5);
     if (row >= rows) return;
     const int nvec = D / VN;
-    const T* a = after + row * D;
-    const T* b = before + row * D;
+    const uint4* a = reinterpret_cast<const uint4*>(after + row * D);
+    const uint4* b = reinterpret_cast<const uint4*>(before + row * D);
     float acc = 0.f, aa = 0.f, bb = 0.f;
     for (int base = 0; base < nvec; base += 32 * UNROLL) {
-        Vec16<T> va[UNROLL], vb[UNROLL];
+        uint4 ra[UNROLL], rb[UNROLL];
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u) {
             const int iv = base + u * 32 + lane;
-            if (iv < nvec) { va[u].load(a + iv * VN); vb[u].load(b + iv * VN); }
+            if (iv < nvec) { ra[u] = ld_stream(a + iv); rb[u] = ld_stream(b + iv); }
         }
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u) {
             const int iv = base + u * 32 + lane;
             if (iv < nvec) {
+                float va[VN], vb[VN];
+                unpack16<T>(ra[u], va);
+                unpack16<T>(rb[u], vb);
 #pragma unroll
                 for (int e = 0; e < VN; ++e) {
-                    if (DIST == 0) { const float d = va[u].v[e] - vb[u].v[e]; acc = fmaf(d, d, acc); }
-                    else if (DIST == 1) { acc += fabsf(va[u].v[e] - vb[u].v[e]); }
+                    if (DIST == 0) { const float d = va[e] - vb[e]; acc = fmaf(d, d, acc); }
+                    else if (DIST == 1) { acc += fabsf(va[e] - vb[e]); }
                     else {
-                        acc = fmaf(va[u].v[e], vb[u].v[e], acc);
-                        aa = fmaf(va[u].v[e], va[u].v[e], aa);
-                        bb = fmaf(vb[u].v[e], vb[u].v[e], bb);
+                        acc = fmaf(va[e], vb[e], acc);
+                        aa = fmaf(va[e], va[e], aa);
+                        bb = fmaf(vb[e], vb[e], bb);
                     }
                 }
             }

@@ -207,6 +207,22 @@ select_small_kernel(const float* __restrict__ scores, int nparts, float* __restr
     if (keep && pos < K) keep_idx[(long long)b * K + pos] = i;
 }
 
+// Nothing dropped (K == N): every token is kept, in order; only the scores remain to be
+// finished when they arrive as per-tile partial sums of squares.
+__global__ void __launch_bounds__(256)
+keep_all_kernel(const float* __restrict__ scores, int nparts, float* __restrict__ scores_out, long long T, int N,
+                int32_t* __restrict__ keep_idx) {
+    const long long t = (long long)blockIdx.x * 256 + threadIdx.x;
+    if (t >= T) return;
+    if (nparts > 0 && scores_out) {
+        const float* p = scores + t * nparts;
+        float acc = 0.f;
+        for (int j = 0; j < nparts; ++j) acc += p[j];
+        scores_out[t] = sqrtf(acc);
+    }
+    keep_idx[t] = (int32_t)(t % N);
+}
+
 // x_out[b, j, :] = x[b, keep_idx[b, j], :]; one warp per kept row, 16-byte vectors,
 // all loads of a row issued before the first store.
 template <int MAXV>
@@ -246,6 +262,11 @@ cudaError_t select_init() {
 cudaError_t launch_select(const float* scores, int nparts, float* scores_out, int B, int N, int K,
                           int has_cls, int32_t* keep_idx, cudaStream_t st) {
     if (B == 0) return cudaSuccess;
+    if (K == N) {
+        const long long T = (long long)B * N;
+        keep_all_kernel<<<(unsigned)((T + 255) / 256), 256, 0, st>>>(scores, nparts, scores_out, T, N, keep_idx);
+        return cudaGetLastError();
+    }
     if (N <= 1024) {
         select_small_kernel<<<B, (N + 31) / 32 * 32, 0, st>>>(scores, nparts, scores_out, N, K, has_cls, keep_idx);
         return cudaGetLastError();
