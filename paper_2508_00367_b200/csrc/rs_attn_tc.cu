@@ -18,6 +18,7 @@
 #include <math.h>
 
 #include "rs_internal.h"
+#include "rs_device.cuh"
 #include "rs_tc.cuh"
 
 namespace rs {
@@ -204,6 +205,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    // Everything above touched no global memory and may overlap the previous kernel's tail.
+    grid_dep_launch();
+    grid_dep_wait();
     // The third warpgroup (TMA, MMA and two idle warps) hands most of its registers to the
     // two softmax warpgroups, which hold a whole 128-column row of S per thread.
     if (warp >= 8) {
@@ -509,8 +513,7 @@ cudaError_t launch_attn_tc(rs_ctx* ctx, const rs_attn_desc& d, const void* q, co
     // from the hardware handing the next item to whichever SM is free first.
     const int nkv = (d.N + BKV - 1) / BKV;
     const int grid = (nkv >= 16 || args.n_items < ctx->sm_count) ? args.n_items : ctx->sm_count;
-    attn_tc_kernel<<<grid, kThreads, kSmem, st>>>(tmQ, tmK, tmV, args);
-    return cudaGetLastError();
+    return launch_pdl(attn_tc_kernel, dim3(grid), dim3(kThreads), kSmem, st, tmQ, tmK, tmV, args);
 }
 
 }  // namespace rs

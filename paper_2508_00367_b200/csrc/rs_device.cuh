@@ -6,6 +6,14 @@
 
 namespace rs {
 
+// Programmatic dependent launch: a kernel launched with the programmatic-serialization attribute
+// may start while its predecessor in the stream is still draining.  grid_dep_launch() lets the
+// successor be scheduled early; grid_dep_wait() blocks until the predecessor has completed and
+// its writes are visible, and must come before the first access to global memory.  Both are
+// no-ops for a kernel launched the ordinary way.
+__device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // 16-byte read of data that is used once: read-only path, no L1 allocation.
 __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
     uint4 v;

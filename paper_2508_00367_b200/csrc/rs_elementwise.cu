@@ -41,6 +41,8 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32)
 layernorm_kernel(const TI* __restrict__ x, const float* __restrict__ gamma,
                  const float* __restrict__ beta, float eps, long long T, int D, TO* __restrict__ out) {
     constexpr int VN = Vec16<TI>::N;
+    grid_dep_launch();
+    grid_dep_wait();
     const int lane = threadIdx.x & 31;
     const long long row = (long long)blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5);
     if (row >= T) return;
@@ -112,6 +114,8 @@ shift_score_kernel(const T* __restrict__ after, const T* __restrict__ before, lo
                    float* __restrict__ scores) {
     constexpr int VN = Vec16<T>::N;
     constexpr int UNROLL = 4;
+    grid_dep_launch();
+    grid_dep_wait();
     const int lane = threadIdx.x & 31;
     const long long row = (long long)blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5);
     if (row >= rows) return;
@@ -197,12 +201,10 @@ cudaError_t ln_dispatch(const void* x, const float* g, const float* b, float eps
     const int nvec = D / Vec16<TI>::N;
     const dim3 grid(row_grid(T)), block(kWarpsPerCta * 32);
     if (nvec <= 32 * 4)
-        layernorm_kernel<TI, TO, 4><<<grid, block, 0, st>>>((const TI*)x, g, b, eps, T, D, (TO*)out);
+        return launch_pdl(layernorm_kernel<TI, TO, 4>, grid, block, 0, st, (const TI*)x, g, b, eps, T, D, (TO*)out);
     else if (nvec <= 32 * 8)
-        layernorm_kernel<TI, TO, 8><<<grid, block, 0, st>>>((const TI*)x, g, b, eps, T, D, (TO*)out);
-    else
-        return cudaErrorInvalidValue;
-    return cudaGetLastError();
+        return launch_pdl(layernorm_kernel<TI, TO, 8>, grid, block, 0, st, (const TI*)x, g, b, eps, T, D, (TO*)out);
+    return cudaErrorInvalidValue;
 }
 
 }  // namespace
@@ -222,7 +224,7 @@ cudaError_t launch_shift_score(rs_dtype dtype, rs_dist dist, long long T, int D,
     if (T == 0) return cudaSuccess;
     const dim3 grid(row_grid(T)), block(kWarpsPerCta * 32);
 #define RS_SCORE_CASE(TT, DD)                                                                   \
-    shift_score_kernel<TT, DD><<<grid, block, 0, st>>>((const TT*)after, (const TT*)before, T, D, scores)
+    return launch_pdl(shift_score_kernel<TT, DD>, grid, block, 0, st, (const TT*)after, (const TT*)before, T, D, scores)
     if (dtype == RS_BF16) {
         if (dist == RS_DIST_L2) RS_SCORE_CASE(__nv_bfloat16, 0);
         else if (dist == RS_DIST_L1) RS_SCORE_CASE(__nv_bfloat16, 1);

@@ -17,6 +17,7 @@
 //   EPI_SCORE      m = acc + b;  out = m + x';  partial sums of (m - x')^2 (or m^2) per row
 //                                                          -> bf16/fp32 (FC2 + residual + shift score)
 #include "rs_internal.h"
+#include "rs_device.cuh"
 #include "rs_tc.cuh"
 
 namespace rs {
@@ -120,6 +121,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     cluster_sync();                              // the peer's barriers exist before anything signals them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    // Everything above touched no global memory and may overlap the previous kernel's tail.
+    grid_dep_launch();
+    grid_dep_wait();
 
     if (warp == 0) {
         // ---------------- TMA producer (both CTAs; each loads its own halves) ----------------
@@ -355,13 +359,15 @@ cudaError_t launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUt
     cfg.blockDim = dim3(kThreads, 1, 1);
     cfg.dynamicSmemBytes = C::SMEM;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // see grid_dep_wait() in the kernel
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<BN, EPI, OutT>, tmA, tmB, tmOut, args);
 }
 

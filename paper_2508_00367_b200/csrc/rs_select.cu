@@ -62,6 +62,8 @@ select_kernel(const float* __restrict__ scores, int nparts, float* __restrict__ 
     __shared__ int wsum[32];
     __shared__ int sh_bin, sh_remaining, sh_total;
 
+    grid_dep_launch();
+    grid_dep_wait();
     const int b = blockIdx.x;
     const int tid = threadIdx.x;
     const int first = has_cls ? 1 : 0;     // token 0 is kept unconditionally when has_cls
@@ -164,6 +166,8 @@ select_small_kernel(const float* __restrict__ scores, int nparts, float* __restr
     __shared__ uint32_t keys[1024];
     __shared__ int wsum[32];
     __shared__ int sh_total;
+    grid_dep_launch();
+    grid_dep_wait();
     const int b = blockIdx.x, i = threadIdx.x;
     const int first = has_cls ? 1 : 0, want = K - first;
     uint32_t key = 0;
@@ -212,6 +216,8 @@ select_small_kernel(const float* __restrict__ scores, int nparts, float* __restr
 __global__ void __launch_bounds__(256)
 keep_all_kernel(const float* __restrict__ scores, int nparts, float* __restrict__ scores_out, long long T, int N,
                 int32_t* __restrict__ keep_idx) {
+    grid_dep_launch();
+    grid_dep_wait();
     const long long t = (long long)blockIdx.x * 256 + threadIdx.x;
     if (t >= T) return;
     if (nparts > 0 && scores_out) {
@@ -229,6 +235,8 @@ template <int MAXV>
 __global__ void __launch_bounds__(256)
 gather_kernel(const uint4* __restrict__ x, const int32_t* __restrict__ keep_idx, long long rows, int N,
               int K, int row_vecs, uint4* __restrict__ x_out) {
+    grid_dep_launch();
+    grid_dep_wait();
     const int lane = threadIdx.x & 31;
     const long long row = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
     if (row >= rows) return;
@@ -264,16 +272,13 @@ cudaError_t launch_select(const float* scores, int nparts, float* scores_out, in
     if (B == 0) return cudaSuccess;
     if (K == N) {
         const long long T = (long long)B * N;
-        keep_all_kernel<<<(unsigned)((T + 255) / 256), 256, 0, st>>>(scores, nparts, scores_out, T, N, keep_idx);
-        return cudaGetLastError();
+        return launch_pdl(keep_all_kernel, dim3((unsigned)((T + 255) / 256)), dim3(256), 0, st, scores, nparts, scores_out, T, N, keep_idx);
     }
     if (N <= 1024) {
-        select_small_kernel<<<B, (N + 31) / 32 * 32, 0, st>>>(scores, nparts, scores_out, N, K, has_cls, keep_idx);
-        return cudaGetLastError();
+        return launch_pdl(select_small_kernel, dim3(B), dim3((N + 31) / 32 * 32), 0, st, scores, nparts, scores_out, N, K, has_cls, keep_idx);
     }
-    select_kernel<<<B, kSelThreads, select_smem_bytes(N), st>>>(scores, nparts, scores_out, N, K, has_cls,
-                                                               keep_idx);
-    return cudaGetLastError();
+    return launch_pdl(select_kernel, dim3(B), dim3(kSelThreads), select_smem_bytes(N), st, scores, nparts, scores_out, N, K,
+                      has_cls, keep_idx);
 }
 
 cudaError_t launch_gather(rs_dtype dtype, const void* x, const int32_t* keep_idx, int B, int N, int K,
@@ -282,8 +287,8 @@ cudaError_t launch_gather(rs_dtype dtype, const void* x, const int32_t* keep_idx
     if (rows == 0) return cudaSuccess;
     const int row_vecs = (int)((size_t)D * dtype_size(dtype) / 16);
     const unsigned grid = (unsigned)((rows + 7) / 8);
-    gather_kernel<4><<<grid, 256, 0, st>>>((const uint4*)x, keep_idx, rows, N, K, row_vecs, (uint4*)x_out);
-    return cudaGetLastError();
+    return launch_pdl(gather_kernel<4>, dim3(grid), dim3(256), 0, st, (const uint4*)x, keep_idx, rows, N, K, row_vecs,
+                      (uint4*)x_out);
 }
 
 }  // namespace rs
