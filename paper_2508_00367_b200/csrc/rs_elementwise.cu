@@ -34,67 +34,7 @@ template <> __device__ __forceinline__ void store_n<__nv_bfloat16, 8>(__nv_bfloa
     *reinterpret_cast<uint4*>(p) = make_uint4(w[0], w[1], w[2], w[3]);
 }
 
-// ---------------------------------------------------------------- LayerNorm
-// LN of Eq. att / Eq. MLP: mean and biased variance over D, then affine.
-template <typename TI, typename TO, int MAXV>
-__global__ void __launch_bounds__(kWarpsPerCta * 32)
-layernorm_kernel(const TI* __restrict__ x, const float* __restrict__ gamma,
-                 const float* __restrict__ beta, float eps, long long T, int D, TO* __restrict__ out) {
-    constexpr int VN = Vec16<TI>::N;
-    grid_dep_launch();
-    grid_dep_wait();
-    const int lane = threadIdx.x & 31;
-    const long long row = (long long)blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5);
-    if (row >= T) return;
-    const int nvec = D / VN;
-    const TI* xr = x + row * D;
-    Vec16<TI> v[MAXV];
-    float sum = 0.f;
-#pragma unroll
-    for (int j = 0; j < MAXV; ++j) {
-        const int iv = j * 32 + lane;
-        if (iv < nvec) {
-            v[j].load(xr + iv * VN);
-#pragma unroll
-            for (int e = 0; e < VN; ++e) sum += v[j].v[e];
-        }
-    }
-    const float mu = warp_sum(sum) / (float)D;
-    float sq = 0.f;
-#pragma unroll
-    for (int j = 0; j < MAXV; ++j) {
-        const int iv = j * 32 + lane;
-        if (iv < nvec) {
-#pragma unroll
-            for (int e = 0; e < VN; ++e) { const float d = v[j].v[e] - mu; sq += d * d; }
-        }
-    }
-    const float rstd = rsqrtf(warp_sum(sq) / (float)D + eps);
-    TO* orow = out + row * D;
-#pragma unroll
-    for (int j = 0; j < MAXV; ++j) {
-        const int iv = j * 32 + lane;
-        if (iv < nvec) {
-            float y[VN];
-#pragma unroll
-            for (int e = 0; e < VN; e += 4) {
-                const float4 g = *reinterpret_cast<const float4*>(gamma + iv * VN + e);
-                const float4 b = *reinterpret_cast<const float4*>(beta + iv * VN + e);
-                y[e + 0] = (v[j].v[e + 0] - mu) * rstd * g.x + b.x;
-                y[e + 1] = (v[j].v[e + 1] - mu) * rstd * g.y + b.y;
-                y[e + 2] = (v[j].v[e + 2] - mu) * rstd * g.z + b.z;
-                y[e + 3] = (v[j].v[e + 3] - mu) * rstd * g.w + b.w;
-            }
-            store_n<TO, VN>(orow + iv * VN, y);
-        }
-    }
-}
-
-// ---------------------------------------------------------------- shift score
-// s = D(F(x), x) per token (Sec. 3.2); DIST 0: L2, 1: L1, 2: cosine distance.
-// One warp per token.  The 16-byte pieces stay packed in registers until they are reduced, so
-// that eight loads per lane are in flight at about 48 registers per thread and enough warps
-// fit an SM to cover the HBM latency.
+// 16 bytes of T as floats.
 template <typename T> __device__ __forceinline__ void unpack16(const uint4& r, float (&v)[Vec16<T>::N]);
 template <> __device__ __forceinline__ void unpack16<float>(const uint4& r, float (&v)[4]) {
     v[0] = __uint_as_float(r.x); v[1] = __uint_as_float(r.y); v[2] = __uint_as_float(r.z); v[3] = __uint_as_float(r.w);
@@ -108,6 +48,76 @@ template <> __device__ __forceinline__ void unpack16<__nv_bfloat16>(const uint4&
     }
 }
 
+// ---------------------------------------------------------------- LayerNorm
+// LN of Eq. att / Eq. MLP: mean and biased variance over D, then affine.  One warp per row; the
+// row stays in registers as packed 16-byte pieces (unpacked once per pass over it), which keeps
+// the kernel at 48 to 64 registers so that four or five CTAs per SM cover the memory latency.
+template <typename TI, typename TO, int MAXV>
+__global__ void __launch_bounds__(kWarpsPerCta * 32, MAXV <= 4 ? 5 : 4)
+layernorm_kernel(const TI* __restrict__ x, const float* __restrict__ gamma,
+                 const float* __restrict__ beta, float eps, long long T, int D, TO* __restrict__ out) {
+    constexpr int VN = Vec16<TI>::N;
+    grid_dep_launch();
+    grid_dep_wait();
+    const int lane = threadIdx.x & 31;
+    const long long row = (long long)blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5);
+    if (row >= T) return;
+    const int nvec = D / VN;
+    const uint4* xr = reinterpret_cast<const uint4*>(x + row * D);
+    uint4 raw[MAXV];
+#pragma unroll
+    for (int j = 0; j < MAXV; ++j) {
+        const int iv = j * 32 + lane;
+        if (iv < nvec) raw[j] = ld_stream(xr + iv);
+    }
+    float sum = 0.f;
+#pragma unroll
+    for (int j = 0; j < MAXV; ++j) {
+        if (j * 32 + lane < nvec) {
+            float v[VN];
+            unpack16<TI>(raw[j], v);
+#pragma unroll
+            for (int e = 0; e < VN; ++e) sum += v[e];
+        }
+    }
+    const float mu = warp_sum(sum) / (float)D;
+    float sq = 0.f;
+#pragma unroll
+    for (int j = 0; j < MAXV; ++j) {
+        if (j * 32 + lane < nvec) {
+            float v[VN];
+            unpack16<TI>(raw[j], v);
+#pragma unroll
+            for (int e = 0; e < VN; ++e) { const float dd = v[e] - mu; sq += dd * dd; }
+        }
+    }
+    const float rstd = rsqrtf(warp_sum(sq) / (float)D + eps);
+    TO* orow = out + row * D;
+#pragma unroll
+    for (int j = 0; j < MAXV; ++j) {
+        const int iv = j * 32 + lane;
+        if (iv < nvec) {
+            float v[VN], y[VN];
+            unpack16<TI>(raw[j], v);
+#pragma unroll
+            for (int e = 0; e < VN; e += 4) {
+                const float4 g = __ldg(reinterpret_cast<const float4*>(gamma + iv * VN + e));
+                const float4 bt = __ldg(reinterpret_cast<const float4*>(beta + iv * VN + e));
+                y[e + 0] = (v[e + 0] - mu) * rstd * g.x + bt.x;
+                y[e + 1] = (v[e + 1] - mu) * rstd * g.y + bt.y;
+                y[e + 2] = (v[e + 2] - mu) * rstd * g.z + bt.z;
+                y[e + 3] = (v[e + 3] - mu) * rstd * g.w + bt.w;
+            }
+            store_n<TO, VN>(orow + iv * VN, y);
+        }
+    }
+}
+
+// ---------------------------------------------------------------- shift score
+// s = D(F(x), x) per token (Sec. 3.2); DIST 0: L2, 1: L1, 2: cosine distance.
+// One warp per token.  The 16-byte pieces stay packed in registers until they are reduced, so
+// that eight loads per lane are in flight at about 48 registers per thread and enough warps
+// fit an SM to cover the HBM latency.
 template <typename T, int DIST>
 __global__ void __launch_bounds__(kWarpsPerCta * 32, 5)
 shift_score_kernel(const T* __restrict__ after, const T* __restrict__ before, long long rows, int D,
