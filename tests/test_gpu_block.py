@@ -177,3 +177,24 @@ def test_model_free_running_matches_until_first_swap(ctx):
             assert err.max() <= 0.125   # a handful of elements sit several ulps off by block 4
             compared += 1
     assert compared >= 2
+
+
+def test_graph_replay_equals_eager(ctx):
+    """PrunedViT.forward(graph=True) replays the same kernels: outputs are bit-identical to the
+    eager loop, on a first and on a repeated replay."""
+    import paper_2508_00367_b200 as rs
+    from paper_2508_00367_b200 import synth
+    B, N, D, H, L = 3, 150, 256, 4, 3
+    x = synth.make_tokens(B, N, D, "bf16", seed=5).to(torch.bfloat16).cuda()
+    blocks = [synth.make_block_weights(D, 4 * D, "bf16", seed=10 + l) for l in range(L)]
+    model = rs.PrunedViT(ctx, blocks, H, [10, 0, 7], torch.bfloat16)
+    eager = [{k: v.clone() for k, v in o.items()} for o in model.forward(x)]
+    for _ in range(2):
+        outs = model.forward(x, graph=True)
+        torch.cuda.synchronize()
+        for a, b in zip(eager, outs):
+            assert torch.equal(a["keep_idx"], b["keep_idx"])
+            assert torch.equal(a["x_out"].view(torch.int16), b["x_out"].view(torch.int16))
+            assert torch.equal(a["scores"], b["scores"])
+    assert model.launches_per_forward(B, N, D) == 9 * L - 1      # the block that drops nothing has no gather
+    ctx.async_status()

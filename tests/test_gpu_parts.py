@@ -173,6 +173,19 @@ def test_attn_separate_buffers_scale_and_large_logits(ctx, dtype):
     parity.check_float(got, orc.round_to(want, dtype), dtype, rounded_output=True)
 
 
+def test_attn_full_size_video_shape_sampled(ctx):
+    # video ViT-L/14 token count (16 x 256 + 1), two heads of one sample; the oracle on sampled query rows
+    B, N, H = 1, 4097, 2
+    qkv = _tok((B, N, 3, H, 64), torch.bfloat16, 99)
+    dq = qkv.cuda()
+    got = ctx.attn_fwd(dq[:, :, 0], dq[:, :, 1], dq[:, :, 2]).cpu().double().numpy()
+    f = qkv.double().numpy()
+    rows = np.unique(np.concatenate([np.arange(0, 3), np.arange(126, 131), np.arange(N - 3, N),
+                                     np.random.default_rng(1).integers(0, N, 48)]))
+    want = orc.attn(f[:, :, 0], f[:, :, 1], f[:, :, 2]).reshape(B, N, H * 64)[:, rows]
+    parity.check_float(got[:, rows], orc.round_to(want, "bf16"), "bf16", rounded_output=True)
+
+
 def test_attn_rejects_bad_arguments(ctx):
     import paper_2508_00367_b200 as rs
     q = torch.zeros(1, 4, 2, 32, device="cuda")

@@ -103,3 +103,26 @@ def test_batch_sharding_two_ranks_gloo(tmp_path):
     for p, o in zip(procs, outs):
         assert p.returncode == 0, o
         assert "OK" in o
+
+
+def test_gelu_polynomial_matches_exact_erf_gelu():
+    """The FC1 epilogue's GELU constants come from csrc/fit_gelu.py: refit and check the bound
+    the kernel's comment states (fp32 Horner evaluation against the erf definition)."""
+    import importlib.util
+    import re
+    here = os.path.dirname(os.path.abspath(__file__))
+    csrc = os.path.join(os.path.dirname(here), "paper_2508_00367_b200", "csrc")
+    spec = importlib.util.spec_from_file_location("fit_gelu", os.path.join(csrc, "fit_gelu.py"))
+    fg = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(fg)
+    import numpy as np
+    coef = fg.fit()
+    assert fg.max_error_fp32(coef) < 1e-6
+    assert coef[-1] > 0                       # 2^-q -> 0 for large |v|
+    # the constants compiled into the kernel are these coefficients
+    src = open(os.path.join(csrc, "rs_gemm_tc.cu")).read()
+    body = src[src.index("float gelu_erf(float v)"):]
+    body = body[:body.index("return v *")]
+    consts = [float(m) for m in re.findall(r"(-?\d+\.\d+(?:e-?\d+)?)f", body)]
+    in_kernel = np.array(consts[:6][::-1], dtype=np.float64)     # Horner order is highest degree first
+    assert fg.max_error_fp32(in_kernel) < 1e-6
