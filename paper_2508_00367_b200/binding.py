@@ -19,7 +19,7 @@ LIB_PATH = os.path.join(_HERE, "librs.so")
 RS_OK = 0
 RS_F32, RS_BF16 = 0, 1
 DIST = {"l2": 0, "l1": 1, "cos": 2}
-SCORE_MODE = {"mlp": 0, "mlp_delta": 1}
+SCORE_MODE = {"mlp": 0, "mlp_delta": 1, "attn": 2, "block": 3}
 STATUS_NAMES = {0: "RS_OK", 1: "RS_ERR_INVALID_ARG", 2: "RS_ERR_UNSUPPORTED", 3: "RS_ERR_WORKSPACE",
                 4: "RS_ERR_CUDA", 5: "RS_ERR_TIMEOUT"}
 

@@ -172,12 +172,13 @@ shift_score_kernel(const T* __restrict__ after, const T* __restrict__ before, lo
 }
 
 // ---------------------------------------------------------------- residual add + score
-// x_hat = m + x' and s = |m - x'| (or |m|): the score rides on the residual-add
-// pass, which already has both operands in registers (Eq. MLP, Sec. 3.2).
-template <typename TO, int MODE>
+// x_hat = m + x' and the score of the chosen pair of representations (Sec. 3.3 "Operation
+// choice"): MODE 0 |m - x'| (ii), 1 |m|, 2 |SA(LN(x)) - x| = |x' - 2x| (i), 3 |x_hat - x| (iii).
+// The score rides on the residual-add pass, which already has the operands in registers.
+template <typename TO, typename TX, int MODE>
 __global__ void __launch_bounds__(kWarpsPerCta * 32)
-residual_score_kernel(const float* __restrict__ m, const float* __restrict__ xp, long long rows, int D,
-                      TO* __restrict__ x_hat, float* __restrict__ scores) {
+residual_score_kernel(const float* __restrict__ m, const float* __restrict__ xp, const TX* __restrict__ x0,
+                      long long rows, int D, TO* __restrict__ x_hat, float* __restrict__ scores) {
     const int lane = threadIdx.x & 31;
     const long long row = (long long)blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5);
     if (row >= rows) return;
@@ -186,16 +187,19 @@ residual_score_kernel(const float* __restrict__ m, const float* __restrict__ xp,
     for (int iv = lane; iv < nvec; iv += 32) {
         const float4 a = *reinterpret_cast<const float4*>(m + row * D + iv * 4);
         const float4 b = *reinterpret_cast<const float4*>(xp + row * D + iv * 4);
-        const float y[4] = {a.x + b.x, a.y + b.y, a.z + b.z, a.w + b.w};
-        if (MODE == 0) {
+        const float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
+        float y[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            y[e] = av[e] + bv[e];
             float d;
-            d = a.x - b.x; acc = fmaf(d, d, acc);
-            d = a.y - b.y; acc = fmaf(d, d, acc);
-            d = a.z - b.z; acc = fmaf(d, d, acc);
-            d = a.w - b.w; acc = fmaf(d, d, acc);
-        } else {
-            acc = fmaf(a.x, a.x, acc); acc = fmaf(a.y, a.y, acc);
-            acc = fmaf(a.z, a.z, acc); acc = fmaf(a.w, a.w, acc);
+            if (MODE == 0) d = av[e] - bv[e];
+            else if (MODE == 1) d = av[e];
+            else {
+                const float x = to_float(x0[row * D + iv * 4 + e]);
+                d = MODE == 2 ? bv[e] - 2.f * x : y[e] - x;
+            }
+            acc = fmaf(d, d, acc);
         }
         store_n<TO, 4>(x_hat + row * D + iv * 4, y);
     }
@@ -248,18 +252,27 @@ cudaError_t launch_shift_score(rs_dtype dtype, rs_dist dist, long long T, int D,
     return cudaGetLastError();
 }
 
-cudaError_t launch_residual_score(const float* m, const float* x_prime, long long T, int D,
-                                  rs_score_mode mode, rs_dtype out_dtype, void* x_hat, float* scores,
-                                  cudaStream_t st) {
+cudaError_t launch_residual_score(const float* m, const float* x_prime, const void* x, rs_dtype x_dtype,
+                                  long long T, int D, rs_score_mode mode, rs_dtype out_dtype, void* x_hat,
+                                  float* scores, cudaStream_t st) {
     if (T == 0) return cudaSuccess;
     const dim3 grid(row_grid(T)), block(kWarpsPerCta * 32);
+#define RS_RES_CASE(TO, TX, MD)                                                                                  \
+    residual_score_kernel<TO, TX, MD><<<grid, block, 0, st>>>(m, x_prime, (const TX*)x, T, D, (TO*)x_hat, scores)
+#define RS_RES_MODE(TO, TX)                                     \
+    do {                                                        \
+        if (mode == RS_SCORE_MLP) RS_RES_CASE(TO, TX, 0);       \
+        else if (mode == RS_SCORE_MLP_DELTA) RS_RES_CASE(TO, TX, 1); \
+        else if (mode == RS_SCORE_ATTN) RS_RES_CASE(TO, TX, 2); \
+        else RS_RES_CASE(TO, TX, 3);                            \
+    } while (0)
     if (out_dtype == RS_BF16) {
-        if (mode == RS_SCORE_MLP) residual_score_kernel<__nv_bfloat16, 0><<<grid, block, 0, st>>>(m, x_prime, T, D, (__nv_bfloat16*)x_hat, scores);
-        else residual_score_kernel<__nv_bfloat16, 1><<<grid, block, 0, st>>>(m, x_prime, T, D, (__nv_bfloat16*)x_hat, scores);
+        if (x_dtype == RS_BF16) RS_RES_MODE(__nv_bfloat16, __nv_bfloat16); else RS_RES_MODE(__nv_bfloat16, float);
     } else {
-        if (mode == RS_SCORE_MLP) residual_score_kernel<float, 0><<<grid, block, 0, st>>>(m, x_prime, T, D, (float*)x_hat, scores);
-        else residual_score_kernel<float, 1><<<grid, block, 0, st>>>(m, x_prime, T, D, (float*)x_hat, scores);
+        if (x_dtype == RS_BF16) RS_RES_MODE(float, __nv_bfloat16); else RS_RES_MODE(float, float);
     }
+#undef RS_RES_MODE
+#undef RS_RES_CASE
     return cudaGetLastError();
 }
 

@@ -13,8 +13,9 @@
 // Epilogues (Eq. att, Eq. MLP, Sec. 3.2):
 //   EPI_BIAS       out = acc + b                          -> bf16      (QKV projection)
 //   EPI_BIAS_GELU  out = GELU(acc + b)                    -> bf16      (FC1)
-//   EPI_RESID      out = acc + b + x                      -> fp32      (projection + residual = x')
-//   EPI_SCORE      m = acc + b;  out = m + x';  partial sums of (m - x')^2 (or m^2) per row
+//   EPI_RESID      a = acc + b;  out = a + x              -> fp32      (projection + residual = x');
+//                  optionally partial sums of (a - x)^2 per row    (shift through attention, choice (i))
+//   EPI_SCORE      m = acc + b;  out = m + x';  partial sums of (m - x')^2, m^2 or (out - x)^2 per row
 //                                                          -> bf16/fp32 (FC2 + residual + shift score)
 #include "rs_internal.h"
 #include "rs_device.cuh"
@@ -51,8 +52,9 @@ struct GemmArgs {
     int M, N, K;
     const float* bias;        // [N] or null
     const void* residual;     // EPI_RESID: bf16 [M, N];  EPI_SCORE: fp32 [M, N]
-    float* partials;          // EPI_SCORE: [M, 2 * N / BN] sums of squares
-    int score_delta;          // EPI_SCORE: 1 => sum m^2 instead of (m - x')^2
+    const void* residual2;    // EPI_SCORE, score_kind 2: bf16 [M, N] block input x
+    float* partials;          // EPI_SCORE (and EPI_RESID when non-null): [M, 2 * N / BN] sums of squares
+    int score_kind;           // EPI_SCORE: 0 => (m - x')^2, 1 => m^2, 2 => (m + x' - x)^2
     int* status;
 };
 
@@ -258,21 +260,49 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         const uint32_t w[4] = {res[j].x, res[j].y, res[j].z, res[j].w};
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
-                            v[8 * j + 2 * e] += __uint_as_float(w[e] << 16);
-                            v[8 * j + 2 * e + 1] += __uint_as_float(w[e] & 0xffff0000u);
+                            const float x0 = __uint_as_float(w[e] << 16), x1 = __uint_as_float(w[e] & 0xffff0000u);
+                            const float d0 = v[8 * j + 2 * e] - x0, d1 = v[8 * j + 2 * e + 1] - x1;   // SA(LN(x)) - x
+                            sq = fmaf(d0, d0, sq);
+                            sq = fmaf(d1, d1, sq);
+                            v[8 * j + 2 * e] += x0;
+                            v[8 * j + 2 * e + 1] += x1;
                         }
                     }
                 } else if (EPI == EPI_SCORE) {
+                    if (args.score_kind == 2) {
+                        // whole-block shift: x^ - x, with the block input x read here (rows past M: zeros)
+                        const uint4* x0p = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(args.residual2) +
+                                                                          (size_t)row * args.N + col);
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        const float xs[4] = {__uint_as_float(res[j].x), __uint_as_float(res[j].y),
-                                             __uint_as_float(res[j].z), __uint_as_float(res[j].w)};
+                        for (int j = 0; j < 4; ++j) {
+                            const uint4 xv = valid ? __ldg(x0p + j) : make_uint4(0u, 0u, 0u, 0u);
+                            const uint32_t w[4] = {xv.x, xv.y, xv.z, xv.w};
+                            const float xp[8] = {__uint_as_float(res[2 * j].x), __uint_as_float(res[2 * j].y),
+                                                 __uint_as_float(res[2 * j].z), __uint_as_float(res[2 * j].w),
+                                                 __uint_as_float(res[2 * j + 1].x), __uint_as_float(res[2 * j + 1].y),
+                                                 __uint_as_float(res[2 * j + 1].z), __uint_as_float(res[2 * j + 1].w)};
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const float m = v[4 * j + e];
-                            const float d = args.score_delta ? m : m - xs[e];
-                            sq = fmaf(d, d, sq);
-                            v[4 * j + e] = m + xs[e];
+                            for (int e = 0; e < 4; ++e) {
+                                const float xa = __uint_as_float(w[e] << 16), xb = __uint_as_float(w[e] & 0xffff0000u);
+                                const float ya = v[8 * j + 2 * e] + xp[2 * e], yb = v[8 * j + 2 * e + 1] + xp[2 * e + 1];
+                                sq = fmaf(ya - xa, ya - xa, sq);
+                                sq = fmaf(yb - xb, yb - xb, sq);
+                                v[8 * j + 2 * e] = ya;
+                                v[8 * j + 2 * e + 1] = yb;
+                            }
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            const float xs[4] = {__uint_as_float(res[j].x), __uint_as_float(res[j].y),
+                                                 __uint_as_float(res[j].z), __uint_as_float(res[j].w)};
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const float m = v[4 * j + e];
+                                const float d = args.score_kind ? m : m - xs[e];
+                                sq = fmaf(d, d, sq);
+                                v[4 * j + e] = m + xs[e];
+                            }
                         }
                     }
                 }
@@ -305,7 +335,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     ++blk_ctr;
                 }
             }
-            if (EPI == EPI_SCORE && valid)
+            if ((EPI == EPI_SCORE || (EPI == EPI_RESID && args.partials)) && valid)
                 args.partials[(size_t)row * (2 * num_n) + 2 * nt + half] = sq;
         }
         if (storer) tma_store_wait<0>();                 // all output written before the CTA exits
@@ -409,7 +439,7 @@ int gemm_tc_score_parts(const rs_ctx* ctx, long long M, int N) {
 }
 
 cudaError_t launch_gemm_tc(rs_ctx* ctx, int epi, const void* A, const void* W, const float* bias,
-                           const void* residual, void* out, rs_dtype out_dtype, float* partials, int score_delta,
+                           const void* residual, const void* residual2, void* out, rs_dtype out_dtype, float* partials, int score_kind,
                            long long M, int N, int K, cudaStream_t st) {
     if (!ctx->encode_tiled) return cudaErrorNotSupported;
     const int bn = pick_bn(M, N, ctx->sm_count);
@@ -421,7 +451,7 @@ cudaError_t launch_gemm_tc(rs_ctx* ctx, int epi, const void* A, const void* W, c
         return cudaErrorInvalidValue;
     GemmArgs args;
     args.M = (int)M; args.N = N; args.K = K; args.bias = bias; args.residual = residual;
-    args.partials = partials; args.score_delta = score_delta; args.status = ctx->d_status;
+    args.residual2 = residual2; args.partials = partials; args.score_kind = score_kind; args.status = ctx->d_status;
     const int sms = ctx->sm_count;
 #define RS_GEMM_CASE(E, T)                                                                       \
     return bn == 256   ? launch_one<256, E, T>(tmA, tmB, tmOut, args, sms, st)                  \

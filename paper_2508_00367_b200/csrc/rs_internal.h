@@ -60,10 +60,11 @@ cudaError_t launch_layernorm(rs_dtype in_dtype, rs_dtype out_dtype, const void* 
 cudaError_t launch_shift_score(rs_dtype dtype, rs_dist dist, long long T, int D, const void* after,
                                const void* before, float* scores, cudaStream_t st);
 // Residual-add epilogue with the score fused in: x_hat = m + x_prime (out_dtype);
-// s = |m - x_prime| (mode MLP) or |m| (mode MLP_DELTA).  m, x_prime fp32.
-cudaError_t launch_residual_score(const float* m, const float* x_prime, long long T, int D,
-                                  rs_score_mode mode, rs_dtype out_dtype, void* x_hat, float* scores,
-                                  cudaStream_t st);
+// s = |m - x_prime| (MLP), |m| (MLP_DELTA), |x_prime - 2 x| = |SA(LN(x)) - x| (ATTN) or
+// |x_hat - x| (BLOCK).  m, x_prime fp32; x (the block input, x_dtype) only for ATTN and BLOCK.
+cudaError_t launch_residual_score(const float* m, const float* x_prime, const void* x, rs_dtype x_dtype,
+                                  long long T, int D, rs_score_mode mode, rs_dtype out_dtype, void* x_hat,
+                                  float* scores, cudaStream_t st);
 
 // ---- selection and compaction (rs_select.cu) ----
 // scores: [B, N] fp32, or if nparts > 0 partial sums of squares [B*N, nparts] whose row
@@ -90,8 +91,8 @@ bool gemm_tc_supported(long long M, int N, int K);
 int gemm_tc_score_parts(const rs_ctx* ctx, long long M, int N);   // partial sums per row written by RS_EPI_SCORE
 // out[M, N] = epilogue(A[M, K] . W[N, K]^T); see rs_gemm_tc.cu for the epilogues.
 cudaError_t launch_gemm_tc(rs_ctx* ctx, int epi, const void* A, const void* W, const float* bias,
-                           const void* residual, void* out, rs_dtype out_dtype, float* partials,
-                           int score_delta, long long M, int N, int K, cudaStream_t st);
+                           const void* residual, const void* residual2, void* out, rs_dtype out_dtype,
+                           float* partials, int score_kind, long long M, int N, int K, cudaStream_t st);
 
 // ---- tcgen05 attention (rs_attn_tc.cu): bf16, head dimension 64 ----
 bool attn_tc_supported(const rs_attn_desc& d);

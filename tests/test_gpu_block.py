@@ -34,14 +34,16 @@ def _run_block(ctx, x, w, H, r, dtype, out_dtype=None, score_mode="mlp", has_cls
     return {k: v.cpu() for k, v in res.items()}
 
 
-def _check_block(res, ref, dtype, out_dtype, has_cls=True):
+def _check_block(res, ref, dtype, out_dtype, has_cls=True, score_rel=None):
     od = "f32" if out_dtype == torch.float32 else dtype
     rounded = od == "bf16"
     want_full = orc.round_to(ref["x_hat"], od)
     stats = parity.check_float(res["x_full"].double().numpy(), want_full, dtype, rounded)
     s = res["scores"].double().numpy()
     rel = np.abs(s - ref["scores"]) / np.maximum(np.abs(ref["scores"]), 1e-30)
-    assert rel.max() < (1e-5 if dtype == "f32" else 5e-4), f"score rel err {rel.max():.3e}"
+    if score_rel is None:
+        score_rel = 1e-5 if dtype == "f32" else 5e-4
+    assert rel.max() < score_rel, f"score rel err {rel.max():.3e}"
     swaps = parity.check_keep(ref["scores"], ref["keep_idx"], res["keep_idx"].numpy(), has_cls)
     # compaction is an exact row copy of the GPU's own un-pruned output
     keep = res["keep_idx"].long()
@@ -87,6 +89,22 @@ def test_block_delta_score_mode_and_no_cls(ctx):
     rel = np.abs(resb["scores"].double().numpy() - refb["scores"]) / refb["scores"]
     assert rel.max() < 3e-3
     parity.check_float(resb["x_full"].double().numpy(), refb["x_hat"], "bf16", False)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("mode", ["attn", "block"])
+def test_block_other_operation_choices(ctx, dtype, mode):
+    """Sec. 3.3 operation choices (i) and (iii): the shift through attention, fused into the
+    projection epilogue, and through the whole block, fused into the FC2 epilogue."""
+    B, N, D, H, r = 2, 150, 384, 6, 11
+    x = synth.make_tokens(B, N, D, dtype, seed=41)
+    w = synth.make_block_weights(D, 4 * D, dtype, seed=42)
+    ref = orc.block_fwd(x.double().numpy(), _np(w), H, r, score_mode=mode)
+    out_dtype = torch.float32 if dtype == "bf16" else None
+    res = _run_block(ctx, x, w, H, r, dtype, out_dtype, score_mode=mode)
+    # These scores are norms of the sub-layer outputs themselves (no exact x' term dominates them as in
+    # the default mode), so they carry the bf16 operand rounding of the contractions in full: 2e-3.
+    _check_block(res, ref, dtype, out_dtype, score_rel=(1e-5 if dtype == "f32" else 2e-3))
 
 
 def test_block_video_tokens_ar1(ctx):
