@@ -152,7 +152,7 @@ typedef struct {
     float ln_eps;          /* 0 => 1e-6 */
     float scale;           /* 0 => 1/sqrt(D/H) */
     rs_score_mode score_mode;
-    rs_dist dist;          /* only RS_DIST_L2 inside the block */
+    rs_dist dist;          /* distance D of the score (Sec. 3.3 "Distance metrics") */
 } rs_block_desc;
 
 typedef struct {           /* all dev pointers */

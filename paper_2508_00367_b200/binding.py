@@ -261,11 +261,11 @@ class Context:
                   out_dtype=None, score_mode: str = "mlp", ln_eps: float = 0.0, scale: float = 0.0,
                   want_full: bool = False, workspace: Optional[torch.Tensor] = None,
                   x_out: Optional[torch.Tensor] = None, scores: Optional[torch.Tensor] = None,
-                  keep_idx: Optional[torch.Tensor] = None) -> Dict[str, torch.Tensor]:
+                  keep_idx: Optional[torch.Tensor] = None, dist: str = "l2") -> Dict[str, torch.Tensor]:
         """One block + pruning.  Returns dict(x_out, scores, keep_idx[, x_full])."""
         assert x.is_cuda and x.is_contiguous()
         B, N, D = x.shape
-        desc = self.block_desc(B, N, D, H, weights.D_mlp, r, x.dtype, out_dtype, has_cls, ln_eps, scale, score_mode)
+        desc = self.block_desc(B, N, D, H, weights.D_mlp, r, x.dtype, out_dtype, has_cls, ln_eps, scale, score_mode, dist)
         odt = _torch_dt(desc.out_dtype)
         K = N - r
         need = self.block_workspace_bytes(desc)

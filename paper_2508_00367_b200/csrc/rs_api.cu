@@ -208,7 +208,7 @@ rs_status rs_linear_fwd(rs_ctx* ctx, rs_dtype dtype, rs_linear_epilogue epi, lon
     const rs_dtype out_dtype = epi == RS_LIN_BIAS_RESIDUAL ? RS_F32 : dtype;
     if (ctx->use_tc && dtype == RS_BF16 && rs::gemm_tc_supported(M, N, K)) {
         const int e = epi == RS_LIN_BIAS ? rs::RS_EPI_BIAS : epi == RS_LIN_BIAS_GELU ? rs::RS_EPI_BIAS_GELU : rs::RS_EPI_RESID;
-        RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_tc(ctx, e, A, W, bias, residual, nullptr, out, out_dtype, nullptr, 0, M, N, K, st), "tensor-core GEMM");
+        RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_tc(ctx, e, A, W, bias, residual, nullptr, out, out_dtype, nullptr, 0, 0, M, N, K, st), "tensor-core GEMM");
     } else {
         RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_simt(dtype, A, W, bias, epi == RS_LIN_BIAS_GELU, epi == RS_LIN_BIAS_RESIDUAL ? residual : nullptr, dtype, out, out_dtype, M, N, K, st), "GEMM");
     }
@@ -275,7 +275,7 @@ rs_status rs_block_fwd(rs_ctx* ctx, const rs_block_desc* d, const rs_block_weigh
     if (d->D > 1024 && d->dtype == RS_F32) return fail(ctx, RS_ERR_UNSUPPORTED, "rs_block_fwd: D > 1024 in fp32");
     if (d->N > 32768) return fail(ctx, RS_ERR_UNSUPPORTED, "rs_block_fwd: N > 32768");
     if (d->r < 0 || d->r > d->N - 1) return fail(ctx, RS_ERR_INVALID_ARG, "rs_block_fwd: need 0 <= r <= N-1");
-    if (d->dist != RS_DIST_L2) return fail(ctx, RS_ERR_UNSUPPORTED, "rs_block_fwd: only the L2 distance is fused into the block");
+    if (d->dist < RS_DIST_L2 || d->dist > RS_DIST_COS) return fail(ctx, RS_ERR_INVALID_ARG, "rs_block_fwd: bad dist");
     if (d->score_mode < RS_SCORE_MLP || d->score_mode > RS_SCORE_BLOCK)
         return fail(ctx, RS_ERR_INVALID_ARG, "rs_block_fwd: bad score_mode");
     if (d->dtype == RS_F32 && d->out_dtype != RS_F32)
@@ -324,12 +324,12 @@ rs_status rs_block_fwd(rs_ctx* ctx, const rs_block_desc* d, const rs_block_weigh
     // x' = SA(LN(x)) + x                                                  (Eq. att)
     RS_CHECK_LAUNCH(ctx, RS_K_LAYERNORM, st, rs::launch_layernorm(d->dtype, d->dtype, x, w->ln1_g, w->ln1_b, eps, T, D, u, st), "LN1");
     if (tc) {
-        RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_tc(ctx, rs::RS_EPI_BIAS, u, w->w_qkv, w->b_qkv, nullptr, nullptr, qkv, RS_BF16, nullptr, 0, T, 3 * D, D, st), "QKV");
+        RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_tc(ctx, rs::RS_EPI_BIAS, u, w->w_qkv, w->b_qkv, nullptr, nullptr, qkv, RS_BF16, nullptr, 0, 0, T, 3 * D, D, st), "QKV");
         RS_CHECK_LAUNCH(ctx, RS_K_ATTN, st, rs::launch_attn_tc(ctx, ad, qkv, kp, vp, o, st), "attention");
         // shift through attention (operation choice (i)): partial sums of (SA(LN(x)) - x)^2 from this epilogue
         nparts = rs::gemm_tc_score_parts(ctx, T, D);
         float* attn_parts = d->score_mode == RS_SCORE_ATTN ? m : nullptr;
-        RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_tc(ctx, rs::RS_EPI_RESID, o, w->w_o, w->b_o, x, nullptr, x_prime, RS_F32, attn_parts, 0, T, D, D, st), "proj");
+        RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_tc(ctx, rs::RS_EPI_RESID, o, w->w_o, w->b_o, x, nullptr, x_prime, RS_F32, attn_parts, 0, (int)d->dist, T, D, D, st), "proj");
     } else {
         RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_simt(d->dtype, u, w->w_qkv, w->b_qkv, 0, nullptr, RS_F32, qkv, d->dtype, T, 3 * D, D, st), "QKV");
         RS_CHECK_LAUNCH(ctx, RS_K_ATTN, st, rs::launch_attn_simt(ad, qkv, kp, vp, o, st), "attention");
@@ -341,18 +341,18 @@ rs_status rs_block_fwd(rs_ctx* ctx, const rs_block_desc* d, const rs_block_weigh
         // The FC2 epilogue adds the residual and leaves per-tile partial sums of squares of the
         // shift in `m`; the selection kernel adds them up in a fixed order.
         // (when the score came from the projection, this epilogue's partial sums go to a second array)
-        float* fc2_parts = d->score_mode == RS_SCORE_ATTN ? m + (size_t)T * nparts : m;
+        float* fc2_parts = d->score_mode == RS_SCORE_ATTN ? m + (size_t)T * nparts * 3 : m;
         const int kind = d->score_mode == RS_SCORE_MLP_DELTA ? 1 : d->score_mode == RS_SCORE_BLOCK ? 2 : 0;
-        RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_tc(ctx, rs::RS_EPI_BIAS_GELU, u, w->w_fc1, w->b_fc1, nullptr, nullptr, h, RS_BF16, nullptr, 0, T, Dm, D, st), "FC1");
-        RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_tc(ctx, rs::RS_EPI_SCORE, h, w->w_fc2, w->b_fc2, x_prime, x, x_hat, d->out_dtype, fc2_parts, kind, T, D, Dm, st), "FC2+residual+score");
+        RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_tc(ctx, rs::RS_EPI_BIAS_GELU, u, w->w_fc1, w->b_fc1, nullptr, nullptr, h, RS_BF16, nullptr, 0, 0, T, Dm, D, st), "FC1");
+        RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_tc(ctx, rs::RS_EPI_SCORE, h, w->w_fc2, w->b_fc2, x_prime, x, x_hat, d->out_dtype, fc2_parts, kind, (int)d->dist, T, D, Dm, st), "FC2+residual+score");
     } else {
         RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_simt(d->dtype, u, w->w_fc1, w->b_fc1, 1, nullptr, RS_F32, h, d->dtype, T, Dm, D, st), "FC1");
         RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_simt(d->dtype, h, w->w_fc2, w->b_fc2, 0, nullptr, RS_F32, m, RS_F32, T, D, Dm, st), "FC2");
-        RS_CHECK_LAUNCH(ctx, RS_K_SCORE, st, rs::launch_residual_score(m, x_prime, x, d->dtype, T, D, d->score_mode, d->out_dtype, x_hat, s, st), "residual+score");
+        RS_CHECK_LAUNCH(ctx, RS_K_SCORE, st, rs::launch_residual_score(m, x_prime, x, d->dtype, T, D, d->score_mode, d->dist, d->out_dtype, x_hat, s, st), "residual+score");
     }
     // reduced token set                                                   (Sec. 3.1)
     if (nparts > 0)
-        RS_CHECK_LAUNCH(ctx, RS_K_SELECT, st, rs::launch_select(m, nparts, s, d->B, d->N, K, d->has_cls ? 1 : 0, keep, st), "select");
+        RS_CHECK_LAUNCH(ctx, RS_K_SELECT, st, rs::launch_select(m, nparts | ((int)d->dist << 16), s, d->B, d->N, K, d->has_cls ? 1 : 0, keep, st), "select");
     else
         RS_CHECK_LAUNCH(ctx, RS_K_SELECT, st, rs::launch_select(s, 0, nullptr, d->B, d->N, K, d->has_cls ? 1 : 0, keep, st), "select");
     if (x_hat != x_out)

@@ -178,12 +178,12 @@ shift_score_kernel(const T* __restrict__ after, const T* __restrict__ before, lo
 template <typename TO, typename TX, int MODE>
 __global__ void __launch_bounds__(kWarpsPerCta * 32)
 residual_score_kernel(const float* __restrict__ m, const float* __restrict__ xp, const TX* __restrict__ x0,
-                      long long rows, int D, TO* __restrict__ x_hat, float* __restrict__ scores) {
+                      long long rows, int D, int dist, TO* __restrict__ x_hat, float* __restrict__ scores) {
     const int lane = threadIdx.x & 31;
     const long long row = (long long)blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5);
     if (row >= rows) return;
     const int nvec = D / 4;
-    float acc = 0.f;
+    float acc = 0.f, uu = 0.f, vv = 0.f;
     for (int iv = lane; iv < nvec; iv += 32) {
         const float4 a = *reinterpret_cast<const float4*>(m + row * D + iv * 4);
         const float4 b = *reinterpret_cast<const float4*>(xp + row * D + iv * 4);
@@ -192,19 +192,27 @@ residual_score_kernel(const float* __restrict__ m, const float* __restrict__ xp,
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
             y[e] = av[e] + bv[e];
-            float d;
-            if (MODE == 0) d = av[e] - bv[e];
-            else if (MODE == 1) d = av[e];
+            float u, v;                              // the scored pair
+            if (MODE == 0) { u = av[e]; v = bv[e]; }
+            else if (MODE == 1) { u = y[e]; v = bv[e]; }
             else {
                 const float x = to_float(x0[row * D + iv * 4 + e]);
-                d = MODE == 2 ? bv[e] - 2.f * x : y[e] - x;
+                u = MODE == 2 ? bv[e] - x : y[e];    // SA(LN(x)) = x' - x
+                v = x;
             }
-            acc = fmaf(d, d, acc);
+            if (dist == RS_DIST_L2) { const float d = u - v; acc = fmaf(d, d, acc); }
+            else if (dist == RS_DIST_L1) acc += fabsf(u - v);
+            else { acc = fmaf(u, v, acc); uu = fmaf(u, u, uu); vv = fmaf(v, v, vv); }
         }
         store_n<TO, 4>(x_hat + row * D + iv * 4, y);
     }
     acc = warp_sum(acc);
-    if (lane == 0 && scores) scores[row] = sqrtf(acc);
+    float sc = dist == RS_DIST_L2 ? sqrtf(acc) : acc;
+    if (dist == RS_DIST_COS) {
+        uu = warp_sum(uu); vv = warp_sum(vv);
+        sc = 1.f - acc / fmaxf(sqrtf(uu) * sqrtf(vv), 1e-12f);
+    }
+    if (lane == 0 && scores) scores[row] = sc;
 }
 
 inline unsigned row_grid(long long rows) { return (unsigned)((rows + kWarpsPerCta - 1) / kWarpsPerCta); }
@@ -253,12 +261,12 @@ cudaError_t launch_shift_score(rs_dtype dtype, rs_dist dist, long long T, int D,
 }
 
 cudaError_t launch_residual_score(const float* m, const float* x_prime, const void* x, rs_dtype x_dtype,
-                                  long long T, int D, rs_score_mode mode, rs_dtype out_dtype, void* x_hat,
-                                  float* scores, cudaStream_t st) {
+                                  long long T, int D, rs_score_mode mode, rs_dist dist, rs_dtype out_dtype,
+                                  void* x_hat, float* scores, cudaStream_t st) {
     if (T == 0) return cudaSuccess;
     const dim3 grid(row_grid(T)), block(kWarpsPerCta * 32);
 #define RS_RES_CASE(TO, TX, MD)                                                                                  \
-    residual_score_kernel<TO, TX, MD><<<grid, block, 0, st>>>(m, x_prime, (const TX*)x, T, D, (TO*)x_hat, scores)
+    residual_score_kernel<TO, TX, MD><<<grid, block, 0, st>>>(m, x_prime, (const TX*)x, T, D, (int)dist, (TO*)x_hat, scores)
 #define RS_RES_MODE(TO, TX)                                     \
     do {                                                        \
         if (mode == RS_SCORE_MLP) RS_RES_CASE(TO, TX, 0);       \

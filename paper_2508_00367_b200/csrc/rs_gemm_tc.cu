@@ -54,7 +54,8 @@ struct GemmArgs {
     const void* residual;     // EPI_RESID: bf16 [M, N];  EPI_SCORE: fp32 [M, N]
     const void* residual2;    // EPI_SCORE, score_kind 2: bf16 [M, N] block input x
     float* partials;          // EPI_SCORE (and EPI_RESID when non-null): [M, 2 * N / BN] sums of squares
-    int score_kind;           // EPI_SCORE: 0 => (m - x')^2, 1 => m^2, 2 => (m + x' - x)^2
+    int score_kind;           // EPI_SCORE: scored pair (u, v) = 0: (m, x'), 1: (x^, x'), 2: (x^, x)
+    int dist;                 // rs_dist of the score: L2 / L1 sums of (u - v)^2 / |u - v|, cosine sums of u.v, u.u, v.v
     int* status;
 };
 
@@ -74,6 +75,13 @@ __device__ __forceinline__ float gelu_erf(float v) {
     float e;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(-q));
     return v * (v >= 0.f ? 1.f - e : e);
+}
+
+// Adds one element of the scored pair (u, v) to the running sums of the chosen distance (Sec. 3.3).
+__device__ __forceinline__ void score_acc(int dist, float u, float v, float& s0, float& s1, float& s2) {
+    if (dist == RS_DIST_L2) { const float d = u - v; s0 = fmaf(d, d, s0); }
+    else if (dist == RS_DIST_L1) { s0 += fabsf(u - v); }
+    else { s0 = fmaf(u, v, s0); s1 = fmaf(u, u, s1); s2 = fmaf(v, v, s2); }
 }
 
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
@@ -222,7 +230,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             if (half_fail[half]) break;
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + a * BN;
-            float sq = 0.f;
+            float sq = 0.f, sq1 = 0.f, sq2 = 0.f;
 #pragma unroll 1
             for (int c = c_begin; c < c_end; c += 32) {
                 const int cb = (c / 32) % CHUNKS_PER_BLK;            // chunk inside the staged block
@@ -261,9 +269,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
                             const float x0 = __uint_as_float(w[e] << 16), x1 = __uint_as_float(w[e] & 0xffff0000u);
-                            const float d0 = v[8 * j + 2 * e] - x0, d1 = v[8 * j + 2 * e + 1] - x1;   // SA(LN(x)) - x
-                            sq = fmaf(d0, d0, sq);
-                            sq = fmaf(d1, d1, sq);
+                            if (args.partials) {                      // (u, v) = (SA(LN(x)), x)
+                                score_acc(args.dist, v[8 * j + 2 * e], x0, sq, sq1, sq2);
+                                score_acc(args.dist, v[8 * j + 2 * e + 1], x1, sq, sq1, sq2);
+                            }
                             v[8 * j + 2 * e] += x0;
                             v[8 * j + 2 * e + 1] += x1;
                         }
@@ -285,8 +294,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                             for (int e = 0; e < 4; ++e) {
                                 const float xa = __uint_as_float(w[e] << 16), xb = __uint_as_float(w[e] & 0xffff0000u);
                                 const float ya = v[8 * j + 2 * e] + xp[2 * e], yb = v[8 * j + 2 * e + 1] + xp[2 * e + 1];
-                                sq = fmaf(ya - xa, ya - xa, sq);
-                                sq = fmaf(yb - xb, yb - xb, sq);
+                                score_acc(args.dist, ya, xa, sq, sq1, sq2);
+                                score_acc(args.dist, yb, xb, sq, sq1, sq2);
                                 v[8 * j + 2 * e] = ya;
                                 v[8 * j + 2 * e + 1] = yb;
                             }
@@ -298,10 +307,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                                                  __uint_as_float(res[j].z), __uint_as_float(res[j].w)};
 #pragma unroll
                             for (int e = 0; e < 4; ++e) {
-                                const float m = v[4 * j + e];
-                                const float d = args.score_kind ? m : m - xs[e];
-                                sq = fmaf(d, d, sq);
-                                v[4 * j + e] = m + xs[e];
+                                const float m = v[4 * j + e], y = m + xs[e];
+                                score_acc(args.dist, args.score_kind ? y : m, xs[e], sq, sq1, sq2);
+                                v[4 * j + e] = y;
                             }
                         }
                     }
@@ -335,8 +343,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     ++blk_ctr;
                 }
             }
-            if ((EPI == EPI_SCORE || (EPI == EPI_RESID && args.partials)) && valid)
-                args.partials[(size_t)row * (2 * num_n) + 2 * nt + half] = sq;
+            if ((EPI == EPI_SCORE || (EPI == EPI_RESID && args.partials)) && valid) {
+                const size_t pi = (size_t)row * (2 * num_n) + 2 * nt + half;
+                if (args.dist == RS_DIST_COS) {
+                    args.partials[3 * pi] = sq; args.partials[3 * pi + 1] = sq1; args.partials[3 * pi + 2] = sq2;
+                } else {
+                    args.partials[pi] = sq;
+                }
+            }
         }
         if (storer) tma_store_wait<0>();                 // all output written before the CTA exits
     }
@@ -439,7 +453,7 @@ int gemm_tc_score_parts(const rs_ctx* ctx, long long M, int N) {
 }
 
 cudaError_t launch_gemm_tc(rs_ctx* ctx, int epi, const void* A, const void* W, const float* bias,
-                           const void* residual, const void* residual2, void* out, rs_dtype out_dtype, float* partials, int score_kind,
+                           const void* residual, const void* residual2, void* out, rs_dtype out_dtype, float* partials, int score_kind, int dist,
                            long long M, int N, int K, cudaStream_t st) {
     if (!ctx->encode_tiled) return cudaErrorNotSupported;
     const int bn = pick_bn(M, N, ctx->sm_count);
@@ -451,7 +465,7 @@ cudaError_t launch_gemm_tc(rs_ctx* ctx, int epi, const void* A, const void* W, c
         return cudaErrorInvalidValue;
     GemmArgs args;
     args.M = (int)M; args.N = N; args.K = K; args.bias = bias; args.residual = residual;
-    args.residual2 = residual2; args.partials = partials; args.score_kind = score_kind; args.status = ctx->d_status;
+    args.residual2 = residual2; args.partials = partials; args.score_kind = score_kind; args.dist = dist; args.status = ctx->d_status;
     const int sms = ctx->sm_count;
 #define RS_GEMM_CASE(E, T)                                                                       \
     return bn == 256   ? launch_one<256, E, T>(tmA, tmB, tmOut, args, sms, st)                  \

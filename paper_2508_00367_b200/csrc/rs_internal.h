@@ -63,12 +63,13 @@ cudaError_t launch_shift_score(rs_dtype dtype, rs_dist dist, long long T, int D,
 // s = |m - x_prime| (MLP), |m| (MLP_DELTA), |x_prime - 2 x| = |SA(LN(x)) - x| (ATTN) or
 // |x_hat - x| (BLOCK).  m, x_prime fp32; x (the block input, x_dtype) only for ATTN and BLOCK.
 cudaError_t launch_residual_score(const float* m, const float* x_prime, const void* x, rs_dtype x_dtype,
-                                  long long T, int D, rs_score_mode mode, rs_dtype out_dtype, void* x_hat,
-                                  float* scores, cudaStream_t st);
+                                  long long T, int D, rs_score_mode mode, rs_dist dist, rs_dtype out_dtype,
+                                  void* x_hat, float* scores, cudaStream_t st);
 
 // ---- selection and compaction (rs_select.cu) ----
-// scores: [B, N] fp32, or if nparts > 0 partial sums of squares [B*N, nparts] whose row
-// sum's square root is the score (then also written to scores_out when non-null).
+// scores: [B, N] fp32; or, if nparts > 0, the per-tile partial sums a GEMM epilogue left
+// (nparts = tiles | rs_dist << 16; [B*N, tiles] sums, three per tile for the cosine distance),
+// from which the score is finished here (and written to scores_out when non-null).
 cudaError_t launch_select(const float* scores, int nparts, float* scores_out, int B, int N, int K,
                           int has_cls, int32_t* keep_idx, cudaStream_t st);
 cudaError_t launch_gather(rs_dtype dtype, const void* x, const int32_t* keep_idx, int B, int N, int K,
@@ -92,7 +93,7 @@ int gemm_tc_score_parts(const rs_ctx* ctx, long long M, int N);   // partial sum
 // out[M, N] = epilogue(A[M, K] . W[N, K]^T); see rs_gemm_tc.cu for the epilogues.
 cudaError_t launch_gemm_tc(rs_ctx* ctx, int epi, const void* A, const void* W, const float* bias,
                            const void* residual, const void* residual2, void* out, rs_dtype out_dtype,
-                           float* partials, int score_kind, long long M, int N, int K, cudaStream_t st);
+                           float* partials, int score_kind, int dist, long long M, int N, int K, cudaStream_t st);
 
 // ---- tcgen05 attention (rs_attn_tc.cu): bf16, head dimension 64 ----
 bool attn_tc_supported(const rs_attn_desc& d);

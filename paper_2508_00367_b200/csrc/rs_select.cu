@@ -17,6 +17,22 @@ namespace {
 
 constexpr int kSelThreads = 512;
 
+// Score of one token from the per-tile partial sums the GEMM epilogues leave (fixed summation
+// order: run-to-run identical).  `enc` = number of tiles | distance << 16.  L2: sqrt of the sum of
+// squares; L1: the sum; cosine: three sums per tile (u.v, u.u, v.v) -> 1 - u.v / (|u||v|).
+__device__ __forceinline__ float finish_score(const float* __restrict__ p, int enc) {
+    const int nparts = enc & 0xffff, dist = enc >> 16;
+    if (dist == RS_DIST_COS) {
+        float uv = 0.f, uu = 0.f, vv = 0.f;
+        for (int j = 0; j < nparts; ++j) { uv += p[3 * j]; uu += p[3 * j + 1]; vv += p[3 * j + 2]; }
+        return 1.f - uv / fmaxf(sqrtf(uu) * sqrtf(vv), 1e-12f);
+    }
+    float acc = 0.f;
+    for (int j = 0; j < nparts; ++j) acc += p[j];
+    return dist == RS_DIST_L1 ? acc : sqrtf(acc);
+}
+__device__ __forceinline__ int partial_stride(int enc) { return (enc & 0xffff) * ((enc >> 16) == RS_DIST_COS ? 3 : 1); }
+
 __device__ __forceinline__ uint32_t score_key(float s) {
     if (s != s) return 0u;                 // NaN ranks below every number
     if (s == 0.f) s = 0.f;                 // -0 and +0 tie
@@ -71,11 +87,8 @@ select_kernel(const float* __restrict__ scores, int nparts, float* __restrict__ 
 
     for (int i = tid; i < N; i += kSelThreads) {
         float s;
-        if (nparts > 0) {                  // fixed-order sum of the per-tile partial sums of squares
-            const float* p = scores + ((long long)b * N + i) * nparts;
-            float acc = 0.f;
-            for (int j = 0; j < nparts; ++j) acc += p[j];
-            s = sqrtf(acc);
+        if (nparts > 0) {                  // per-tile partial sums from the GEMM epilogue
+            s = finish_score(scores + ((long long)b * N + i) * partial_stride(nparts), nparts);
             if (scores_out) scores_out[(long long)b * N + i] = s;
         } else {
             s = scores[(long long)b * N + i];
@@ -173,11 +186,8 @@ select_small_kernel(const float* __restrict__ scores, int nparts, float* __restr
     uint32_t key = 0;
     if (i < N) {
         float s;
-        if (nparts > 0) {                  // fixed-order sum of the per-tile partial sums of squares
-            const float* p = scores + ((long long)b * N + i) * nparts;
-            float acc = 0.f;
-            for (int j = 0; j < nparts; ++j) acc += p[j];
-            s = sqrtf(acc);
+        if (nparts > 0) {                  // per-tile partial sums from the GEMM epilogue
+            s = finish_score(scores + ((long long)b * N + i) * partial_stride(nparts), nparts);
             if (scores_out) scores_out[(long long)b * N + i] = s;
         } else {
             s = scores[(long long)b * N + i];
@@ -220,12 +230,7 @@ keep_all_kernel(const float* __restrict__ scores, int nparts, float* __restrict_
     grid_dep_wait();
     const long long t = (long long)blockIdx.x * 256 + threadIdx.x;
     if (t >= T) return;
-    if (nparts > 0 && scores_out) {
-        const float* p = scores + t * nparts;
-        float acc = 0.f;
-        for (int j = 0; j < nparts; ++j) acc += p[j];
-        scores_out[t] = sqrtf(acc);
-    }
+    if (nparts > 0 && scores_out) scores_out[t] = finish_score(scores + t * partial_stride(nparts), nparts);
     keep_idx[t] = (int32_t)(t % N);
 }
 

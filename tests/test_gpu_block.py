@@ -25,11 +25,11 @@ def _np(w):
     return {k: v.double().numpy() for k, v in w.items()}
 
 
-def _run_block(ctx, x, w, H, r, dtype, out_dtype=None, score_mode="mlp", has_cls=True):
+def _run_block(ctx, x, w, H, r, dtype, out_dtype=None, score_mode="mlp", has_cls=True, dist="l2"):
     import paper_2508_00367_b200 as rs
     dw = rs.DeviceBlockWeights(w, DT[dtype], ctx.device)
     res = ctx.block_fwd(x.to(DT[dtype]).cuda(), dw, H, r, has_cls=has_cls, out_dtype=out_dtype,
-                        score_mode=score_mode, want_full=True)
+                        score_mode=score_mode, want_full=True, dist=dist)
     torch.cuda.synchronize()
     return {k: v.cpu() for k, v in res.items()}
 
@@ -105,6 +105,29 @@ def test_block_other_operation_choices(ctx, dtype, mode):
     # These scores are norms of the sub-layer outputs themselves (no exact x' term dominates them as in
     # the default mode), so they carry the bf16 operand rounding of the contractions in full: 2e-3.
     _check_block(res, ref, dtype, out_dtype, score_rel=(1e-5 if dtype == "f32" else 2e-3))
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("mode,dist", [("mlp", "l1"), ("mlp", "cos"), ("mlp_delta", "cos"), ("attn", "l1"),
+                                       ("attn", "cos"), ("block", "cos"), ("block", "l1")])
+def test_block_other_distances(ctx, dtype, mode, dist):
+    """Sec. 3.3 distance metrics (L1, cosine) fused into the same epilogues as the default L2."""
+    B, N, D, H, r = 2, 140, 256, 4, 9
+    x = synth.make_tokens(B, N, D, dtype, seed=51)
+    w = synth.make_block_weights(D, 4 * D, dtype, seed=52)
+    ref = orc.block_fwd(x.double().numpy(), _np(w), H, r, score_mode=mode, dist=dist)
+    out_dtype = torch.float32 if dtype == "bf16" else None
+    res = _run_block(ctx, x, w, H, r, dtype, out_dtype, score_mode=mode, dist=dist)
+    full = res["x_full"].double().numpy()
+    parity.check_float(full, orc.round_to(ref["x_hat"], "f32"), dtype, False)
+    s = res["scores"].double().numpy()
+    if dist == "cos":          # a distance in [0, 2]: absolute tolerance
+        tol = 1e-5 if dtype == "f32" else 2e-3
+        assert np.abs(s - ref["scores"]).max() < tol, np.abs(s - ref["scores"]).max()
+    else:
+        rel = np.abs(s - ref["scores"]) / np.maximum(np.abs(ref["scores"]), 1e-30)
+        assert rel.max() < (1e-5 if dtype == "f32" else 2e-3), rel.max()
+    assert res["keep_idx"].shape == (B, N - r) and (res["keep_idx"][:, 0] == 0).all()
 
 
 def test_block_video_tokens_ar1(ctx):
