@@ -174,6 +174,32 @@ RS_API rs_status rs_block_fwd(rs_ctx* ctx, const rs_block_desc* desc /*host*/,
                        const void* x, void* x_out, float* scores, int32_t* keep_idx, void* x_full,
                        void* workspace, size_t workspace_bytes, void* stream);
 
+/* ---- rs_vit_fwd: the layer loop (Sec. 3.2: tokens are dropped after the listed blocks and ----
+ * every later block runs on the reduced set).  Runs L blocks back to back on `stream`;
+ * block l (0-based) drops drops[l] tokens after its MLP (0 = none), so block l+1 sees
+ * N_{l+1} = N_l - drops[l] tokens.  Everything else is as in rs_block_fwd, with one
+ * descriptor for the whole stack.
+ * weights (host): array of L structs of dev pointers.  drops (host): L ints, each in
+ * [0, N_l - 1].  x (dev): [B, N, D].  x_out (dev): [B, N_L, D] with N_L = N - sum(drops).
+ * scores_last / keep_last (dev, optional): the last block's scores [B, N_{L-1}] and kept
+ * indices [B, N_L].  workspace (dev): at least rs_vit_workspace_bytes() bytes, 256-byte
+ * aligned; it holds one block's scratch and two token buffers the blocks alternate between. */
+typedef struct {
+    rs_dtype dtype;
+    int B, N, D, H, D_mlp, L;
+    int has_cls;
+    float ln_eps;          /* 0 => 1e-6 */
+    float scale;           /* 0 => 1/sqrt(D/H) */
+    rs_score_mode score_mode;
+    rs_dist dist;
+} rs_vit_desc;
+
+RS_API size_t rs_vit_workspace_bytes(const rs_vit_desc* desc /*host*/, const int* drops /*host[L]*/);
+RS_API rs_status rs_vit_fwd(rs_ctx* ctx, const rs_vit_desc* desc /*host*/,
+                            const rs_block_weights* weights /*host[L]*/, const int* drops /*host[L]*/,
+                            const void* x, void* x_out, float* scores_last, int32_t* keep_last,
+                            void* workspace, size_t workspace_bytes, void* stream);
+
 /* ---- rs_block_fwd_static: rs_block_fwd for callers that cannot allocate ----------------
  * (The paper has no counterpart; this is a packaging variant of rs_block_fwd.)
  * Some callers have no way to obtain device memory when they reach the block:

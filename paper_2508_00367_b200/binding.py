@@ -26,7 +26,7 @@ STATUS_NAMES = {0: "RS_OK", 1: "RS_ERR_INVALID_ARG", 2: "RS_ERR_UNSUPPORTED", 3:
 EXPORTS = ("rs_create", "rs_destroy", "rs_last_error", "rs_async_status", "rs_uses_tensor_cores",
            "rs_launch_count", "rs_attn_fwd", "rs_shift_score", "rs_topk_compact",
            "rs_block_workspace_bytes", "rs_block_fwd", "rs_timing_enable", "rs_timing_read",
-           "rs_static_scratch_bytes", "rs_block_fwd_static", "rs_linear_fwd")
+           "rs_static_scratch_bytes", "rs_block_fwd_static", "rs_linear_fwd", "rs_vit_workspace_bytes", "rs_vit_fwd")
 LIN_EPILOGUE = {"bias": 0, "gelu": 1, "residual": 2}
 KERNEL_CLASSES = ("layernorm", "gemm", "attn", "score", "select", "gather")
 
@@ -53,6 +53,13 @@ class BlockDesc(ctypes.Structure):
                 ("N", ctypes.c_int), ("D", ctypes.c_int), ("H", ctypes.c_int), ("D_mlp", ctypes.c_int),
                 ("r", ctypes.c_int), ("has_cls", ctypes.c_int), ("ln_eps", ctypes.c_float),
                 ("scale", ctypes.c_float), ("score_mode", ctypes.c_int), ("dist", ctypes.c_int)]
+
+
+class VitDesc(ctypes.Structure):
+    _fields_ = [("dtype", ctypes.c_int), ("B", ctypes.c_int), ("N", ctypes.c_int), ("D", ctypes.c_int),
+                ("H", ctypes.c_int), ("D_mlp", ctypes.c_int), ("L", ctypes.c_int), ("has_cls", ctypes.c_int),
+                ("ln_eps", ctypes.c_float), ("scale", ctypes.c_float), ("score_mode", ctypes.c_int),
+                ("dist", ctypes.c_int)]
 
 
 class BlockWeights(ctypes.Structure):
@@ -108,6 +115,11 @@ def load_library() -> ctypes.CDLL:
     lib.rs_block_fwd_static.argtypes = [ctypes.POINTER(BlockDesc), ctypes.POINTER(BlockWeights), vp, vp, vp, vp, vp,
                                         vp, ctypes.c_char_p, ctypes.c_size_t]
     lib.rs_block_fwd_static.restype = ci
+    lib.rs_vit_workspace_bytes.argtypes = [ctypes.POINTER(VitDesc), ctypes.POINTER(ci)]
+    lib.rs_vit_workspace_bytes.restype = ctypes.c_size_t
+    lib.rs_vit_fwd.argtypes = [vp, ctypes.POINTER(VitDesc), ctypes.POINTER(BlockWeights), ctypes.POINTER(ci), vp, vp, vp,
+                               vp, vp, ctypes.c_size_t, vp]
+    lib.rs_vit_fwd.restype = ci
     _lib = lib
     return lib
 
@@ -245,6 +257,31 @@ class Context:
         self._check(self.lib.rs_topk_compact(self.handle, dt, B, N, D, r, int(has_cls), _ptr(scores), _ptr(x),
                                              _ptr(x_out), _ptr(keep_idx), _stream(scores.device)))
         return x_out, keep_idx
+
+    # ---- rs_vit_fwd ----
+    def vit_fwd(self, x: torch.Tensor, weights: Sequence["DeviceBlockWeights"], H: int, drops: Sequence[int],
+                has_cls: bool = True, score_mode: str = "mlp", dist: str = "l2",
+                workspace: Optional[torch.Tensor] = None) -> Dict[str, torch.Tensor]:
+        """The whole layer loop in one library call.  Returns dict(x_out, scores, keep_idx) of the last block."""
+        assert x.is_cuda and x.is_contiguous() and len(weights) == len(drops)
+        B, N, D = x.shape
+        L = len(weights)
+        desc = VitDesc(_dt(x), B, N, D, H, weights[0].D_mlp, L, int(has_cls), 0.0, 0.0, SCORE_MODE[score_mode], DIST[dist])
+        cdrops = (ctypes.c_int * L)(*[int(r) for r in drops])
+        warr = (BlockWeights * L)(*[w.struct for w in weights])
+        need = int(self.lib.rs_vit_workspace_bytes(ctypes.byref(desc), cdrops))
+        if need == 0:
+            raise RsError(1, "rs_vit_fwd: bad descriptor or schedule")
+        if workspace is None:
+            workspace = torch.empty(need, dtype=torch.uint8, device=x.device)
+        n_last = N - sum(int(r) for r in drops[:-1])
+        n_out = n_last - int(drops[-1])
+        x_out = torch.empty(B, n_out, D, dtype=x.dtype, device=x.device)
+        scores = torch.empty(B, n_last, dtype=torch.float32, device=x.device)
+        keep = torch.empty(B, n_out, dtype=torch.int32, device=x.device)
+        self._check(self.lib.rs_vit_fwd(self.handle, ctypes.byref(desc), warr, cdrops, _ptr(x), _ptr(x_out), _ptr(scores),
+                                        _ptr(keep), _ptr(workspace), workspace.numel(), _stream(x.device)))
+        return dict(x_out=x_out, scores=scores, keep_idx=keep)
 
     # ---- rs_block_fwd ----
     def block_desc(self, B, N, D, H, D_mlp, r, dtype, out_dtype=None, has_cls=True, ln_eps=0.0, scale=0.0,

@@ -361,3 +361,70 @@ rs_status rs_block_fwd(rs_ctx* ctx, const rs_block_desc* d, const rs_block_weigh
 }
 
 }  // extern "C"
+
+namespace {
+
+// Plan of the layer loop: per-block descriptors, the largest block scratch and the size of one
+// of the two token buffers the blocks alternate between.  False on a bad descriptor / schedule.
+struct VitPlan { size_t block_ws, act_bytes, total; int n_final; };
+
+bool vit_plan(const rs_vit_desc& d, const int* drops, VitPlan* p) {
+    if (!drops || d.L < 1 || d.B < 1 || d.N < 1) return false;
+    size_t block_ws = 0;
+    int n = d.N;
+    for (int l = 0; l < d.L; ++l) {
+        if (drops[l] < 0 || drops[l] > n - 1) return false;
+        rs_block_desc bd = {d.dtype, d.dtype, d.B, n, d.D, d.H, d.D_mlp, drops[l], d.has_cls, d.ln_eps, d.scale, d.score_mode, d.dist};
+        const size_t w = rs_block_workspace_bytes(&bd);
+        if (w == 0) return false;
+        if (w > block_ws) block_ws = w;
+        n -= drops[l];
+    }
+    p->block_ws = rs::align_up(block_ws, 256);
+    p->act_bytes = rs::align_up((size_t)d.B * d.N * d.D * rs::dtype_size(d.dtype), 256);
+    p->total = p->block_ws + 2 * p->act_bytes;
+    p->n_final = n;
+    return true;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t rs_vit_workspace_bytes(const rs_vit_desc* d, const int* drops) {
+    VitPlan p;
+    if (!d || !valid_dtype(d->dtype) || !vit_plan(*d, drops, &p)) return 0;
+    return p.total;
+}
+
+rs_status rs_vit_fwd(rs_ctx* ctx, const rs_vit_desc* d, const rs_block_weights* weights, const int* drops,
+                     const void* x, void* x_out, float* scores_last, int32_t* keep_last, void* workspace,
+                     size_t workspace_bytes, void* stream) {
+    if (!ctx) return RS_ERR_INVALID_ARG;
+    if (!d || !weights || !drops || !x || !x_out) return fail(ctx, RS_ERR_INVALID_ARG, "rs_vit_fwd: null argument");
+    VitPlan p;
+    if (!valid_dtype(d->dtype) || !vit_plan(*d, drops, &p))
+        return fail(ctx, RS_ERR_INVALID_ARG, "rs_vit_fwd: bad descriptor or schedule (need 0 <= drops[l] <= N_l - 1)");
+    if (!workspace || workspace_bytes < p.total)
+        return fail(ctx, RS_ERR_WORKSPACE, "rs_vit_fwd: workspace of %zu bytes needed, %zu given", p.total, workspace_bytes);
+    if (reinterpret_cast<uintptr_t>(workspace) & 255u)
+        return fail(ctx, RS_ERR_INVALID_ARG, "rs_vit_fwd: workspace must be 256-byte aligned");
+    char* base = (char*)workspace;
+    void* act[2] = {base + p.block_ws, base + p.block_ws + p.act_bytes};
+    const void* cur = x;
+    int n = d->N;
+    for (int l = 0; l < d->L; ++l) {
+        const bool last = l == d->L - 1;
+        rs_block_desc bd = {d->dtype, d->dtype, d->B, n, d->D, d->H, d->D_mlp, drops[l], d->has_cls, d->ln_eps, d->scale,
+                            d->score_mode, d->dist};
+        void* out = last ? x_out : act[l & 1];
+        rs_status st = rs_block_fwd(ctx, &bd, &weights[l], cur, out, last ? scores_last : nullptr, last ? keep_last : nullptr,
+                                    nullptr, base, p.block_ws, stream);
+        if (st != RS_OK) return st;
+        cur = out;
+        n -= drops[l];
+    }
+    return RS_OK;
+}
+
+}  // extern "C"

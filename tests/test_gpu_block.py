@@ -239,3 +239,23 @@ def test_graph_replay_equals_eager(ctx):
             assert torch.equal(a["scores"], b["scores"])
     assert model.launches_per_forward(B, N, D) == 9 * L - 1      # the block that drops nothing has no gather
     ctx.async_status()
+
+
+def test_vit_fwd_equals_the_block_loop(ctx):
+    """rs_vit_fwd is the layer loop inside the library: same kernels, bit-identical to chaining rs_block_fwd."""
+    import paper_2508_00367_b200 as rs
+    from paper_2508_00367_b200 import synth
+    B, N, D, H = 2, 197, 384, 6
+    drops = [16, 0, 20, 5]
+    x = synth.make_tokens(B, N, D, "bf16", seed=61).to(torch.bfloat16).cuda()
+    blocks = [synth.make_block_weights(D, 4 * D, "bf16", seed=70 + l) for l in range(len(drops))]
+    model = rs.PrunedViT(ctx, blocks, H, drops, torch.bfloat16)
+    want = model.forward(x)[-1]
+    got = ctx.vit_fwd(x, model.weights, H, drops)
+    torch.cuda.synchronize()
+    assert torch.equal(got["keep_idx"], want["keep_idx"])
+    assert torch.equal(got["scores"], want["scores"])
+    assert torch.equal(got["x_out"].view(torch.int16), want["x_out"].view(torch.int16))
+    with pytest.raises(rs.RsError):
+        ctx.vit_fwd(x, model.weights, H, [16, 0, 20, 161])      # the last block cannot drop all its tokens
+    ctx.async_status()

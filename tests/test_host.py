@@ -42,6 +42,18 @@ def test_workspace_query_needs_no_gpu():
     assert lib.rs_block_workspace_bytes(ctypes.byref(bad)) == 0
 
 
+def test_vit_workspace_query_needs_no_gpu():
+    from paper_2508_00367_b200 import binding
+    lib = binding.load_library()
+    d = binding.VitDesc(1, 64, 197, 768, 12, 3072, 3, 1, 0.0, 0.0, 0, 0)
+    drops = (ctypes.c_int * 3)(16, 0, 16)
+    n = lib.rs_vit_workspace_bytes(ctypes.byref(d), drops)
+    blk = lib.rs_block_workspace_bytes(ctypes.byref(binding.BlockDesc(1, 1, 64, 197, 768, 12, 3072, 16, 1, 0.0, 0.0, 0, 0)))
+    assert n >= blk + 2 * 64 * 197 * 768 * 2          # largest block scratch + two token buffers
+    bad = (ctypes.c_int * 3)(16, 0, 181)               # the last block would drop all of its 181 tokens
+    assert lib.rs_vit_workspace_bytes(ctypes.byref(d), bad) == 0
+
+
 def test_workload_schedules():
     from paper_2508_00367_b200 import synth
     w = synth.WORKLOADS
