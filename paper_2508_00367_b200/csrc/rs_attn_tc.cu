@@ -392,6 +392,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 }
                 // Tile B's first pass of an item starts when tile A's has ended: the two groups then
                 // stay out of step, and one group's loads, stores and waits hide behind the other's pass.
+                // (Tile A cannot get two items ahead of this wait: its item n+2 needs the MMA thread past
+                // tile B's P V of item n, and tile B reaches its next wait about a pass sooner than tile A
+                // can arrive again; were that ever inverted, the wait is bounded and reports.)
                 if (j == 0 && g == 1 && !__all_sync(0xffffffffu, mbar_wait(first_pass, item_n & 1u, abort_flag))) { ok = false; break; }
                 l_run += valid == BKV ? exp_pass<128, false>(r, sl, -m_l2, valid)
                          : ncol == 128 ? exp_pass<128, true>(r, sl, -m_l2, valid)
