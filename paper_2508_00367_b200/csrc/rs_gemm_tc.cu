@@ -421,7 +421,7 @@ cudaError_t launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUt
 int pick_bn(long long M, int N, int sm_count) {
     const long long pairs = sm_count / 2, mt = (M + 2 * BM - 1) / (2 * BM);
     const int widths[3] = {256, 192, 128};
-    const int penalty[3] = {100, 104, 112};
+    const int penalty[3] = {100, 110, 116};
     int best = 128;
     long long best_cost = -1;
     for (int i = 0; i < 3; ++i) {
