@@ -141,6 +141,19 @@ def test_block_video_tokens_ar1(ctx):
     _check_block(res, ref, "bf16", torch.float32)
 
 
+def test_block_video_vit_l14_token_count(ctx):
+    """One block at the video ViT-L/14 size (16 frames x 256 patches + CLS = 4097 tokens, D = 1024,
+    16 heads, 25 % dropped), one sample: the long-sequence attention path (33 key tiles, one CTA per
+    item), the radix selection and every GEMM shape of that workload, against the oracle."""
+    B, N, D, H = 1, 4097, 1024, 16
+    x = synth.make_tokens(B, N, D, "bf16", frames=16, seed=3)
+    w = synth.make_block_weights(D, 4 * D, "bf16", seed=4)
+    r = N // 4
+    ref = orc.block_fwd(x.double().numpy(), _np(w), H, r)
+    res = _run_block(ctx, x, w, H, r, "bf16", torch.float32)
+    _check_block(res, ref, "bf16", torch.float32)
+
+
 def test_block_rejects_bad_arguments(ctx):
     import paper_2508_00367_b200 as rs
     x = synth.make_tokens(1, 8, 64, "bf16", seed=1)
