@@ -343,7 +343,7 @@ def run_gpu(args, wl):
     n_launch = sum(v["launches"] for v in per.values()) / tsteps
     raw_ms = {k: v["ms"] / tsteps for k, v in per.items()}
     ev_us = max(0.0, (sum(raw_ms.values()) - ms_eager) / max(n_launch, 1.0) * 1e3)
-    cls_ms = {k: max(raw_ms[k] - per[k]["launches"] / tsteps * ev_us * 1e-3, 1e-9) for k in per}
+    cls_ms = {k: (max(raw_ms[k] - per[k]["launches"] / tsteps * ev_us * 1e-3, 1e-9) if per[k]["launches"] else 0.0) for k in per}
     gemm_ms, attn_ms = cls_ms["gemm"], cls_ms["attn"]
     tc = ctx.uses_tensor_cores(tdt)
     peak_tf = peaks["bf16_tflops_sustained"]
@@ -363,7 +363,8 @@ def run_gpu(args, wl):
     parts = {
         "attn": dict(ms_per_step=attn_ms, tflops=af / (attn_ms * 1e-3) / 1e12,
                      frac_of_bf16_peak=af / (attn_ms * 1e-3) / 1e12 / peaks["bf16_tflops"]),
-        "gather": dict(ms_per_step=cls_ms["gather"], gbs=gather_bytes / (cls_ms["gather"] * 1e-3) / 1e9),
+        "gather": dict(ms_per_step=cls_ms["gather"], gbs=(gather_bytes / (cls_ms["gather"] * 1e-3) / 1e9 if cls_ms["gather"] else 0.0),
+                       note="selection and gather are one kernel for N <= 1024"),
         "select": dict(ms_per_step=cls_ms["select"]),
         "layernorm": dict(ms_per_step=cls_ms["layernorm"]),
         "note": "in-situ, event overhead subtracted; activations between kernels sit in the 126 MB L2 "

@@ -251,6 +251,10 @@ rs_status rs_topk_compact(rs_ctx* ctx, rs_dtype dtype, int B, int N, int D, int 
         const size_t xbytes = (size_t)B * N * D * sz, obytes = (size_t)B * K * D * sz;
         if (xa < xo + obytes && xo < xa + xbytes) return fail(ctx, RS_ERR_INVALID_ARG, "rs_topk_compact: x_out overlaps x");
     }
+    if (x && rs::select_gather_fusable(N, K)) {
+        RS_CHECK_LAUNCH(ctx, RS_K_GATHER, st, rs::launch_select_gather(scores, 0, nullptr, B, N, K, has_cls ? 1 : 0, keep_idx, dtype, x, D, x_out, ctx->sm_count, st), "select+gather launch");
+        return RS_OK;
+    }
     RS_CHECK_LAUNCH(ctx, RS_K_SELECT, st, rs::launch_select(scores, 0, nullptr, B, N, K, has_cls ? 1 : 0, keep_idx, st), "select launch");
     if (x) RS_CHECK_LAUNCH(ctx, RS_K_GATHER, st, rs::launch_gather(dtype, x, keep_idx, B, N, K, D, x_out, st), "gather launch");
     return RS_OK;
@@ -351,10 +355,14 @@ rs_status rs_block_fwd(rs_ctx* ctx, const rs_block_desc* d, const rs_block_weigh
         RS_CHECK_LAUNCH(ctx, RS_K_SCORE, st, rs::launch_residual_score(m, x_prime, x, d->dtype, T, D, d->score_mode, d->dist, d->out_dtype, x_hat, s, st), "residual+score");
     }
     // reduced token set                                                   (Sec. 3.1)
-    if (nparts > 0)
-        RS_CHECK_LAUNCH(ctx, RS_K_SELECT, st, rs::launch_select(m, nparts | ((int)d->dist << 16), s, d->B, d->N, K, d->has_cls ? 1 : 0, keep, st), "select");
-    else
-        RS_CHECK_LAUNCH(ctx, RS_K_SELECT, st, rs::launch_select(s, 0, nullptr, d->B, d->N, K, d->has_cls ? 1 : 0, keep, st), "select");
+    const float* sel_in = nparts > 0 ? m : s;
+    const int sel_enc = nparts > 0 ? (nparts | ((int)d->dist << 16)) : 0;
+    float* sel_out = nparts > 0 ? s : nullptr;
+    if (x_hat != x_out && rs::select_gather_fusable(d->N, K)) {
+        RS_CHECK_LAUNCH(ctx, RS_K_GATHER, st, rs::launch_select_gather(sel_in, sel_enc, sel_out, d->B, d->N, K, d->has_cls ? 1 : 0, keep, d->out_dtype, x_hat, D, x_out, ctx->sm_count, st), "select+gather");
+        return RS_OK;
+    }
+    RS_CHECK_LAUNCH(ctx, RS_K_SELECT, st, rs::launch_select(sel_in, sel_enc, sel_out, d->B, d->N, K, d->has_cls ? 1 : 0, keep, st), "select");
     if (x_hat != x_out)
         RS_CHECK_LAUNCH(ctx, RS_K_GATHER, st, rs::launch_gather(d->out_dtype, x_hat, keep, d->B, d->N, K, D, x_out, st), "gather");
     return RS_OK;

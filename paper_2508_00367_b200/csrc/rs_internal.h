@@ -74,6 +74,11 @@ cudaError_t launch_select(const float* scores, int nparts, float* scores_out, in
                           int has_cls, int32_t* keep_idx, cudaStream_t st);
 cudaError_t launch_gather(rs_dtype dtype, const void* x, const int32_t* keep_idx, int B, int N, int K,
                           int D, void* x_out, cudaStream_t st);
+// Selection and compaction in one kernel (N <= 1024 and something is dropped).
+bool select_gather_fusable(int N, int K);
+cudaError_t launch_select_gather(const float* scores, int nparts, float* scores_out, int B, int N, int K, int has_cls,
+                                 int32_t* keep_idx, rs_dtype dtype, const void* x, int D, void* x_out, int sm_count,
+                                 cudaStream_t st);
 size_t select_smem_bytes(int N);
 cudaError_t select_init();   // opt in to large dynamic shared memory once per process/device
 

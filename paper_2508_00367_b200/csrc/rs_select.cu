@@ -221,6 +221,86 @@ select_small_kernel(const float* __restrict__ scores, int nparts, float* __restr
     if (keep && pos < K) keep_idx[(long long)b * K + pos] = i;
 }
 
+// Selection and compaction in one launch for N <= 1024.  Grid (G, B): every CTA of sample b
+// repeats the (cheap) counting selection of select_small_kernel, so no CTA waits for another;
+// CTA 0 of the sample writes the index list (and the finished scores), and each CTA copies its
+// share of the kept rows, a warp per row, all 16-byte loads of a row before its stores.
+template <int MAXV>
+__global__ void __launch_bounds__(1024)
+select_gather_small_kernel(const float* __restrict__ scores, int nparts, float* __restrict__ scores_out, int N,
+                           int K, int has_cls, int32_t* __restrict__ keep_idx, const uint4* __restrict__ x,
+                           int row_vecs, uint4* __restrict__ x_out) {
+    __shared__ uint32_t keys[1024];
+    __shared__ int32_t kept[1024];
+    __shared__ int wsum[32];
+    __shared__ int sh_total;
+    grid_dep_launch();
+    grid_dep_wait();
+    const int b = blockIdx.y, i = threadIdx.x;
+    const int first = has_cls ? 1 : 0, want = K - first;
+    uint32_t key = 0;
+    if (i < N) {
+        float s;
+        if (nparts > 0) {                  // per-tile partial sums from the GEMM epilogue
+            s = finish_score(scores + ((long long)b * N + i) * partial_stride(nparts), nparts);
+            if (scores_out && blockIdx.x == 0) scores_out[(long long)b * N + i] = s;
+        } else {
+            s = scores[(long long)b * N + i];
+        }
+        key = score_key(s);
+        keys[i] = key;
+    }
+    __syncthreads();
+    int keep = 0;
+    if (i < N) {
+        if (i < first) {
+            keep = 1;
+        } else if (want > 0) {
+            int rank = 0;
+            int j = first;
+            for (; j + 4 <= N; j += 4) {   // keys[j] is a broadcast read: every thread reads the same word
+                const uint32_t k0 = keys[j], k1 = keys[j + 1], k2 = keys[j + 2], k3 = keys[j + 3];
+                rank += (k0 > key) || (k0 == key && j < i);
+                rank += (k1 > key) || (k1 == key && j + 1 < i);
+                rank += (k2 > key) || (k2 == key && j + 2 < i);
+                rank += (k3 > key) || (k3 == key && j + 3 < i);
+            }
+            for (; j < N; ++j) {
+                const uint32_t k0 = keys[j];
+                rank += (k0 > key) || (k0 == key && j < i);
+            }
+            keep = rank < want;
+        }
+    }
+    const int pos = block_exclusive_scan(keep, wsum, &sh_total);
+    if (keep && pos < K) {
+        kept[pos] = i;
+        if (blockIdx.x == 0) keep_idx[(long long)b * K + pos] = i;
+    }
+    __syncthreads();
+    // rows [lo, hi) of the sample's K kept rows belong to this CTA
+    const int G = gridDim.x, per = (K + G - 1) / G;
+    const int lo = blockIdx.x * per, hi = min(lo + per, K);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    for (int r = lo + warp; r < hi; r += nwarps) {
+        const uint4* src = x + ((long long)b * N + kept[r]) * row_vecs;
+        uint4* dst = x_out + ((long long)b * K + r) * row_vecs;
+        for (int base = 0; base < row_vecs; base += 32 * MAXV) {
+            uint4 v[MAXV];
+#pragma unroll
+            for (int j = 0; j < MAXV; ++j) {
+                const int iv = base + j * 32 + lane;
+                if (iv < row_vecs) v[j] = __ldg(src + iv);
+            }
+#pragma unroll
+            for (int j = 0; j < MAXV; ++j) {
+                const int iv = base + j * 32 + lane;
+                if (iv < row_vecs) dst[iv] = v[j];
+            }
+        }
+    }
+}
+
 // Nothing dropped (K == N): every token is kept, in order; only the scores remain to be
 // finished when they arrive as per-tile partial sums of squares.
 __global__ void __launch_bounds__(256)
@@ -284,6 +364,22 @@ cudaError_t launch_select(const float* scores, int nparts, float* scores_out, in
     }
     return launch_pdl(select_kernel, dim3(B), dim3(kSelThreads), select_smem_bytes(N), st, scores, nparts, scores_out, N, K,
                       has_cls, keep_idx);
+}
+
+bool select_gather_fusable(int N, int K) { return N <= 1024 && K < N; }
+
+cudaError_t launch_select_gather(const float* scores, int nparts, float* scores_out, int B, int N, int K, int has_cls,
+                                 int32_t* keep_idx, rs_dtype dtype, const void* x, int D, void* x_out, int sm_count,
+                                 cudaStream_t st) {
+    if (B == 0) return cudaSuccess;
+    const int row_vecs = (int)((size_t)D * dtype_size(dtype) / 16);
+    // enough CTAs per sample for about three waves over the SMs, at least a few rows each
+    int G = (3 * sm_count + B - 1) / B;
+    G = G < 1 ? 1 : G;
+    if (G > (K + 3) / 4) G = (K + 3) / 4;
+    if (G < 1) G = 1;
+    return launch_pdl(select_gather_small_kernel<4>, dim3(G, B), dim3((N + 31) / 32 * 32 < 128 ? 128 : (N + 31) / 32 * 32), 0, st,
+                      scores, nparts, scores_out, N, K, has_cls, keep_idx, (const uint4*)x, row_vecs, (uint4*)x_out);
 }
 
 cudaError_t launch_gather(rs_dtype dtype, const void* x, const int32_t* keep_idx, int B, int N, int K,

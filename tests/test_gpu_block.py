@@ -250,7 +250,7 @@ def test_graph_replay_equals_eager(ctx):
             assert torch.equal(a["keep_idx"], b["keep_idx"])
             assert torch.equal(a["x_out"].view(torch.int16), b["x_out"].view(torch.int16))
             assert torch.equal(a["scores"], b["scores"])
-    assert model.launches_per_forward(B, N, D) == 9 * L - 1      # the block that drops nothing has no gather
+    assert model.launches_per_forward(B, N, D) == 8 * L          # selection and gather are one kernel here; the block that drops nothing has neither
     ctx.async_status()
 
 
