@@ -45,7 +45,8 @@ template <int BN> struct Cfg {
     static constexpr int SPLIT = (BN == 128) ? 64 : 128;           // epilogue warps 2-5 take columns [0, SPLIT)
     static constexpr int OFF_STG = STAGES * STAGE_BYTES;
     static constexpr int OFF_BAR = OFF_STG + kStgBufs * STG_BYTES;
-    static constexpr size_t SMEM = (size_t)OFF_BAR + 256 /*barriers*/ + 1024 /*align slack*/;
+    static constexpr int OFF_BIAS = OFF_BAR + 256;                 // float [2 halves][128]: the tile's bias slice
+    static constexpr size_t SMEM = (size_t)OFF_BIAS + 1024 + 1024 /*align slack*/;
 };
 
 struct GemmArgs {
@@ -201,6 +202,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const uint32_t stg_row = (uint32_t)(trow >> 3) * 1024u + (uint32_t)(trow & 7) * 128u;
         const int r8 = trow & 7;
         const bool storer = (q == 0 && lane == 0);       // issues this half's TMA stores
+        float* bias_s = reinterpret_cast<float*>(smem + C::OFF_BIAS) + half * 128;
+        const int t128 = ((warp - 2) & 3) * 32 + lane;   // this thread's index among the 128 of its half
         const uint32_t lead_tempty[2] = {map_to_cta(smem_u32(&tempty[0]), 0), map_to_cta(smem_u32(&tempty[1]), 0)};
         uint32_t tl = 0, blk_ctr = 0;
         constexpr int RES_VECS = EPI == EPI_RESID ? 4 : EPI == EPI_SCORE ? 8 : 1;   // 16-byte loads per 32 columns
@@ -225,6 +228,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             load_res(c_begin, res_next);
             // The four warps of a column half decide together whether to go on: the named
             // barriers below have no time limit, so no warp may leave the loop alone.
+            // this half's slice of the bias goes to shared memory while the accumulator is still being
+            // computed (the barrier below publishes it): the chunk loop then has no global read on its chain
+            if (c_begin + t128 < c_end) bias_s[t128] = args.bias ? __ldg(args.bias + n0 + c_begin + t128) : 0.f;
             if (!__all_sync(0xffffffffu, mbar_wait(&tfull[a], aph, abort_flag))) half_fail[half] = 1;
             named_barrier(1 + half, 128);
             if (half_fail[half]) break;
@@ -252,8 +258,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 float v[32];
 #pragma unroll
                 for (int j = 0; j < 32; j += 4) {
-                    float4 b = args.bias ? __ldg(reinterpret_cast<const float4*>(args.bias + col + j))
-                                         : make_float4(0.f, 0.f, 0.f, 0.f);
+                    const float4 b = *reinterpret_cast<const float4*>(bias_s + (c - c_begin) + j);
                     v[j] = __uint_as_float(r[j]) + b.x;
                     v[j + 1] = __uint_as_float(r[j + 1]) + b.y;
                     v[j + 2] = __uint_as_float(r[j + 2]) + b.z;
