@@ -158,6 +158,8 @@ rs_status rs_async_status(rs_ctx* ctx, void* stream) {
     if (e != cudaSuccess) return cuda_fail(ctx, e, "status read");
     if (word != RS_DEV_OK) {
         cudaMemset(ctx->d_status, 0, sizeof(int));
+        if (word == RS_DEV_SMEM_ALIGN)
+            return fail(ctx, RS_ERR_CUDA, "device status word = %d (a kernel's shared memory window was not 1024-byte aligned)", word);
         return fail(ctx, RS_ERR_TIMEOUT, "device status word = %d (a bounded wait expired)", word);
     }
     return RS_OK;

@@ -8,7 +8,8 @@
 // pair tile does twice the arithmetic of a 128 x 128 tile, which is what lifts the kernel off
 // the L2 -> SM bandwidth bound.  The fp32 accumulator is double-buffered in tensor memory, so
 // the eight epilogue warps of each CTA drain tile i (tcgen05.ld -> bias / GELU / residual /
-// score -> swizzled shared memory -> TMA store) while the main loop of tile i+1 runs.
+// score -> swizzled shared memory -> one TMA store per warp and 128-byte column block) while the
+// main loop of tile i+1 runs.
 //
 // Epilogues (Eq. att, Eq. MLP, Sec. 3.2):
 //   EPI_BIAS       out = acc + b                          -> bf16      (QKV projection)
@@ -34,8 +35,8 @@ constexpr int BK = 64;
 constexpr int kThreads = 320;                 // warp 0: TMA, warp 1: MMA (leader CTA), warps 2-9: epilogue
 constexpr int kEpiWarps = 8;
 constexpr int A_BYTES = BM * BK * 2;          // 16 KB
-constexpr int STG_BYTES = 128 * 128;          // one staged output block: 128 rows of 128 bytes
-constexpr int kStgBufs = 4;                   // two per column half
+constexpr int STG_BYTES = 32 * 128;           // one staged output block of a warp: its 32 rows of 128 bytes
+constexpr int kStgBufs = 2 * kEpiWarps;       // two per epilogue warp
 
 template <int BN> struct Cfg {
     static constexpr int B_BYTES = (BN / 2) * BK * 2;              // this CTA's half of the W tile
@@ -45,8 +46,9 @@ template <int BN> struct Cfg {
     static constexpr int SPLIT = (BN == 128) ? 64 : 128;           // epilogue warps 2-5 take columns [0, SPLIT)
     static constexpr int OFF_STG = STAGES * STAGE_BYTES;
     static constexpr int OFF_BAR = OFF_STG + kStgBufs * STG_BYTES;
-    static constexpr int OFF_BIAS = OFF_BAR + 256;                 // float [2 halves][128]: the tile's bias slice
-    static constexpr size_t SMEM = (size_t)OFF_BIAS + 1024 + 1024 /*align slack*/;
+    static constexpr int OFF_BIAS = OFF_BAR + 256;                 // float [2 tile parities][2 halves][128]: bias slices
+    static constexpr size_t SMEM = (size_t)OFF_BIAS + 2048;        // the window itself must be 1024-byte aligned
+    static_assert(SMEM <= 227 * 1024, "shared memory of one CTA");
 };
 
 struct GemmArgs {
@@ -95,8 +97,14 @@ __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmOut, const GemmArgs args) {
     using C = Cfg<BN>;
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    // The 128-byte swizzle wants 1024-byte aligned stage and staging buffers, and the layout leaves no
+    // room to round the base up: a window that is not aligned is reported, and nothing else is done.
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    uint8_t* smem = smem_raw;
+    if (smem_u32(smem) & 1023u) {
+        if (threadIdx.x == 0) atomicExch(args.status, RS_DEV_SMEM_ALIGN);
+        return;
+    }
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::OFF_BAR);
     uint64_t* full = bars;                       // [STAGES] leader's: both CTAs' operands landed
     uint64_t* empty = bars + C::STAGES;          // [STAGES] per CTA: the MMAs reading the stage retired
@@ -199,10 +207,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         constexpr int BLK_COLS = 128 / (int)sizeof(OutT);            // columns in one staged 128-byte row
         constexpr int CHUNKS_PER_BLK = BLK_COLS / 32;                // 32-column TMEM loads per staged block
         const int trow = q * 32 + lane;                  // row inside this CTA's half of the tile
-        const uint32_t stg_row = (uint32_t)(trow >> 3) * 1024u + (uint32_t)(trow & 7) * 128u;
-        const int r8 = trow & 7;
-        const bool storer = (q == 0 && lane == 0);       // issues this half's TMA stores
-        float* bias_s = reinterpret_cast<float*>(smem + C::OFF_BIAS) + half * 128;
+        const uint32_t stg_row = (uint32_t)(lane >> 3) * 1024u + (uint32_t)(lane & 7) * 128u;   // inside the warp's 32-row slab
+        const int r8 = lane & 7;
         const int t128 = ((warp - 2) & 3) * 32 + lane;   // this thread's index among the 128 of its half
         const uint32_t lead_tempty[2] = {map_to_cta(smem_u32(&tempty[0]), 0), map_to_cta(smem_u32(&tempty[1]), 0)};
         uint32_t tl = 0, blk_ctr = 0;
@@ -229,7 +235,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             // The four warps of a column half decide together whether to go on: the named
             // barriers below have no time limit, so no warp may leave the loop alone.
             // this half's slice of the bias goes to shared memory while the accumulator is still being
-            // computed (the barrier below publishes it): the chunk loop then has no global read on its chain
+            // computed (the barrier below publishes it): the chunk loop then has no global read on its chain.
+            // Two copies, by tile parity: a warp may still be reading the last tile's slice.
+            float* bias_s = reinterpret_cast<float*>(smem + C::OFF_BIAS) + (tl & 1u) * 256 + half * 128;
             if (c_begin + t128 < c_end) bias_s[t128] = args.bias ? __ldg(args.bias + n0 + c_begin + t128) : 0.f;
             if (!__all_sync(0xffffffffu, mbar_wait(&tfull[a], aph, abort_flag))) half_fail[half] = 1;
             named_barrier(1 + half, 128);
@@ -240,7 +248,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll 1
             for (int c = c_begin; c < c_end; c += 32) {
                 const int cb = (c / 32) % CHUNKS_PER_BLK;            // chunk inside the staged block
-                uint8_t* stg = smem + C::OFF_STG + (half * 2 + (blk_ctr & 1u)) * STG_BYTES;
+                uint8_t* stg = smem + C::OFF_STG + ((warp - 2) * 2 + (blk_ctr & 1u)) * STG_BYTES;
+                if (cb == 0) {
+                    // the store that last read this buffer (two blocks ago) must be done with it
+                    if (lane == 0) tma_store_wait_read<1>();
+                    __syncwarp();
+                }
                 uint4 res[RES_VECS];
 #pragma unroll
                 for (int j = 0; j < RES_VECS; ++j) res[j] = res_next[j];
@@ -335,14 +348,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                             make_float4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
                 }
                 if (cb == CHUNKS_PER_BLK - 1) {
+                    // Every warp stores its own 32 rows: no barrier between the warps of a tile.
                     fence_async_smem();                  // staged data visible to the TMA engine
-                    // One barrier per block: before it the storer makes sure the previous store has
-                    // finished reading the other buffer, so after it that buffer is free for the
-                    // next block while this block's store is in flight.
-                    if (storer) tma_store_wait_read<0>();
-                    named_barrier(1 + half, 128);
-                    if (storer && m0 < args.M) {          // rows past M are dropped by the tensor map's bounds
-                        tma_store_2d(&tmOut, stg, col + 32 - BLK_COLS, m0);
+                    __syncwarp();
+                    if (lane == 0) {
+                        if (m0 + q * 32 < args.M)        // rows past M are dropped by the tensor map's bounds
+                            tma_store_2d(&tmOut, stg, col + 32 - BLK_COLS, m0 + q * 32);
                         tma_store_commit();
                     }
                     ++blk_ctr;
@@ -357,7 +368,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 }
             }
         }
-        if (storer) tma_store_wait<0>();                 // all output written before the CTA exits
+        if (lane == 0) tma_store_wait<0>();              // all output written before the CTA exits
     }
 
     tc_fence_before();
@@ -466,7 +477,7 @@ cudaError_t launch_gemm_tc(rs_ctx* ctx, int epi, const void* A, const void* W, c
     CUtensorMap tmA, tmB, tmOut;
     if (!make_tmap_2d(ctx->encode_tiled, &tmA, A, 2, (uint64_t)M, (uint64_t)K, BM) ||
         !make_tmap_2d(ctx->encode_tiled, &tmB, W, 2, (uint64_t)N, (uint64_t)K, (uint32_t)(bn / 2)) ||
-        !make_tmap_2d(ctx->encode_tiled, &tmOut, out, out_bytes, (uint64_t)M, (uint64_t)N, BM))
+        !make_tmap_2d(ctx->encode_tiled, &tmOut, out, out_bytes, (uint64_t)M, (uint64_t)N, 32))
         return cudaErrorInvalidValue;
     GemmArgs args;
     args.M = (int)M; args.N = N; args.K = K; args.bias = bias; args.residual = residual;

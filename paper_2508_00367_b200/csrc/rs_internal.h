@@ -25,7 +25,7 @@ struct rs_ctx {
 enum { kMaxTimed = 8192 };
 
 // Device status word values.
-enum { RS_DEV_OK = 0, RS_DEV_TIMEOUT = 1 };
+enum { RS_DEV_OK = 0, RS_DEV_TIMEOUT = 1, RS_DEV_SMEM_ALIGN = 2 };
 
 namespace rs {
 
