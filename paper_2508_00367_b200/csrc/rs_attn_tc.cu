@@ -244,7 +244,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     } else if (warp == 9) {
         // ---------------- MMA issuer ----------------
         if (elect_one() && blockIdx.x < args.n_items) {
-            const uint32_t idesc_o = idesc_bf16(BQ, DH, 0, 1);
+            constexpr uint32_t idesc_o = idesc_bf16(BQ, DH, 0, 1), idesc_s_full = idesc_bf16(BQ, BKV, 0, 0);
+            // descriptors as halves: per product only the low half moves (address >> 4)
+            constexpr uint32_t kTile16 = TILE_BYTES >> 4;
+            const uint32_t desc_hi = smem_desc_hi(smem_desc_sw128(0, 16, 1024));
+            const uint32_t q_lo = smem_desc_lo(smem_desc_sw128(smem_u32(smem + OFF_Q), 16, 1024));
+            const uint32_t k_lo = smem_desc_lo(smem_desc_sw128(smem_u32(smem + OFF_K), 16, 1024));
+            const uint32_t v_lo = smem_desc_lo(smem_desc_sw128(smem_u32(smem + OFF_V), 16, 1024));
             uint32_t ns[2] = {0, 0}, np[2] = {0, 0};     // S tiles / P V products issued so far per query tile
             bool ok = true;
             // S_g = Q_g K^T : both operands K-major (head dimension contiguous).  The S columns must
@@ -252,12 +258,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             auto issue_s = [&](int g, uint32_t qb, int stage, int valid) {
                 if (ns[g] > 0 && !mbar_wait(&s_free[g], (ns[g] - 1) & 1u, abort_flag)) { ok = false; return; }
                 tc_fence_after();
-                const uint32_t idesc_s = idesc_bf16(BQ, (valid + 15) & ~15, 0, 0);
-                const uint64_t dq = smem_desc_sw128(smem_u32(smem + OFF_Q + (qb * 2 + g) * TILE_BYTES), 16, 1024);
-                const uint64_t dk = smem_desc_sw128(smem_u32(smem + OFF_K + stage * TILE_BYTES), 16, 1024);
+                const uint32_t idesc_s = valid == BKV ? idesc_s_full : idesc_bf16(BQ, (valid + 15) & ~15, 0, 0);
+                const uint32_t dq = q_lo + (qb * 2 + g) * kTile16, dk = k_lo + (uint32_t)stage * kTile16;
 #pragma unroll
-                for (int k = 0; k < DH / 16; ++k)
-                    mma_ss(tmem_base + g * BKV, dq + 2u * k, dk + 2u * k, idesc_s, k != 0);
+                for (int k = 0; k < DH / 16; ++k)        // 16 head-dimension columns = 32 bytes per step
+                    mma_ss_lh(tmem_base + g * BKV, dq + 2u * k, dk + 2u * k, desc_hi, idesc_s, k != 0);
                 mma_commit(&s_full[g]);
                 ++ns[g];
             };
@@ -266,11 +271,17 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             auto issue_pv = [&](int g, int stage, int valid, bool first) {
                 if (!mbar_wait(&p_ready[g], np[g] & 1u, abort_flag)) { ok = false; return; }
                 tc_fence_after();
-                const int ksteps = (valid + 15) >> 4;
-                const uint32_t sv = smem_u32(smem + OFF_V + stage * TILE_BYTES);
-                for (int k = 0; k < ksteps; ++k)
-                    mma_ts(tmem_base + kOCol + g * DH, tmem_base + kPCol + g * DH + 8 * k,
-                           smem_desc_sw128(sv + (uint32_t)k * 2048u, 16, 1024), idesc_o, !(first && k == 0));
+                const uint32_t dv = v_lo + (uint32_t)stage * kTile16;
+                const uint32_t o_col = tmem_base + kOCol + g * DH, p_col = tmem_base + kPCol + g * DH;
+                if (valid == BKV) {
+#pragma unroll
+                    for (int k = 0; k < BKV / 16; ++k)
+                        mma_ts_lh(o_col, p_col + 8 * k, dv + 128u * k, desc_hi, idesc_o, k == 0 ? !first : 1u);
+                } else {
+                    const int ksteps = (valid + 15) >> 4;
+                    for (int k = 0; k < ksteps; ++k)
+                        mma_ts_lh(o_col, p_col + 8 * k, dv + 128u * k, desc_hi, idesc_o, !(first && k == 0));
+                }
                 mma_commit(&o_done[g]);
                 ++np[g];
             };
