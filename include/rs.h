@@ -183,7 +183,8 @@ RS_API rs_status rs_block_fwd(rs_ctx* ctx, const rs_block_desc* desc /*host*/,
  * [0, N_l - 1].  x (dev): [B, N, D].  x_out (dev): [B, N_L, D] with N_L = N - sum(drops).
  * scores_last / keep_last (dev, optional): the last block's scores [B, N_{L-1}] and kept
  * indices [B, N_L].  workspace (dev): at least rs_vit_workspace_bytes() bytes, 256-byte
- * aligned; it holds one block's scratch and two token buffers the blocks alternate between. */
+ * aligned; it holds one block's scratch, two token buffers the blocks alternate between and
+ * one buffer for the normalised input of the next block. */
 typedef struct {
     rs_dtype dtype;
     int B, N, D, H, D_mlp, L;
@@ -194,7 +195,23 @@ typedef struct {
     rs_dist dist;
 } rs_vit_desc;
 
+/* Optional per-block outputs of the layer loop.  Each member is NULL or a host array of L device
+ * pointers, any of which may be NULL (x_out[L-1], the result, is required).  x_out[l]: block l's
+ * compacted output [B, N_{l+1}, D]; scores[l]: [B, N_l] fp32; keep_idx[l]: [B, N_{l+1}] int32. */
+typedef struct {
+    void* const* x_out;
+    float* const* scores;
+    int32_t* const* keep_idx;
+} rs_vit_taps;
+
 RS_API size_t rs_vit_workspace_bytes(const rs_vit_desc* desc /*host*/, const int* drops /*host[L]*/);
+/* The layer loop with every block's outputs available.  Same computation as rs_vit_fwd.  In both,
+ * the compaction kernel of a block that drops tokens also writes LN1 of the next block's input
+ * (the kept row is in its registers), so a block after a pruning block launches no LN1 kernel. */
+RS_API rs_status rs_vit_fwd_taps(rs_ctx* ctx, const rs_vit_desc* desc /*host*/,
+                                 const rs_block_weights* weights /*host[L]*/, const int* drops /*host[L]*/,
+                                 const void* x, const rs_vit_taps* taps /*host*/, void* workspace,
+                                 size_t workspace_bytes, void* stream);
 RS_API rs_status rs_vit_fwd(rs_ctx* ctx, const rs_vit_desc* desc /*host*/,
                             const rs_block_weights* weights /*host[L]*/, const int* drops /*host[L]*/,
                             const void* x, void* x_out, float* scores_last, int32_t* keep_last,

@@ -26,7 +26,8 @@ STATUS_NAMES = {0: "RS_OK", 1: "RS_ERR_INVALID_ARG", 2: "RS_ERR_UNSUPPORTED", 3:
 EXPORTS = ("rs_create", "rs_destroy", "rs_last_error", "rs_async_status", "rs_uses_tensor_cores",
            "rs_launch_count", "rs_attn_fwd", "rs_shift_score", "rs_topk_compact",
            "rs_block_workspace_bytes", "rs_block_fwd", "rs_timing_enable", "rs_timing_read",
-           "rs_static_scratch_bytes", "rs_block_fwd_static", "rs_linear_fwd", "rs_vit_workspace_bytes", "rs_vit_fwd")
+           "rs_static_scratch_bytes", "rs_block_fwd_static", "rs_linear_fwd", "rs_vit_workspace_bytes", "rs_vit_fwd",
+           "rs_vit_fwd_taps")
 LIN_EPILOGUE = {"bias": 0, "gelu": 1, "residual": 2}
 KERNEL_CLASSES = ("layernorm", "gemm", "attn", "score", "select", "gather")
 
@@ -60,6 +61,12 @@ class VitDesc(ctypes.Structure):
                 ("H", ctypes.c_int), ("D_mlp", ctypes.c_int), ("L", ctypes.c_int), ("has_cls", ctypes.c_int),
                 ("ln_eps", ctypes.c_float), ("scale", ctypes.c_float), ("score_mode", ctypes.c_int),
                 ("dist", ctypes.c_int)]
+
+
+class VitTaps(ctypes.Structure):
+    """Host arrays of L device pointers (or NULL): every block's x_out, scores, keep_idx."""
+    _fields_ = [("x_out", ctypes.POINTER(ctypes.c_void_p)), ("scores", ctypes.POINTER(ctypes.c_void_p)),
+                ("keep_idx", ctypes.POINTER(ctypes.c_void_p))]
 
 
 class BlockWeights(ctypes.Structure):
@@ -120,6 +127,9 @@ def load_library() -> ctypes.CDLL:
     lib.rs_vit_fwd.argtypes = [vp, ctypes.POINTER(VitDesc), ctypes.POINTER(BlockWeights), ctypes.POINTER(ci), vp, vp, vp,
                                vp, vp, ctypes.c_size_t, vp]
     lib.rs_vit_fwd.restype = ci
+    lib.rs_vit_fwd_taps.argtypes = [vp, ctypes.POINTER(VitDesc), ctypes.POINTER(BlockWeights), ctypes.POINTER(ci), vp,
+                                    ctypes.POINTER(VitTaps), vp, ctypes.c_size_t, vp]
+    lib.rs_vit_fwd_taps.restype = ci
     _lib = lib
     return lib
 
@@ -391,19 +401,26 @@ class PrunedViT:
         if self._plan and self._plan["key"] == key:
             return self._plan
         dev = self.ctx.device
-        descs, outs, need, n = [], [], 256, N
-        for l, r in enumerate(self.drops):
-            d = self.ctx.block_desc(B, n, D, self.H, self.weights[l].D_mlp, r, self.dtype, None, self.has_cls,
-                                    0.0, 0.0, self.score_mode)
-            need = max(need, self.ctx.block_workspace_bytes(d))
+        L = len(self.drops)
+        outs, n = [], N
+        for r in self.drops:
             k = n - r
             outs.append(dict(x_out=torch.empty(B, k, D, dtype=self.dtype, device=dev),
                              scores=torch.empty(B, n, dtype=torch.float32, device=dev),
                              keep_idx=torch.empty(B, k, dtype=torch.int32, device=dev)))
-            descs.append(d)
             n = k
+        code = RS_BF16 if self.dtype == torch.bfloat16 else RS_F32
+        desc = VitDesc(code, B, N, D, self.H, self.weights[0].D_mlp, L, int(self.has_cls), 0.0, 0.0,
+                       SCORE_MODE[self.score_mode], DIST["l2"])
+        cdrops = (ctypes.c_int * L)(*[int(r) for r in self.drops])
+        warr = (BlockWeights * L)(*[w.struct for w in self.weights])
+        need = int(self.ctx.lib.rs_vit_workspace_bytes(ctypes.byref(desc), cdrops))
+        if need == 0:
+            raise RsError(1, "rs_vit_fwd: bad descriptor or schedule")
+        arrs = {k: (ctypes.c_void_p * L)(*[o[k].data_ptr() for o in outs]) for k in ("x_out", "scores", "keep_idx")}
+        taps = VitTaps(arrs["x_out"], arrs["scores"], arrs["keep_idx"])
         ws = torch.empty(need, dtype=torch.uint8, device=dev)
-        self._plan = dict(key=key, descs=descs, outs=outs, ws=ws)
+        self._plan = dict(key=key, desc=desc, drops=cdrops, warr=warr, arrs=arrs, taps=taps, outs=outs, ws=ws)
         return self._plan
 
     def forward(self, x: torch.Tensor, graph: bool = False):
@@ -442,14 +459,8 @@ class PrunedViT:
         return int(self.plan(B, N, D).get("launches_per_forward", 0))
 
     def _run(self, x: torch.Tensor, p):
-        lib, h = self.ctx.lib, self.ctx.handle
-        st = _stream(x.device)
-        cur = x
-        for l, d in enumerate(p["descs"]):
-            o = p["outs"][l]
-            rc = lib.rs_block_fwd(h, ctypes.byref(d), ctypes.byref(self.weights[l].struct), _ptr(cur),
-                                  _ptr(o["x_out"]), _ptr(o["scores"]), _ptr(o["keep_idx"]), None,
-                                  _ptr(p["ws"]), p["ws"].numel(), st)
-            if rc != RS_OK:
-                raise RsError(rc, self.ctx.last_error())
-            cur = o["x_out"]
+        """One library call: the layer loop with every block's outputs written to the plan's buffers."""
+        rc = self.ctx.lib.rs_vit_fwd_taps(self.ctx.handle, ctypes.byref(p["desc"]), p["warr"], p["drops"], _ptr(x),
+                                          ctypes.byref(p["taps"]), _ptr(p["ws"]), p["ws"].numel(), _stream(x.device))
+        if rc != RS_OK:
+            raise RsError(rc, self.ctx.last_error())

@@ -7,6 +7,7 @@
 #include <string.h>
 
 #include "rs_internal.h"
+#include <vector>
 
 namespace {
 
@@ -254,11 +255,11 @@ rs_status rs_topk_compact(rs_ctx* ctx, rs_dtype dtype, int B, int N, int D, int 
         if (xa < xo + obytes && xo < xa + xbytes) return fail(ctx, RS_ERR_INVALID_ARG, "rs_topk_compact: x_out overlaps x");
     }
     if (x && rs::select_gather_fusable(N, K)) {
-        RS_CHECK_LAUNCH(ctx, RS_K_GATHER, st, rs::launch_select_gather(scores, 0, nullptr, B, N, K, has_cls ? 1 : 0, keep_idx, dtype, x, D, x_out, ctx->sm_count, st), "select+gather launch");
+        RS_CHECK_LAUNCH(ctx, RS_K_GATHER, st, rs::launch_select_gather(scores, 0, nullptr, B, N, K, has_cls ? 1 : 0, keep_idx, dtype, x, D, x_out, nullptr, ctx->sm_count, st), "select+gather launch");
         return RS_OK;
     }
     RS_CHECK_LAUNCH(ctx, RS_K_SELECT, st, rs::launch_select(scores, 0, nullptr, B, N, K, has_cls ? 1 : 0, keep_idx, st), "select launch");
-    if (x) RS_CHECK_LAUNCH(ctx, RS_K_GATHER, st, rs::launch_gather(dtype, x, keep_idx, B, N, K, D, x_out, st), "gather launch");
+    if (x) RS_CHECK_LAUNCH(ctx, RS_K_GATHER, st, rs::launch_gather(dtype, x, keep_idx, B, N, K, D, x_out, nullptr, st), "gather launch");
     return RS_OK;
 }
 
@@ -268,9 +269,16 @@ size_t rs_block_workspace_bytes(const rs_block_desc* d) {
     return ws.total;
 }
 
-rs_status rs_block_fwd(rs_ctx* ctx, const rs_block_desc* d, const rs_block_weights* w, const void* x,
-                       void* x_out, float* scores, int32_t* keep_idx, void* x_full, void* workspace,
-                       size_t workspace_bytes, void* stream) {
+// The block, with the two hooks the layer loop uses to save one kernel per block: `x_ln`, when
+// non-null, is LN1(x) already computed (by the previous block's compaction); `next_ln`, when
+// non-null, asks for LN(x_out) with the next block's LN1 parameters in next_ln->out, written by the
+// compaction kernel.  *ln_done tells whether that happened (it cannot when nothing is dropped, or
+// when a row does not fit one warp's registers): if not, the next block normalises its input itself.
+static rs_status block_fwd_impl(rs_ctx* ctx, const rs_block_desc* d, const rs_block_weights* w, const void* x,
+                                const void* x_ln, void* x_out, float* scores, int32_t* keep_idx, void* x_full,
+                                void* workspace, size_t workspace_bytes, void* stream, const rs::LnFuse* next_ln,
+                                bool* ln_done) {
+    if (ln_done) *ln_done = false;
     if (!ctx) return RS_ERR_INVALID_ARG;
     if (!d || !w || !x || !x_out) return fail(ctx, RS_ERR_INVALID_ARG, "rs_block_fwd: null argument");
     BlockWs ws;
@@ -328,16 +336,19 @@ rs_status rs_block_fwd(rs_ctx* ctx, const rs_block_desc* d, const rs_block_weigh
     int nparts = 0;
 
     // x' = SA(LN(x)) + x                                                  (Eq. att)
-    RS_CHECK_LAUNCH(ctx, RS_K_LAYERNORM, st, rs::launch_layernorm(d->dtype, d->dtype, x, w->ln1_g, w->ln1_b, eps, T, D, u, st), "LN1");
+    if (!x_ln) {
+        RS_CHECK_LAUNCH(ctx, RS_K_LAYERNORM, st, rs::launch_layernorm(d->dtype, d->dtype, x, w->ln1_g, w->ln1_b, eps, T, D, u, st), "LN1");
+        x_ln = u;
+    }
     if (tc) {
-        RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_tc(ctx, rs::RS_EPI_BIAS, u, w->w_qkv, w->b_qkv, nullptr, nullptr, qkv, RS_BF16, nullptr, 0, 0, T, 3 * D, D, st), "QKV");
+        RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_tc(ctx, rs::RS_EPI_BIAS, x_ln, w->w_qkv, w->b_qkv, nullptr, nullptr, qkv, RS_BF16, nullptr, 0, 0, T, 3 * D, D, st), "QKV");
         RS_CHECK_LAUNCH(ctx, RS_K_ATTN, st, rs::launch_attn_tc(ctx, ad, qkv, kp, vp, o, st), "attention");
         // shift through attention (operation choice (i)): partial sums of (SA(LN(x)) - x)^2 from this epilogue
         nparts = rs::gemm_tc_score_parts(ctx, T, D);
         float* attn_parts = d->score_mode == RS_SCORE_ATTN ? m : nullptr;
         RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_tc(ctx, rs::RS_EPI_RESID, o, w->w_o, w->b_o, x, nullptr, x_prime, RS_F32, attn_parts, 0, (int)d->dist, T, D, D, st), "proj");
     } else {
-        RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_simt(d->dtype, u, w->w_qkv, w->b_qkv, 0, nullptr, RS_F32, qkv, d->dtype, T, 3 * D, D, st), "QKV");
+        RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_simt(d->dtype, x_ln, w->w_qkv, w->b_qkv, 0, nullptr, RS_F32, qkv, d->dtype, T, 3 * D, D, st), "QKV");
         RS_CHECK_LAUNCH(ctx, RS_K_ATTN, st, rs::launch_attn_simt(ad, qkv, kp, vp, o, st), "attention");
         RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_simt(d->dtype, o, w->w_o, w->b_o, 0, x, d->dtype, x_prime, RS_F32, T, D, D, st), "proj");
     }
@@ -360,14 +371,23 @@ rs_status rs_block_fwd(rs_ctx* ctx, const rs_block_desc* d, const rs_block_weigh
     const float* sel_in = nparts > 0 ? m : s;
     const int sel_enc = nparts > 0 ? (nparts | ((int)d->dist << 16)) : 0;
     float* sel_out = nparts > 0 ? s : nullptr;
+    const rs::LnFuse* ln = (next_ln && x_hat != x_out && rs::ln_fusable(d->out_dtype, D)) ? next_ln : nullptr;
+    if (ln && ln_done) *ln_done = true;
     if (x_hat != x_out && rs::select_gather_fusable(d->N, K)) {
-        RS_CHECK_LAUNCH(ctx, RS_K_GATHER, st, rs::launch_select_gather(sel_in, sel_enc, sel_out, d->B, d->N, K, d->has_cls ? 1 : 0, keep, d->out_dtype, x_hat, D, x_out, ctx->sm_count, st), "select+gather");
+        RS_CHECK_LAUNCH(ctx, RS_K_GATHER, st, rs::launch_select_gather(sel_in, sel_enc, sel_out, d->B, d->N, K, d->has_cls ? 1 : 0, keep, d->out_dtype, x_hat, D, x_out, ln, ctx->sm_count, st), "select+gather");
         return RS_OK;
     }
     RS_CHECK_LAUNCH(ctx, RS_K_SELECT, st, rs::launch_select(sel_in, sel_enc, sel_out, d->B, d->N, K, d->has_cls ? 1 : 0, keep, st), "select");
     if (x_hat != x_out)
-        RS_CHECK_LAUNCH(ctx, RS_K_GATHER, st, rs::launch_gather(d->out_dtype, x_hat, keep, d->B, d->N, K, D, x_out, st), "gather");
+        RS_CHECK_LAUNCH(ctx, RS_K_GATHER, st, rs::launch_gather(d->out_dtype, x_hat, keep, d->B, d->N, K, D, x_out, ln, st), "gather");
     return RS_OK;
+}
+
+rs_status rs_block_fwd(rs_ctx* ctx, const rs_block_desc* d, const rs_block_weights* w, const void* x,
+                       void* x_out, float* scores, int32_t* keep_idx, void* x_full, void* workspace,
+                       size_t workspace_bytes, void* stream) {
+    return block_fwd_impl(ctx, d, w, x, nullptr, x_out, scores, keep_idx, x_full, workspace, workspace_bytes, stream,
+                          nullptr, nullptr);
 }
 
 }  // extern "C"
@@ -392,7 +412,7 @@ bool vit_plan(const rs_vit_desc& d, const int* drops, VitPlan* p) {
     }
     p->block_ws = rs::align_up(block_ws, 256);
     p->act_bytes = rs::align_up((size_t)d.B * d.N * d.D * rs::dtype_size(d.dtype), 256);
-    p->total = p->block_ws + 2 * p->act_bytes;
+    p->total = p->block_ws + 3 * p->act_bytes;   // block scratch, two token buffers, one LN buffer
     p->n_final = n;
     return true;
 }
@@ -407,11 +427,12 @@ size_t rs_vit_workspace_bytes(const rs_vit_desc* d, const int* drops) {
     return p.total;
 }
 
-rs_status rs_vit_fwd(rs_ctx* ctx, const rs_vit_desc* d, const rs_block_weights* weights, const int* drops,
-                     const void* x, void* x_out, float* scores_last, int32_t* keep_last, void* workspace,
-                     size_t workspace_bytes, void* stream) {
+rs_status rs_vit_fwd_taps(rs_ctx* ctx, const rs_vit_desc* d, const rs_block_weights* weights, const int* drops,
+                          const void* x, const rs_vit_taps* taps, void* workspace, size_t workspace_bytes,
+                          void* stream) {
     if (!ctx) return RS_ERR_INVALID_ARG;
-    if (!d || !weights || !drops || !x || !x_out) return fail(ctx, RS_ERR_INVALID_ARG, "rs_vit_fwd: null argument");
+    if (!d || !weights || !drops || !x || !taps || d->L < 1 || !taps->x_out || !taps->x_out[d->L - 1])
+        return fail(ctx, RS_ERR_INVALID_ARG, "rs_vit_fwd: null argument (the last block's x_out is required)");
     VitPlan p;
     if (!valid_dtype(d->dtype) || !vit_plan(*d, drops, &p))
         return fail(ctx, RS_ERR_INVALID_ARG, "rs_vit_fwd: bad descriptor or schedule (need 0 <= drops[l] <= N_l - 1)");
@@ -421,20 +442,41 @@ rs_status rs_vit_fwd(rs_ctx* ctx, const rs_vit_desc* d, const rs_block_weights* 
         return fail(ctx, RS_ERR_INVALID_ARG, "rs_vit_fwd: workspace must be 256-byte aligned");
     char* base = (char*)workspace;
     void* act[2] = {base + p.block_ws, base + p.block_ws + p.act_bytes};
+    void* ln_buf = base + p.block_ws + 2 * p.act_bytes;   // LN1 of the next block's input, from the compaction
+    const float eps = d->ln_eps > 0.f ? d->ln_eps : 1e-6f;
     const void* cur = x;
+    const void* cur_ln = nullptr;
     int n = d->N;
     for (int l = 0; l < d->L; ++l) {
         const bool last = l == d->L - 1;
         rs_block_desc bd = {d->dtype, d->dtype, d->B, n, d->D, d->H, d->D_mlp, drops[l], d->has_cls, d->ln_eps, d->scale,
                             d->score_mode, d->dist};
-        void* out = last ? x_out : act[l & 1];
-        rs_status st = rs_block_fwd(ctx, &bd, &weights[l], cur, out, last ? scores_last : nullptr, last ? keep_last : nullptr,
-                                    nullptr, base, p.block_ws, stream);
+        void* out = taps->x_out[l] ? taps->x_out[l] : act[l & 1];
+        // LN1 of block l+1 rides in this block's compaction: one kernel less per block
+        const rs::LnFuse next = {last ? nullptr : weights[l + 1].ln1_g, last ? nullptr : weights[l + 1].ln1_b, eps, ln_buf};
+        bool ln_done = false;
+        rs_status st = block_fwd_impl(ctx, &bd, &weights[l], cur, cur_ln, out, taps->scores ? taps->scores[l] : nullptr,
+                                      taps->keep_idx ? taps->keep_idx[l] : nullptr, nullptr, base, p.block_ws, stream,
+                                      (last || !next.gamma || !next.beta) ? nullptr : &next, &ln_done);
         if (st != RS_OK) return st;
         cur = out;
+        cur_ln = ln_done ? ln_buf : nullptr;
         n -= drops[l];
     }
     return RS_OK;
+}
+
+rs_status rs_vit_fwd(rs_ctx* ctx, const rs_vit_desc* d, const rs_block_weights* weights, const int* drops,
+                     const void* x, void* x_out, float* scores_last, int32_t* keep_last, void* workspace,
+                     size_t workspace_bytes, void* stream) {
+    if (!ctx) return RS_ERR_INVALID_ARG;
+    if (!d || d->L < 1 || d->L > 4096 || !x_out) return fail(ctx, RS_ERR_INVALID_ARG, "rs_vit_fwd: null argument or bad L");
+    std::vector<void*> xo(d->L, nullptr);
+    std::vector<float*> sc(d->L, nullptr);
+    std::vector<int32_t*> ki(d->L, nullptr);
+    xo[d->L - 1] = x_out; sc[d->L - 1] = scores_last; ki[d->L - 1] = keep_last;
+    const rs_vit_taps taps = {xo.data(), sc.data(), ki.data()};
+    return rs_vit_fwd_taps(ctx, d, weights, drops, x, &taps, workspace, workspace_bytes, stream);
 }
 
 }  // extern "C"

@@ -10,44 +10,6 @@ namespace {
 
 constexpr int kWarpsPerCta = 8;
 
-template <typename TO, int N>
-__device__ __forceinline__ void store_n(TO* p, const float* v);
-template <> __device__ __forceinline__ void store_n<float, 4>(float* p, const float* v) {
-    *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]);
-}
-template <> __device__ __forceinline__ void store_n<float, 8>(float* p, const float* v) {
-    *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]);
-    *reinterpret_cast<float4*>(p + 4) = make_float4(v[4], v[5], v[6], v[7]);
-}
-template <> __device__ __forceinline__ void store_n<__nv_bfloat16, 4>(__nv_bfloat16* p, const float* v) {
-    __nv_bfloat162 a = __floats2bfloat162_rn(v[0], v[1]);
-    __nv_bfloat162 b = __floats2bfloat162_rn(v[2], v[3]);
-    *reinterpret_cast<uint2*>(p) = make_uint2(*reinterpret_cast<uint32_t*>(&a), *reinterpret_cast<uint32_t*>(&b));
-}
-template <> __device__ __forceinline__ void store_n<__nv_bfloat16, 8>(__nv_bfloat16* p, const float* v) {
-    uint32_t w[4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
-        w[i] = *reinterpret_cast<uint32_t*>(&h);
-    }
-    *reinterpret_cast<uint4*>(p) = make_uint4(w[0], w[1], w[2], w[3]);
-}
-
-// 16 bytes of T as floats.
-template <typename T> __device__ __forceinline__ void unpack16(const uint4& r, float (&v)[Vec16<T>::N]);
-template <> __device__ __forceinline__ void unpack16<float>(const uint4& r, float (&v)[4]) {
-    v[0] = __uint_as_float(r.x); v[1] = __uint_as_float(r.y); v[2] = __uint_as_float(r.z); v[3] = __uint_as_float(r.w);
-}
-template <> __device__ __forceinline__ void unpack16<__nv_bfloat16>(const uint4& r, float (&v)[8]) {
-    const uint32_t w[4] = {r.x, r.y, r.z, r.w};
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        v[2 * i] = __uint_as_float(w[i] << 16);
-        v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
-    }
-}
-
 // ---------------------------------------------------------------- LayerNorm
 // LN of Eq. att / Eq. MLP: mean and biased variance over D, then affine.  One warp per row; the
 // row stays in registers as packed 16-byte pieces (unpacked once per pass over it), which keeps
@@ -70,47 +32,7 @@ layernorm_kernel(const TI* __restrict__ x, const float* __restrict__ gamma,
         const int iv = j * 32 + lane;
         if (iv < nvec) raw[j] = ld_stream(xr + iv);
     }
-    float sum = 0.f;
-#pragma unroll
-    for (int j = 0; j < MAXV; ++j) {
-        if (j * 32 + lane < nvec) {
-            float v[VN];
-            unpack16<TI>(raw[j], v);
-#pragma unroll
-            for (int e = 0; e < VN; ++e) sum += v[e];
-        }
-    }
-    const float mu = warp_sum(sum) / (float)D;
-    float sq = 0.f;
-#pragma unroll
-    for (int j = 0; j < MAXV; ++j) {
-        if (j * 32 + lane < nvec) {
-            float v[VN];
-            unpack16<TI>(raw[j], v);
-#pragma unroll
-            for (int e = 0; e < VN; ++e) { const float dd = v[e] - mu; sq += dd * dd; }
-        }
-    }
-    const float rstd = rsqrtf(warp_sum(sq) / (float)D + eps);
-    TO* orow = out + row * D;
-#pragma unroll
-    for (int j = 0; j < MAXV; ++j) {
-        const int iv = j * 32 + lane;
-        if (iv < nvec) {
-            float v[VN], y[VN];
-            unpack16<TI>(raw[j], v);
-#pragma unroll
-            for (int e = 0; e < VN; e += 4) {
-                const float4 g = __ldg(reinterpret_cast<const float4*>(gamma + iv * VN + e));
-                const float4 bt = __ldg(reinterpret_cast<const float4*>(beta + iv * VN + e));
-                y[e + 0] = (v[e + 0] - mu) * rstd * g.x + bt.x;
-                y[e + 1] = (v[e + 1] - mu) * rstd * g.y + bt.y;
-                y[e + 2] = (v[e + 2] - mu) * rstd * g.z + bt.z;
-                y[e + 3] = (v[e + 3] - mu) * rstd * g.w + bt.w;
-            }
-            store_n<TO, VN>(orow + iv * VN, y);
-        }
-    }
+    layernorm_row<TI, TO, MAXV>(raw, nvec, lane, gamma, beta, eps, D, out + row * D);
 }
 
 // ---------------------------------------------------------------- shift score

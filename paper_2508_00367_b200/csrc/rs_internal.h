@@ -72,13 +72,17 @@ cudaError_t launch_residual_score(const float* m, const float* x_prime, const vo
 // from which the score is finished here (and written to scores_out when non-null).
 cudaError_t launch_select(const float* scores, int nparts, float* scores_out, int B, int N, int K,
                           int has_cls, int32_t* keep_idx, cudaStream_t st);
+// The compaction kernels can also write LN(x_out) for the block that follows (its LN1 of Eq. att):
+// the warp that copies a kept row has it in registers.  out: [B, K, D] of the rows' dtype.
+struct LnFuse { const float* gamma; const float* beta; float eps; void* out; };
+bool ln_fusable(rs_dtype dtype, int D);   // the row fits the registers of one warp
 cudaError_t launch_gather(rs_dtype dtype, const void* x, const int32_t* keep_idx, int B, int N, int K,
-                          int D, void* x_out, cudaStream_t st);
+                          int D, void* x_out, const LnFuse* ln /*null: none*/, cudaStream_t st);
 // Selection and compaction in one kernel (N <= 1024 and something is dropped).
 bool select_gather_fusable(int N, int K);
 cudaError_t launch_select_gather(const float* scores, int nparts, float* scores_out, int B, int N, int K, int has_cls,
-                                 int32_t* keep_idx, rs_dtype dtype, const void* x, int D, void* x_out, int sm_count,
-                                 cudaStream_t st);
+                                 int32_t* keep_idx, rs_dtype dtype, const void* x, int D, void* x_out,
+                                 const LnFuse* ln /*null: none*/, int sm_count, cudaStream_t st);
 size_t select_smem_bytes(int N);
 cudaError_t select_init();   // opt in to large dynamic shared memory once per process/device
 

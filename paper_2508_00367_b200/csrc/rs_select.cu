@@ -10,6 +10,7 @@
 // no sort.  Integer work only once the keys are formed, hence bit-exact.
 #include "rs_internal.h"
 #include "rs_device.cuh"
+#include <type_traits>
 
 namespace rs {
 
@@ -221,15 +222,54 @@ select_small_kernel(const float* __restrict__ scores, int nparts, float* __restr
     if (keep && pos < K) keep_idx[(long long)b * K + pos] = i;
 }
 
+// One warp copies one kept row (16-byte pieces, all loads of a pass issued before its first store)
+// to row `orow` of x_out and, with LT given, writes LN of the row to the same row of ln.out.
+template <int MAXV, typename LT>
+__device__ __forceinline__ void copy_row(const uint4* __restrict__ src, long long orow, int row_vecs, int lane,
+                                         uint4* __restrict__ x_out, const LnFuse& ln) {
+    uint4* dst = x_out + orow * row_vecs;
+    if constexpr (std::is_void<LT>::value) {
+        for (int base = 0; base < row_vecs; base += 32 * MAXV) {
+            uint4 v[MAXV];
+#pragma unroll
+            for (int j = 0; j < MAXV; ++j) {
+                const int iv = base + j * 32 + lane;
+                if (iv < row_vecs) v[j] = __ldg(src + iv);
+            }
+#pragma unroll
+            for (int j = 0; j < MAXV; ++j) {
+                const int iv = base + j * 32 + lane;
+                if (iv < row_vecs) dst[iv] = v[j];
+            }
+        }
+    } else {
+        uint4 v[MAXV];
+#pragma unroll
+        for (int j = 0; j < MAXV; ++j) {
+            const int iv = j * 32 + lane;
+            if (iv < row_vecs) v[j] = __ldg(src + iv);
+        }
+#pragma unroll
+        for (int j = 0; j < MAXV; ++j) {
+            const int iv = j * 32 + lane;
+            if (iv < row_vecs) dst[iv] = v[j];
+        }
+        const int D = row_vecs * Vec16<LT>::N;
+        layernorm_row<LT, LT, MAXV>(v, row_vecs, lane, ln.gamma, ln.beta, ln.eps, D, reinterpret_cast<LT*>(ln.out) + orow * D);
+    }
+}
+
 // Selection and compaction in one launch for N <= 1024.  Grid (G, B): every CTA of sample b
 // repeats the (cheap) counting selection of select_small_kernel, so no CTA waits for another;
 // CTA 0 of the sample writes the index list (and the finished scores), and each CTA copies its
 // share of the kept rows, a warp per row, all 16-byte loads of a row before its stores.
-template <int MAXV>
+// LT: void, or the rows' element type when LN of every written row goes to ln.out as well (the
+// whole row then sits in one warp's registers: row_vecs <= 32 * MAXV).
+template <int MAXV, typename LT>
 __global__ void __launch_bounds__(1024)
 select_gather_small_kernel(const float* __restrict__ scores, int nparts, float* __restrict__ scores_out, int N,
                            int K, int has_cls, int32_t* __restrict__ keep_idx, const uint4* __restrict__ x,
-                           int row_vecs, uint4* __restrict__ x_out) {
+                           int row_vecs, uint4* __restrict__ x_out, const LnFuse ln) {
     __shared__ uint32_t keys[1024];
     __shared__ int32_t kept[1024];
     __shared__ int wsum[32];
@@ -282,23 +322,8 @@ select_gather_small_kernel(const float* __restrict__ scores, int nparts, float* 
     const int G = gridDim.x, per = (K + G - 1) / G;
     const int lo = blockIdx.x * per, hi = min(lo + per, K);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
-    for (int r = lo + warp; r < hi; r += nwarps) {
-        const uint4* src = x + ((long long)b * N + kept[r]) * row_vecs;
-        uint4* dst = x_out + ((long long)b * K + r) * row_vecs;
-        for (int base = 0; base < row_vecs; base += 32 * MAXV) {
-            uint4 v[MAXV];
-#pragma unroll
-            for (int j = 0; j < MAXV; ++j) {
-                const int iv = base + j * 32 + lane;
-                if (iv < row_vecs) v[j] = __ldg(src + iv);
-            }
-#pragma unroll
-            for (int j = 0; j < MAXV; ++j) {
-                const int iv = base + j * 32 + lane;
-                if (iv < row_vecs) dst[iv] = v[j];
-            }
-        }
-    }
+    for (int r = lo + warp; r < hi; r += nwarps)
+        copy_row<MAXV, LT>(x + ((long long)b * N + kept[r]) * row_vecs, (long long)b * K + r, row_vecs, lane, x_out, ln);
 }
 
 // Nothing dropped (K == N): every token is kept, in order; only the scores remain to be
@@ -316,10 +341,10 @@ keep_all_kernel(const float* __restrict__ scores, int nparts, float* __restrict_
 
 // x_out[b, j, :] = x[b, keep_idx[b, j], :]; one warp per kept row, 16-byte vectors,
 // all loads of a row issued before the first store.
-template <int MAXV>
+template <int MAXV, typename LT>
 __global__ void __launch_bounds__(256)
 gather_kernel(const uint4* __restrict__ x, const int32_t* __restrict__ keep_idx, long long rows, int N,
-              int K, int row_vecs, uint4* __restrict__ x_out) {
+              int K, int row_vecs, uint4* __restrict__ x_out, const LnFuse ln) {
     grid_dep_launch();
     grid_dep_wait();
     const int lane = threadIdx.x & 31;
@@ -327,21 +352,7 @@ gather_kernel(const uint4* __restrict__ x, const int32_t* __restrict__ keep_idx,
     if (row >= rows) return;
     const long long b = row / K;
     const int src = keep_idx[row];
-    const uint4* s = x + (b * N + src) * row_vecs;
-    uint4* d = x_out + row * row_vecs;
-    for (int base = 0; base < row_vecs; base += 32 * MAXV) {
-        uint4 v[MAXV];
-#pragma unroll
-        for (int j = 0; j < MAXV; ++j) {
-            const int iv = base + j * 32 + lane;
-            if (iv < row_vecs) v[j] = __ldg(s + iv);
-        }
-#pragma unroll
-        for (int j = 0; j < MAXV; ++j) {
-            const int iv = base + j * 32 + lane;
-            if (iv < row_vecs) d[iv] = v[j];
-        }
-    }
+    copy_row<MAXV, LT>(x + (b * N + src) * row_vecs, row, row_vecs, lane, x_out, ln);
 }
 
 }  // namespace
@@ -368,28 +379,44 @@ cudaError_t launch_select(const float* scores, int nparts, float* scores_out, in
 
 bool select_gather_fusable(int N, int K) { return N <= 1024 && K < N; }
 
+bool ln_fusable(rs_dtype dtype, int D) { return (size_t)D * dtype_size(dtype) / 16 <= 32 * 4; }
+
 cudaError_t launch_select_gather(const float* scores, int nparts, float* scores_out, int B, int N, int K, int has_cls,
-                                 int32_t* keep_idx, rs_dtype dtype, const void* x, int D, void* x_out, int sm_count,
-                                 cudaStream_t st) {
+                                 int32_t* keep_idx, rs_dtype dtype, const void* x, int D, void* x_out,
+                                 const LnFuse* ln, int sm_count, cudaStream_t st) {
     if (B == 0) return cudaSuccess;
     const int row_vecs = (int)((size_t)D * dtype_size(dtype) / 16);
-    // enough CTAs per sample for about three waves over the SMs, at least a few rows each
-    int G = (3 * sm_count + B - 1) / B;
+    // enough CTAs per sample for about three waves over the SMs (six when a row is also normalised:
+    // measured), at least a few rows each
+    int G = ((ln ? 6 : 3) * sm_count + B - 1) / B;
     G = G < 1 ? 1 : G;
     if (G > (K + 3) / 4) G = (K + 3) / 4;
     if (G < 1) G = 1;
-    return launch_pdl(select_gather_small_kernel<4>, dim3(G, B), dim3((N + 31) / 32 * 32 < 128 ? 128 : (N + 31) / 32 * 32), 0, st,
-                      scores, nparts, scores_out, N, K, has_cls, keep_idx, (const uint4*)x, row_vecs, (uint4*)x_out);
+    const dim3 grid(G, B), block((N + 31) / 32 * 32 < 128 ? 128 : (N + 31) / 32 * 32);
+    if (ln && !ln_fusable(dtype, D)) return cudaErrorInvalidValue;
+    const LnFuse none = {nullptr, nullptr, 0.f, nullptr};
+#define RS_SG_CASE(LT)                                                                                                  \
+    launch_pdl(select_gather_small_kernel<4, LT>, grid, block, 0, st, scores, nparts, scores_out, N, K, has_cls, keep_idx, \
+               (const uint4*)x, row_vecs, (uint4*)x_out, ln ? *ln : none)
+    if (!ln) return RS_SG_CASE(void);
+    return dtype == RS_BF16 ? RS_SG_CASE(__nv_bfloat16) : RS_SG_CASE(float);
+#undef RS_SG_CASE
 }
 
 cudaError_t launch_gather(rs_dtype dtype, const void* x, const int32_t* keep_idx, int B, int N, int K,
-                          int D, void* x_out, cudaStream_t st) {
+                          int D, void* x_out, const LnFuse* ln, cudaStream_t st) {
     const long long rows = (long long)B * K;
     if (rows == 0) return cudaSuccess;
     const int row_vecs = (int)((size_t)D * dtype_size(dtype) / 16);
     const unsigned grid = (unsigned)((rows + 7) / 8);
-    return launch_pdl(gather_kernel<4>, dim3(grid), dim3(256), 0, st, (const uint4*)x, keep_idx, rows, N, K, row_vecs,
-                      (uint4*)x_out);
+    if (ln && !ln_fusable(dtype, D)) return cudaErrorInvalidValue;
+    const LnFuse none = {nullptr, nullptr, 0.f, nullptr};
+#define RS_G_CASE(LT)                                                                                               \
+    launch_pdl(gather_kernel<4, LT>, dim3(grid), dim3(256), 0, st, (const uint4*)x, keep_idx, rows, N, K, row_vecs, \
+               (uint4*)x_out, ln ? *ln : none)
+    if (!ln) return RS_G_CASE(void);
+    return dtype == RS_BF16 ? RS_G_CASE(__nv_bfloat16) : RS_G_CASE(float);
+#undef RS_G_CASE
 }
 
 }  // namespace rs

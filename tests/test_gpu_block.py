@@ -250,25 +250,44 @@ def test_graph_replay_equals_eager(ctx):
             assert torch.equal(a["keep_idx"], b["keep_idx"])
             assert torch.equal(a["x_out"].view(torch.int16), b["x_out"].view(torch.int16))
             assert torch.equal(a["scores"], b["scores"])
-    assert model.launches_per_forward(B, N, D) == 8 * L          # selection and gather are one kernel here; the block that drops nothing has neither
+    # eight kernels per block (selection and gather are one here); the block after a pruning block
+    # gets its LN1 from that block's compaction kernel and launches none: blocks 0 and 2 -> 8, block 1 -> 7
+    assert model.launches_per_forward(B, N, D) == 8 * L - 1
     ctx.async_status()
 
 
-def test_vit_fwd_equals_the_block_loop(ctx):
-    """rs_vit_fwd is the layer loop inside the library: same kernels, bit-identical to chaining rs_block_fwd."""
+@pytest.mark.parametrize("B,N,D,H,drops,dt", [
+    (2, 197, 384, 6, [16, 0, 20, 5], "bf16"),
+    (1, 1100, 128, 2, [76, 0, 30], "bf16"),        # N > 1024: radix selection and the stand-alone gather kernel
+    (2, 50, 128, 2, [5, 5, 0], "f32"),             # fp32 storage (SIMT kernels)
+])
+def test_vit_fwd_equals_the_block_loop(ctx, B, N, D, H, drops, dt):
+    """rs_vit_fwd / rs_vit_fwd_taps are the layer loop inside the library.  They fold LN1 of the block
+    after a pruning block into the compaction kernel (same row arithmetic), so every block's outputs
+    are bit-identical to chaining rs_block_fwd."""
     import paper_2508_00367_b200 as rs
     from paper_2508_00367_b200 import synth
-    B, N, D, H = 2, 197, 384, 6
-    drops = [16, 0, 20, 5]
-    x = synth.make_tokens(B, N, D, "bf16", seed=61).to(torch.bfloat16).cuda()
-    blocks = [synth.make_block_weights(D, 4 * D, "bf16", seed=70 + l) for l in range(len(drops))]
-    model = rs.PrunedViT(ctx, blocks, H, drops, torch.bfloat16)
-    want = model.forward(x)[-1]
+    tdt = torch.bfloat16 if dt == "bf16" else torch.float32
+    x = synth.make_tokens(B, N, D, dt, seed=61).to(tdt).cuda()
+    blocks = [synth.make_block_weights(D, 4 * D, dt, seed=70 + l) for l in range(len(drops))]
+    model = rs.PrunedViT(ctx, blocks, H, drops, tdt)
+    chain, cur = [], x
+    for l, r in enumerate(drops):
+        o = ctx.block_fwd(cur, model.weights[l], H, r)
+        chain.append(o)
+        cur = o["x_out"]
+    taps = model.forward(x)                                      # rs_vit_fwd_taps: every block's outputs
+    torch.cuda.synchronize()
+    for want, got_l in zip(chain, taps):
+        assert torch.equal(got_l["keep_idx"], want["keep_idx"])
+        assert torch.equal(got_l["scores"], want["scores"])
+        assert torch.equal(got_l["x_out"], want["x_out"])
+    want = chain[-1]
     got = ctx.vit_fwd(x, model.weights, H, drops)
     torch.cuda.synchronize()
     assert torch.equal(got["keep_idx"], want["keep_idx"])
     assert torch.equal(got["scores"], want["scores"])
-    assert torch.equal(got["x_out"].view(torch.int16), want["x_out"].view(torch.int16))
+    assert torch.equal(got["x_out"], want["x_out"])
     with pytest.raises(rs.RsError):
-        ctx.vit_fwd(x, model.weights, H, [16, 0, 20, 161])      # the last block cannot drop all its tokens
+        ctx.vit_fwd(x, model.weights, H, drops[:-1] + [N])       # the last block cannot drop all its tokens
     ctx.async_status()
