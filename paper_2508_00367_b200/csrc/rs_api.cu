@@ -289,6 +289,7 @@ static rs_status block_fwd_impl(rs_ctx* ctx, const rs_block_desc* d, const rs_bl
     if (d->D > 1024 && d->dtype == RS_F32) return fail(ctx, RS_ERR_UNSUPPORTED, "rs_block_fwd: D > 1024 in fp32");
     if (d->N > 32768) return fail(ctx, RS_ERR_UNSUPPORTED, "rs_block_fwd: N > 32768");
     if (d->r < 0 || d->r > d->N - 1) return fail(ctx, RS_ERR_INVALID_ARG, "rs_block_fwd: need 0 <= r <= N-1");
+    if (!(d->scale >= 0.f)) return fail(ctx, RS_ERR_INVALID_ARG, "rs_block_fwd: scale must be >= 0");
     if (d->dist < RS_DIST_L2 || d->dist > RS_DIST_COS) return fail(ctx, RS_ERR_INVALID_ARG, "rs_block_fwd: bad dist");
     if (d->score_mode < RS_SCORE_MLP || d->score_mode > RS_SCORE_BLOCK)
         return fail(ctx, RS_ERR_INVALID_ARG, "rs_block_fwd: bad score_mode");

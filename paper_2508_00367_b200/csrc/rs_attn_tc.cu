@@ -116,8 +116,10 @@ __device__ __forceinline__ uint64_t fadd2(uint64_t a, uint64_t b) {
     return r;
 }
 
-// Maximum of the first NC values of a row of S held in registers (only the first `valid` count).
-template <int NC, bool MASKED>
+// Maximum of the first NC values of a row of S held in registers.  MASK 0: all NC are keys.
+// MASK 1: NC = the 32-column groups that hold keys, so only the last group can hold columns past
+// `valid` and only there the elements are tested.  MASK 2: every element is tested.
+template <int NC, int MASK>
 __device__ __forceinline__ float row_max(const uint32_t (&r)[128], int valid) {
     float m[8];
 #pragma unroll
@@ -127,7 +129,7 @@ __device__ __forceinline__ float row_max(const uint32_t (&r)[128], int valid) {
 #pragma unroll
         for (int c = 0; c < 8; ++c) {
             float a = __uint_as_float(r[i + 2 * c]), b = __uint_as_float(r[i + 2 * c + 1]);
-            if (MASKED) {
+            if (MASK == 2 || (MASK == 1 && i >= NC - 32)) {
                 if (i + 2 * c >= valid) a = -INFINITY;
                 if (i + 2 * c + 1 >= valid) b = -INFINITY;
             }
@@ -137,9 +139,9 @@ __device__ __forceinline__ float row_max(const uint32_t (&r)[128], int valid) {
     return max3(max3(m[0], m[1], m[2]), max3(m[3], m[4], m[5]), fmaxf(m[6], m[7]));
 }
 
-// p_i = exp2(s_i * sl + mneg) for the first `valid` of NC keys (0 for the rest), packed to bf16
-// pairs in place (r[0 .. NC/2) on return); returns the sum of the unrounded p_i.
-template <int NC, bool MASKED>
+// p_i = exp2(s_i * sl + mneg) for the first `valid` of NC keys (0 for the rest; MASK as above),
+// packed to bf16 pairs in place (r[0 .. NC/2) on return); returns the sum of the unrounded p_i.
+template <int NC, int MASK>
 __device__ __forceinline__ float exp_pass(uint32_t (&r)[128], float sl, float mneg, int valid) {
     const uint64_t sl2 = pack2(sl, sl), mneg2 = pack2(mneg, mneg);
     uint64_t l01 = pack2(0.f, 0.f), l23 = l01;
@@ -148,7 +150,7 @@ __device__ __forceinline__ float exp_pass(uint32_t (&r)[128], float sl, float mn
         float x0, x1, x2, x3;
         unpack2(ffma2(pack2(__uint_as_float(r[i]), __uint_as_float(r[i + 1])), sl2, mneg2), x0, x1);
         unpack2(ffma2(pack2(__uint_as_float(r[i + 2]), __uint_as_float(r[i + 3])), sl2, mneg2), x2, x3);
-        if (MASKED) {
+        if (MASK == 2 || (MASK == 1 && i >= NC - 32)) {
             if (i >= valid) x0 = -INFINITY;
             if (i + 1 >= valid) x1 = -INFINITY;
             if (i + 2 >= valid) x2 = -INFINITY;
@@ -166,6 +168,10 @@ __device__ __forceinline__ float exp_pass(uint32_t (&r)[128], float sl, float mn
     return (a + b) + (c + d);
 }
 
+// FINE: partial key tiles are handled by 32-column groups (worth it when a sequence is a few
+// tiles long).  Without it the one partial tile of a long sequence is a full tile with every
+// element tested, and the kernel carries less code around its inner loop, which that loop feels.
+template <bool FINE>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                const __grid_constant__ CUtensorMap tmV, const AttnArgs args) {
@@ -361,24 +367,24 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 if (!__all_sync(0xffffffffu, mbar_wait(&s_full[g], cnt & 1u, abort_flag))) { ok = false; break; }
                 tc_fence_after();
                 // Whole 32-column groups are read even on a partial key tile: columns past the keys
-                // the MMA wrote hold old values, which the masks below never let through.
+                // the MMA wrote hold old values, which the masks of the last group never let through.
                 uint32_t r[128];
-                const int ncol = valid > 64 ? 128 : valid > 32 ? 64 : 32;   // columns worth touching
+                // columns worth touching: whole 32-column groups, or (lean code) half a tile or all of it
+                const int ncol = FINE ? (valid + 31) & ~31 : valid <= 64 ? 64 : BKV;
                 tmem_ld_32x32(s_addr, r);
                 if (ncol > 32) tmem_ld_32x32(s_addr + 32, r + 32);
-                if (ncol > 64) {
-                    tmem_ld_32x32(s_addr + 64, r + 64);
-                    tmem_ld_32x32(s_addr + 96, r + 96);
-                }
+                if (ncol > 64) tmem_ld_32x32(s_addr + 64, r + 64);
+                if (ncol > 96) tmem_ld_32x32(s_addr + 96, r + 96);
                 tmem_wait_ld();
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&s_free[g]);  // the next Q K^T may overwrite S now
                 // running maximum: raised only when the tile tops it by more than 2^kRescaleGap
-                const float mx = valid == BKV ? row_max<128, false>(r, valid)
-                                 : ncol == 128 ? row_max<128, true>(r, valid)
-                                 : ncol == 64  ? row_max<64, true>(r, valid)
-                                               : row_max<32, true>(r, valid);
+                float mx;
+                if (valid == BKV) mx = row_max<128, 0>(r, valid);
+                else if (!FINE) mx = ncol == 64 ? row_max<64, 2>(r, valid) : row_max<128, 2>(r, valid);
+                else mx = ncol == 128 ? row_max<128, 1>(r, valid) : ncol == 96 ? row_max<96, 1>(r, valid)
+                          : ncol == 64 ? row_max<64, 1>(r, valid) : row_max<32, 1>(r, valid);
                 const float mx_l2 = mx * sl;
                 if (j == 0) {
                     m_l2 = mx_l2;
@@ -407,10 +413,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 // tile B's P V of item n, and tile B reaches its next wait about a pass sooner than tile A
                 // can arrive again; were that ever inverted, the wait is bounded and reports.)
                 if (j == 0 && g == 1 && !__all_sync(0xffffffffu, mbar_wait(first_pass, item_n & 1u, abort_flag))) { ok = false; break; }
-                l_run += valid == BKV ? exp_pass<128, false>(r, sl, -m_l2, valid)
-                         : ncol == 128 ? exp_pass<128, true>(r, sl, -m_l2, valid)
-                         : ncol == 64  ? exp_pass<64, true>(r, sl, -m_l2, valid)
-                                       : exp_pass<32, true>(r, sl, -m_l2, valid);
+                if (valid == BKV) l_run += exp_pass<128, 0>(r, sl, -m_l2, valid);
+                else if (!FINE) l_run += ncol == 64 ? exp_pass<64, 2>(r, sl, -m_l2, valid) : exp_pass<128, 2>(r, sl, -m_l2, valid);
+                else l_run += ncol == 128 ? exp_pass<128, 1>(r, sl, -m_l2, valid) : ncol == 96 ? exp_pass<96, 1>(r, sl, -m_l2, valid)
+                              : ncol == 64 ? exp_pass<64, 1>(r, sl, -m_l2, valid) : exp_pass<32, 1>(r, sl, -m_l2, valid);
                 if (j == 0 && g == 0 && lane == 0) mbar_arrive(first_pass);
                 if (cnt > 0) {
                     // P V of the previous key tile reads the P columns: it must have retired
@@ -419,10 +425,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 }
                 tmem_st_32x16(p_addr, r);
                 if (ncol > 32) tmem_st_32x16(p_addr + 16, r + 16);
-                if (ncol > 64) {
-                    tmem_st_32x16(p_addr + 32, r + 32);
-                    tmem_st_32x16(p_addr + 48, r + 48);
-                }
+                if (ncol > 64) tmem_st_32x16(p_addr + 32, r + 32);
+                if (ncol > 96) tmem_st_32x16(p_addr + 48, r + 48);
                 tmem_wait_st();
                 tc_fence_before();
                 __syncwarp();
@@ -502,7 +506,9 @@ cudaError_t launch_attn_tc(rs_ctx* ctx, const rs_attn_desc& d, const void* q, co
     if (!ctx->encode_tiled) return cudaErrorNotSupported;
     static bool attr_done = false;
     if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmem);
+        cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmem);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(attn_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmem);
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
@@ -527,7 +533,9 @@ cudaError_t launch_attn_tc(rs_ctx* ctx, const rs_attn_desc& d, const void* q, co
     // from the hardware handing the next item to whichever SM is free first.
     const int nkv = (d.N + BKV - 1) / BKV;
     const int grid = (nkv >= 16 || args.n_items < ctx->sm_count) ? args.n_items : ctx->sm_count;
-    return launch_pdl(attn_tc_kernel, dim3(grid), dim3(kThreads), kSmem, st, tmQ, tmK, tmV, args);
+    // a partial key tile is worth its own code when it is a good part of the sequence
+    if (nkv <= 12) return launch_pdl(attn_tc_kernel<true>, dim3(grid), dim3(kThreads), kSmem, st, tmQ, tmK, tmV, args);
+    return launch_pdl(attn_tc_kernel<false>, dim3(grid), dim3(kThreads), kSmem, st, tmQ, tmK, tmV, args);
 }
 
 }  // namespace rs
