@@ -291,43 +291,46 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 mma_commit(&o_done[g]);
                 ++np[g];
             };
-            // Issues the Q K^T of step j of an item (for every query tile it has); kv0 = ring position
-            // of the item's first K/V slot.
-            auto issue_s_step = [&](const Item& it, uint32_t qb, uint32_t kv0, int j) {
-#pragma unroll
-                for (int g = 0; g < 2; ++g) {
-                    if (g >= it.ng || !ok) break;
-                    const uint32_t t = kv0 + (args.dual ? g : j);
-                    if (!mbar_wait(&k_full[t % NS], (t / NS) & 1u, abort_flag)) { ok = false; return; }
-                    issue_s(g, qb, t % NS, min(BKV, N - j * BKV));
-                }
+            // Issues the Q K^T of step j of query tile g of an item; kv0 = ring position of the item's
+            // first K/V slot.
+            auto issue_s_one = [&](const Item& it, uint32_t qb, uint32_t kv0, int j, int g) {
+                const uint32_t t = kv0 + (args.dual ? g : j);
+                if (!mbar_wait(&k_full[t % NS], (t / NS) & 1u, abort_flag)) { ok = false; return; }
+                issue_s(g, qb, t % NS, min(BKV, N - j * BKV));
             };
 
             uint32_t item_n = 0, kv0 = 0;
             int w = blockIdx.x;
             Item cur = decode_item(args, w);
             ok = mbar_wait(&q_full[0], 0, abort_flag);
-            if (ok) issue_s_step(cur, 0, kv0, 0);
+#pragma unroll
+            for (int g = 0; g < 2; ++g)
+                if (ok && g < cur.ng) issue_s_one(cur, 0, kv0, 0, g);
             while (ok) {
                 const uint32_t qb = item_n & 1u;
+                const int wn = w + gridDim.x;
+                Item nxt = cur;
                 for (int j = 0; j < cur.nkv && ok; ++j) {
-                    // look ahead: the next Q K^T (of this item, or the first of the next item) goes to
-                    // the tensor pipe before this step's P V, which still waits for the exponentials
+                    // Look ahead, per query tile: the tile's next Q K^T (of this item, or the first of the
+                    // next item) goes to the tensor pipe before its P V of this step, which still waits
+                    // for the exponentials.  Tile by tile, not step by step: tile A's last P V of an item
+                    // then does not queue behind a Q K^T that waits for tile B, which runs half a pass later.
                     const bool last = j + 1 == cur.nkv;
-                    const int wn = w + gridDim.x;
-                    if (!last) {
-                        issue_s_step(cur, qb, kv0, j + 1);
-                    } else if (wn < args.n_items) {
-                        const Item nxt = decode_item(args, wn);
-                        const uint32_t nb = (item_n + 1) & 1u;
+                    const bool ahead = !last || wn < args.n_items;
+                    const uint32_t nb = last ? (item_n + 1) & 1u : qb;
+                    if (last && ahead) {
+                        nxt = decode_item(args, wn);
                         if (!mbar_wait(&q_full[nb], ((item_n + 1) >> 1) & 1u, abort_flag)) { ok = false; break; }
-                        issue_s_step(nxt, nb, kv0 + cur.slots, 0);
                     }
-                    if (!ok) break;
+                    const Item& sit = last ? nxt : cur;
+                    const uint32_t skv0 = last ? kv0 + cur.slots : kv0;
+                    const int sj = last ? 0 : j + 1;
                     const int valid = min(BKV, N - j * BKV);
 #pragma unroll
                     for (int g = 0; g < 2; ++g) {
-                        if (g >= cur.ng || !ok) break;
+                        if (!ok) break;
+                        if (ahead && g < sit.ng) issue_s_one(sit, nb, skv0, sj, g);
+                        if (!ok || g >= cur.ng) continue;
                         const uint32_t t = kv0 + (args.dual ? g : j);
                         if (!mbar_wait(&v_full[t % NS], (t / NS) & 1u, abort_flag)) { ok = false; break; }
                         issue_pv(g, t % NS, valid, j == 0);
@@ -338,9 +341,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 mma_commit(&q_empty[qb]);
                 kv0 += cur.slots;
                 ++item_n;
-                w += gridDim.x;
+                w = wn;
                 if (w >= args.n_items) break;
-                cur = decode_item(args, w);
+                cur = nxt;
             }
         }
     }
