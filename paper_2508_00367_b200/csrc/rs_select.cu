@@ -386,9 +386,9 @@ cudaError_t launch_select_gather(const float* scores, int nparts, float* scores_
                                  const LnFuse* ln, int sm_count, cudaStream_t st) {
     if (B == 0) return cudaSuccess;
     const int row_vecs = (int)((size_t)D * dtype_size(dtype) / 16);
-    // enough CTAs per sample for about three waves over the SMs (six when a row is also normalised:
-    // measured), at least a few rows each
-    int G = ((ln ? 6 : 3) * sm_count + B - 1) / B;
+    // enough CTAs per sample for about three waves over the SMs (six when a row is also normalised
+    // and the selection every CTA repeats is short: measured), at least a few rows each
+    int G = ((ln && N <= 256 ? 6 : 3) * sm_count + B - 1) / B;
     G = G < 1 ? 1 : G;
     if (G > (K + 3) / 4) G = (K + 3) / 4;
     if (G < 1) G = 1;
