@@ -209,6 +209,49 @@ void orc_gather(const double* x, const int32_t* keep_idx, int B, int N, int K, i
                    sizeof(double) * (size_t)D);
 }
 
+/* Line-wise pruning of a 2-D token grid (Sec. 4, "CNN and SSM", variant L-W): the shift is
+ * averaged over every row and over every column of the H x W grid, and the drop_rows rows and
+ * drop_cols columns with the lowest averages go, whole lines at a time.  Both averages are taken
+ * over the full grid (the text orders neither before the other); a line's rank among its peers
+ * follows the token rule (larger average first, lower index on a tie, NaN last).
+ * scores [B,H,W]; keep_rows [B,H-drop_rows], keep_cols [B,W-drop_cols], ascending.
+ * Returns 0, or -1 when a drop count is outside [0, lines-1]. */
+int orc_linewise(const double* scores, int B, int H, int W, int drop_rows, int drop_cols,
+                 int32_t* keep_rows, int32_t* keep_cols) {
+    if (drop_rows < 0 || drop_rows > H - 1 || drop_cols < 0 || drop_cols > W - 1) return -1;
+    double* rm = (double*)malloc(sizeof(double) * (size_t)B * H);
+    double* cm = (double*)malloc(sizeof(double) * (size_t)B * W);
+    for (int b = 0; b < B; ++b) {
+        const double* s = scores + (long)b * H * W;
+        for (int h = 0; h < H; ++h) {
+            double acc = 0.0;
+            for (int w = 0; w < W; ++w) acc += s[(long)h * W + w];
+            rm[(long)b * H + h] = acc / (double)W;
+        }
+        for (int w = 0; w < W; ++w) {
+            double acc = 0.0;
+            for (int h = 0; h < H; ++h) acc += s[(long)h * W + w];
+            cm[(long)b * W + w] = acc / (double)H;
+        }
+    }
+    int rc = orc_topk(rm, B, H, drop_rows, 0, keep_rows);
+    if (rc == 0) rc = orc_topk(cm, B, W, drop_cols, 0, keep_cols);
+    free(cm); free(rm);
+    return rc;
+}
+
+/* The grid that is left: x_out[b, i, j, :] = x[b, keep_rows[b, i], keep_cols[b, j], :].
+ * x [B,H,W,D] (channels last: a position is a token), x_out [B,Hk,Wk,D]. */
+void orc_grid_gather(const double* x, const int32_t* keep_rows, const int32_t* keep_cols, int B, int H, int W,
+                     int Hk, int Wk, int D, double* x_out) {
+    for (int b = 0; b < B; ++b)
+        for (int i = 0; i < Hk; ++i)
+            for (int j = 0; j < Wk; ++j)
+                memcpy(x_out + (((long)b * Hk + i) * Wk + j) * D,
+                       x + (((long)b * H + keep_rows[(long)b * Hk + i]) * W + keep_cols[(long)b * Wk + j]) * D,
+                       sizeof(double) * (size_t)D);
+}
+
 /* One block followed by pruning.
  *   x' = SA(LN(x)) + x            (Eq. att;  SA includes the output projection)
  *   m  = MLP(LN(x'))              (Eq. MLP without the residual)

@@ -42,6 +42,7 @@ def _load():
         _lib.orc_num_threads.restype = ctypes.c_int
         _lib.orc_topk.restype = ctypes.c_int
         _lib.orc_block_fwd.restype = ctypes.c_int
+        _lib.orc_linewise.restype = ctypes.c_int
     return _lib
 
 
@@ -172,6 +173,34 @@ def gather(x, keep_idx):
     out = np.empty((B, K, D), dtype=np.float64)
     _load().orc_gather(xp, keep.ctypes.data_as(_ip), ctypes.c_int(B), ctypes.c_int(N),
                        ctypes.c_int(K), ctypes.c_int(D), out.ctypes.data_as(_dp))
+    return out
+
+
+def linewise(scores, drop_rows, drop_cols):
+    """Sec. 4 (CNN, line-wise variant): scores [B, H, W] -> (keep_rows [B, H - drop_rows],
+    keep_cols [B, W - drop_cols]), the lines whose average shift is not among the lowest."""
+    s, sp = _d(scores)
+    B, H, W = s.shape
+    kr = np.empty((B, max(H - drop_rows, 0)), dtype=np.int32)
+    kc = np.empty((B, max(W - drop_cols, 0)), dtype=np.int32)
+    rc = _load().orc_linewise(sp, ctypes.c_int(B), ctypes.c_int(H), ctypes.c_int(W), ctypes.c_int(drop_rows),
+                              ctypes.c_int(drop_cols), kr.ctypes.data_as(_ip), kc.ctypes.data_as(_ip))
+    if rc != 0:
+        raise ValueError("drop counts must leave at least one row and one column")
+    return kr, kc
+
+
+def grid_gather(x, keep_rows, keep_cols):
+    """x [B, H, W, D] -> [B, Hk, Wk, D]: the rows and columns that are kept."""
+    x, xp = _d(x)
+    B, H, W, D = x.shape
+    kr = np.ascontiguousarray(keep_rows, dtype=np.int32)
+    kc = np.ascontiguousarray(keep_cols, dtype=np.int32)
+    Hk, Wk = kr.shape[1], kc.shape[1]
+    out = np.empty((B, Hk, Wk, D), dtype=np.float64)
+    _load().orc_grid_gather(xp, kr.ctypes.data_as(_ip), kc.ctypes.data_as(_ip), ctypes.c_int(B), ctypes.c_int(H),
+                            ctypes.c_int(W), ctypes.c_int(Hk), ctypes.c_int(Wk), ctypes.c_int(D),
+                            out.ctypes.data_as(_dp))
     return out
 
 

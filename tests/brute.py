@@ -71,3 +71,21 @@ def select(scores, r, has_cls):
                 w = i
         alive.remove(w)
     return np.array(sorted(alive), dtype=np.int32)
+
+
+def linewise(scores, drop_rows, drop_cols):
+    """Line-wise pruning of one H x W grid of scores, from the definition: the average of every
+    row and of every column (exact rational arithmetic, so no summation order enters), then the
+    lines with the lowest averages go, by the same ranking as tokens (no pinned line)."""
+    from fractions import Fraction
+    H, W = len(scores), len(scores[0])
+
+    def avg(vals):
+        if any(math.isnan(v) or math.isinf(v) for v in vals):
+            return float(sum(vals)) / len(vals)
+        return float(sum(Fraction(v) for v in vals) / len(vals))
+
+    rows = [avg([scores[h][w] for w in range(W)]) for h in range(H)]
+    cols = [avg([scores[h][w] for h in range(H)]) for w in range(W)]
+    return select(rows, drop_rows, False), select(cols, drop_cols, False)
+

@@ -342,3 +342,67 @@ def test_fixed_schedule_counts():
     assert Ns[0] == 1569 and Ns[3] == 1099 and Ns[6] == 770 and Ns[9] == 539
     Ns, rs = osched.drops_ratio(4097, 24, 0.25, (4, 8, 12, 16))
     assert [Ns[i] for i in (0, 4, 8, 12, 16)] == [4097, 3073, 2305, 1729, 1297]
+
+
+# ----------------------------------------------------------------- line-wise pruning of a 2-D grid (Sec. 4, CNN)
+
+def test_linewise_vs_brute_force_with_ties():
+    for trial in range(60):
+        H, W = int(RNG.integers(1, 8)), int(RNG.integers(1, 8))
+        dr, dc = int(RNG.integers(0, H)), int(RNG.integers(0, W))
+        s = RNG.integers(0, 3, size=(2, H, W)).astype(np.float64)      # few values: many equal averages
+        kr, kc = orc.linewise(s, dr, dc)
+        assert kr.shape == (2, H - dr) and kc.shape == (2, W - dc)
+        for b in range(2):
+            wr, wc = brute.linewise([list(r) for r in s[b]], dr, dc)
+            np.testing.assert_array_equal(kr[b], wr)
+            np.testing.assert_array_equal(kc[b], wc)
+
+
+def test_linewise_closed_forms():
+    # separable map s[h, w] = a[h] + c[w]: a row's average is a[h] + mean(c), so rows rank by a and
+    # columns by c, whatever the other factor is
+    a = np.array([5.0, 1.0, 4.0, 2.0, 3.0, 0.5])
+    c = np.array([0.25, 9.0, 3.0, 7.0])
+    s = (a[:, None] + c[None, :])[None]
+    kr, kc = orc.linewise(s, 2, 1)
+    np.testing.assert_array_equal(kr[0], [0, 2, 3, 4])     # a = 1.0 and 0.5 go
+    np.testing.assert_array_equal(kc[0], [1, 2, 3])        # c = 0.25 goes
+    # both averages come from the full grid.  Here the row that goes (average -1) holds the weight of
+    # column 1: on the full grid column 0 averages -4/3 and goes; had the row been removed first,
+    # column 0 would average 3 against 0 and column 1 would go instead.
+    s2 = np.array([[[3.0, 0.0], [3.0, 0.0], [-10.0, 8.0]]])
+    kr, kc = orc.linewise(s2, 1, 1)
+    np.testing.assert_array_equal(kr[0], [0, 1])
+    np.testing.assert_array_equal(kc[0], [1])
+    # equal averages: the later line goes
+    s3 = np.array([[[0.0, 9.0], [0.0, 9.0], [50.0, 0.0]]])
+    np.testing.assert_array_equal(orc.linewise(s3, 1, 0)[0][0], [0, 2])
+    # one column: the grid is a token list without a class token
+    t = RNG.normal(size=(3, 11))
+    np.testing.assert_array_equal(orc.linewise(t[:, :, None], 4, 0)[0], orc.topk(t, 4, False))
+    np.testing.assert_array_equal(orc.linewise(t[:, None, :], 0, 4)[1], orc.topk(t, 4, False))
+    # transposing the grid swaps the two answers
+    g = RNG.normal(size=(2, 6, 9))
+    kr, kc = orc.linewise(g, 2, 3)
+    kr_t, kc_t = orc.linewise(np.ascontiguousarray(g.transpose(0, 2, 1)), 3, 2)
+    np.testing.assert_array_equal(kr, kc_t)
+    np.testing.assert_array_equal(kc, kr_t)
+    # nothing dropped: identity; dropping everything is refused
+    kr, kc = orc.linewise(g, 0, 0)
+    np.testing.assert_array_equal(kr[0], np.arange(6))
+    np.testing.assert_array_equal(kc[1], np.arange(9))
+    with pytest.raises(ValueError):
+        orc.linewise(g, 6, 0)
+    with pytest.raises(ValueError):
+        orc.linewise(g, 0, 9)
+
+
+def test_grid_gather_is_fancy_indexing():
+    x = RNG.normal(size=(2, 5, 7, 3))
+    kr = np.array([[0, 2, 4], [1, 2, 3]], dtype=np.int32)
+    kc = np.array([[6, 5], [0, 3]], dtype=np.int32)           # any order is taken as given
+    got = orc.grid_gather(x, kr, kc)
+    for b in range(2):
+        np.testing.assert_array_equal(got[b], x[b][kr[b]][:, kc[b]])
+
