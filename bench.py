@@ -219,6 +219,24 @@ def isolated_parts(ctx, wl, peaks, dev):
     byt = 4 * Bs * N + 4 * Bs * K + 2 * Bs * K * D * 2
     out["select_compact"] = dict(B=Bs, N=N, D=D, r=r, mbytes=byt / 1e6, us=sec * 1e6, gbs=byt / sec / 1e9,
                                  frac_of_hbm_peak=byt / sec / 1e9 / peaks["hbm_gbs"])
+    del a, b, xo
+    # line-wise pruning of a feature map (Sec. 4, CNN): the first-stage output of a ResNet-50 on 224 x 224
+    # images, 56 x 56 positions of 256 channels, 8 rows and 8 columns removed; batch scaled past the L2
+    Hh, Ww, Dc, dr, dc = 56, 56, 256, 8, 8
+    Bl = int(600e6 // (Hh * Ww * Dc * 2)) + 1
+    fm = [torch.randn(Bl, Hh, Ww, Dc, device=dev).to(torch.bfloat16) for _ in range(2)]
+    ls = torch.rand(Bl, Hh, Ww, device=dev)
+    lo = torch.empty(Bl, Hh - dr, Ww - dc, Dc, dtype=torch.bfloat16, device=dev)
+    lr = torch.empty(Bl, Hh - dr, dtype=torch.int32, device=dev)
+    lc = torch.empty(Bl, Ww - dc, dtype=torch.int32, device=dev)
+
+    def linewise():
+        cnt[0] += 1
+        ctx.linewise_compact(ls, fm[cnt[0] % 2], dr, dc, x_out=lo, keep_rows=lr, keep_cols=lc)
+    sec = bench(linewise, 10)
+    byt = 4 * Bl * Hh * Ww + 2 * Bl * (Hh - dr) * (Ww - dc) * Dc * 2
+    out["linewise_compact"] = dict(B=Bl, H=Hh, W=Ww, D=Dc, drop_rows=dr, drop_cols=dc, mbytes=byt / 1e6, us=sec * 1e6,
+                                   gbs=byt / sec / 1e9, frac_of_hbm_peak=byt / sec / 1e9 / peaks["hbm_gbs"])
     return out
 
 

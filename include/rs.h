@@ -138,6 +138,23 @@ RS_API rs_status rs_topk_compact(rs_ctx* ctx, rs_dtype dtype, int B, int N, int 
                           const float* scores, const void* x, void* x_out, int32_t* keep_idx,
                           void* stream);
 
+/* ---- rs_linewise_compact: Sec. 4 "CNN and SSM", line-wise variant (L-W) --------------------
+ * A feature map is an H x W grid of tokens with D channels each (channels last).  The scores
+ * (the representation shift of every position, e.g. from rs_shift_score on the [B, H*W, D]
+ * maps before and after a stage) are averaged over every row and over every column of the
+ * full grid; the drop_rows rows and drop_cols columns with the lowest averages are removed,
+ * whole lines at a time, so the result is again a dense grid.  A line outranks another when
+ * its average is larger, or equal with the lower index; NaN averages rank last.  Averages
+ * are fp64 sums in index order divided by the line length.
+ * scores (dev): [B, H, W] fp32.  x (dev): [B, H, W, D] of `dtype`; x_out (dev):
+ * [B, H-drop_rows, W-drop_cols, D], must not overlap x; both may be NULL to get the indices
+ * only.  keep_rows (dev): [B, H-drop_rows] int32 ascending; keep_cols (dev):
+ * [B, W-drop_cols].  1 <= H, W <= 256; 0 <= drop_rows <= H-1; 0 <= drop_cols <= W-1;
+ * D a multiple of 8.  Errors: RS_ERR_INVALID_ARG / RS_ERR_UNSUPPORTED before any launch. */
+RS_API rs_status rs_linewise_compact(rs_ctx* ctx, rs_dtype dtype, int B, int H, int W, int D, int drop_rows,
+                                     int drop_cols, const float* scores, const void* x, void* x_out,
+                                     int32_t* keep_rows, int32_t* keep_cols, void* stream);
+
 /* ---- rs_block_fwd: Eq. att + Eq. MLP + score + pruning in one call ----------------------
  * dtype: storage type of x, the weight matrices and x_out.  With RS_BF16 the
  * contractions run on the tensor cores with fp32 accumulation; the residual

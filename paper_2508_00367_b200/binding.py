@@ -27,7 +27,7 @@ EXPORTS = ("rs_create", "rs_destroy", "rs_last_error", "rs_async_status", "rs_us
            "rs_launch_count", "rs_attn_fwd", "rs_shift_score", "rs_topk_compact",
            "rs_block_workspace_bytes", "rs_block_fwd", "rs_timing_enable", "rs_timing_read",
            "rs_static_scratch_bytes", "rs_block_fwd_static", "rs_linear_fwd", "rs_vit_workspace_bytes", "rs_vit_fwd",
-           "rs_vit_fwd_taps")
+           "rs_vit_fwd_taps", "rs_linewise_compact")
 LIN_EPILOGUE = {"bias": 0, "gelu": 1, "residual": 2}
 KERNEL_CLASSES = ("layernorm", "gemm", "attn", "score", "select", "gather")
 
@@ -110,6 +110,8 @@ def load_library() -> ctypes.CDLL:
     lib.rs_shift_score.restype = ci
     lib.rs_topk_compact.argtypes = [vp, ci, ci, ci, ci, ci, ci, vp, vp, vp, vp, vp]
     lib.rs_topk_compact.restype = ci
+    lib.rs_linewise_compact.argtypes = [vp, ci, ci, ci, ci, ci, ci, ci, vp, vp, vp, vp, vp, vp]
+    lib.rs_linewise_compact.restype = ci
     lib.rs_block_workspace_bytes.argtypes = [ctypes.POINTER(BlockDesc)]
     lib.rs_block_workspace_bytes.restype = ctypes.c_size_t
     lib.rs_block_fwd.argtypes = [vp, ctypes.POINTER(BlockDesc), ctypes.POINTER(BlockWeights), vp, vp, vp, vp,
@@ -267,6 +269,27 @@ class Context:
         self._check(self.lib.rs_topk_compact(self.handle, dt, B, N, D, r, int(has_cls), _ptr(scores), _ptr(x),
                                              _ptr(x_out), _ptr(keep_idx), _stream(scores.device)))
         return x_out, keep_idx
+
+    # ---- rs_linewise_compact ----
+    def linewise_compact(self, scores: torch.Tensor, x: Optional[torch.Tensor], drop_rows: int, drop_cols: int,
+                         x_out: Optional[torch.Tensor] = None, keep_rows: Optional[torch.Tensor] = None,
+                         keep_cols: Optional[torch.Tensor] = None):
+        """scores [B, H, W] fp32, x [B, H, W, D] or None -> (x_out or None, keep_rows, keep_cols)."""
+        B, H, W = scores.shape
+        assert scores.dtype == torch.float32 and scores.is_contiguous()
+        if keep_rows is None:
+            keep_rows = torch.empty(B, max(H - drop_rows, 0), dtype=torch.int32, device=scores.device)
+        if keep_cols is None:
+            keep_cols = torch.empty(B, max(W - drop_cols, 0), dtype=torch.int32, device=scores.device)
+        D, dt = 8, RS_F32
+        if x is not None:
+            assert x.is_contiguous() and tuple(x.shape[:3]) == (B, H, W)
+            D, dt = x.shape[3], _dt(x)
+            if x_out is None:
+                x_out = torch.empty(B, max(H - drop_rows, 0), max(W - drop_cols, 0), D, dtype=x.dtype, device=x.device)
+        self._check(self.lib.rs_linewise_compact(self.handle, dt, B, H, W, D, drop_rows, drop_cols, _ptr(scores), _ptr(x),
+                                                 _ptr(x_out), _ptr(keep_rows), _ptr(keep_cols), _stream(scores.device)))
+        return x_out, keep_rows, keep_cols
 
     # ---- rs_vit_fwd ----
     def vit_fwd(self, x: torch.Tensor, weights: Sequence["DeviceBlockWeights"], H: int, drops: Sequence[int],

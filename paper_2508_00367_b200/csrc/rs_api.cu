@@ -269,6 +269,36 @@ size_t rs_block_workspace_bytes(const rs_block_desc* d) {
     return ws.total;
 }
 
+rs_status rs_linewise_compact(rs_ctx* ctx, rs_dtype dtype, int B, int H, int W, int D, int drop_rows, int drop_cols,
+                              const float* scores, const void* x, void* x_out, int32_t* keep_rows,
+                              int32_t* keep_cols, void* stream) {
+    if (!ctx) return RS_ERR_INVALID_ARG;
+    if (!valid_dtype(dtype)) return fail(ctx, RS_ERR_INVALID_ARG, "rs_linewise_compact: bad dtype");
+    if (B < 0 || H < 1 || W < 1) return fail(ctx, RS_ERR_INVALID_ARG, "rs_linewise_compact: need B >= 0, H >= 1, W >= 1");
+    if (H > rs::linewise_max_lines() || W > rs::linewise_max_lines())
+        return fail(ctx, RS_ERR_UNSUPPORTED, "rs_linewise_compact: H and W up to %d", rs::linewise_max_lines());
+    if (drop_rows < 0 || drop_rows > H - 1 || drop_cols < 0 || drop_cols > W - 1)
+        return fail(ctx, RS_ERR_INVALID_ARG, "rs_linewise_compact: need 0 <= drop_rows <= H-1 and 0 <= drop_cols <= W-1");
+    if (B == 0) return RS_OK;
+    if (!scores || !keep_rows || !keep_cols) return fail(ctx, RS_ERR_INVALID_ARG, "rs_linewise_compact: null scores or index list");
+    if ((x == nullptr) != (x_out == nullptr))
+        return fail(ctx, RS_ERR_INVALID_ARG, "rs_linewise_compact: x and x_out must both be given or both be NULL");
+    const int Hk = H - drop_rows, Wk = W - drop_cols;
+    if (x) {
+        if (D < 8 || (D % 8) != 0) return fail(ctx, RS_ERR_INVALID_ARG, "rs_linewise_compact: D must be a positive multiple of 8");
+        if (!aligned16(x) || !aligned16(x_out)) return fail(ctx, RS_ERR_INVALID_ARG, "rs_linewise_compact: misaligned pointer");
+        const size_t sz = rs::dtype_size(dtype);
+        const char* xa = (const char*)x;
+        const char* xo = (const char*)x_out;
+        const size_t xbytes = (size_t)B * H * W * D * sz, obytes = (size_t)B * Hk * Wk * D * sz;
+        if (xa < xo + obytes && xo < xa + xbytes) return fail(ctx, RS_ERR_INVALID_ARG, "rs_linewise_compact: x_out overlaps x");
+    }
+    cudaStream_t st = (cudaStream_t)stream;
+    RS_CHECK_LAUNCH(ctx, RS_K_GATHER, st, rs::launch_linewise(scores, B, H, W, Hk, Wk, keep_rows, keep_cols, dtype, x, D, x_out, ctx->sm_count, st),
+                    "line-wise select+gather launch");
+    return RS_OK;
+}
+
 // The block, with the two hooks the layer loop uses to save one kernel per block: `x_ln`, when
 // non-null, is LN1(x) already computed (by the previous block's compaction); `next_ln`, when
 // non-null, asks for LN(x_out) with the next block's LN1 parameters in next_ln->out, written by the

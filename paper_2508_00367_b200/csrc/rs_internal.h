@@ -83,6 +83,12 @@ bool select_gather_fusable(int N, int K);
 cudaError_t launch_select_gather(const float* scores, int nparts, float* scores_out, int B, int N, int K, int has_cls,
                                  int32_t* keep_idx, rs_dtype dtype, const void* x, int D, void* x_out,
                                  const LnFuse* ln /*null: none*/, int sm_count, cudaStream_t st);
+// Line-wise pruning of a 2-D token grid: keep_rows [B, Hk], keep_cols [B, Wk] and, when x is given,
+// x_out[b, i, j, :] = x[b, keep_rows[b, i], keep_cols[b, j], :].  H, W <= linewise_max_lines().
+int linewise_max_lines();
+cudaError_t launch_linewise(const float* scores, int B, int H, int W, int Hk, int Wk, int32_t* keep_rows,
+                            int32_t* keep_cols, rs_dtype dtype, const void* x, int D, void* x_out, int sm_count,
+                            cudaStream_t st);
 size_t select_smem_bytes(int N);
 cudaError_t select_init();   // opt in to large dynamic shared memory once per process/device
 

@@ -355,6 +355,110 @@ gather_kernel(const uint4* __restrict__ x, const int32_t* __restrict__ keep_idx,
     copy_row<MAXV, LT>(x + (b * N + src) * row_vecs, row, row_vecs, lane, x_out, ln);
 }
 
+// Line-wise pruning of an H x W token grid (Sec. 4, CNN variant L-W): the shift is averaged over
+// every row and every column of the full grid, and the lines with the lowest averages go.  Grid
+// (G, B): every CTA of sample b repeats the cheap part — one thread per line sums its line in
+// fp64 in index order (the order a plain loop takes, so the averages are the same doubles on any
+// machine), ranks it among its peers by counting (larger average first, lower index on a tie, NaN
+// last) and the kept lines are numbered by a count over the flags — and then copies its share of
+// the Hk x Wk kept positions, a warp per position.  CTA 0 of the sample writes the two index lists.
+constexpr int kLineMax = 256;
+constexpr int kMapMax = 8192;               // scores of one sample staged in shared memory (32 KB)
+
+__device__ __forceinline__ bool line_outranks(double a, int ia, double b, int ib) {
+    if (a != a) return (b != b) && ia < ib;
+    if (b != b) return true;
+    return a > b || (a == b && ia < ib);
+}
+
+template <int MAXV>
+__global__ void __launch_bounds__(256)
+linewise_kernel(const float* __restrict__ scores, int H, int W, int Hk, int Wk, int32_t* __restrict__ keep_rows,
+                int32_t* __restrict__ keep_cols, const uint4* __restrict__ x, int row_vecs, uint4* __restrict__ x_out) {
+    __shared__ double mean[2 * kLineMax];      // rows, then columns
+    __shared__ int32_t kept[2 * kLineMax];
+    __shared__ unsigned char flag[2 * kLineMax];
+    __shared__ float smap[kMapMax];
+    grid_dep_launch();
+    grid_dep_wait();
+    const int b = blockIdx.y;
+    const float* s = scores + (long long)b * H * W;
+    // a map of up to kMapMax scores is staged in shared memory first (coalesced, all threads), so
+    // that the per-line loops below do not wait on global memory one element at a time
+    const bool staged = H * W <= kMapMax;
+    if (staged) {
+        for (int i = threadIdx.x; i < H * W; i += blockDim.x) smap[i] = s[i];
+        __syncthreads();
+    }
+    const float* sv = staged ? smap : s;
+    for (int l = threadIdx.x; l < H + W; l += blockDim.x) {
+        double acc = 0.0;
+        if (l < H) {
+            for (int w = 0; w < W; ++w) acc += (double)sv[l * W + w];
+            mean[l] = acc / (double)W;
+        } else {
+            const int c = l - H;
+            for (int h = 0; h < H; ++h) acc += (double)sv[h * W + c];
+            mean[kLineMax + c] = acc / (double)H;
+        }
+    }
+    __syncthreads();
+    for (int l = threadIdx.x; l < H + W; l += blockDim.x) {
+        const bool row = l < H;
+        const int i = row ? l : l - H, n = row ? H : W, want = row ? Hk : Wk;
+        const double* m = mean + (row ? 0 : kLineMax);
+        const double mine = m[i];
+        int rank = 0;
+        for (int j = 0; j < n; ++j) rank += (j != i) && line_outranks(m[j], j, mine, i);
+        flag[(row ? 0 : kLineMax) + i] = rank < want;
+    }
+    __syncthreads();
+    for (int l = threadIdx.x; l < H + W; l += blockDim.x) {
+        const bool row = l < H;
+        const int i = row ? l : l - H, off = row ? 0 : kLineMax;
+        if (!flag[off + i]) continue;
+        int pos = 0;
+        for (int j = 0; j < i; ++j) pos += flag[off + j];
+        kept[off + pos] = i;
+        if (blockIdx.x == 0) (row ? keep_rows + (long long)b * Hk : keep_cols + (long long)b * Wk)[pos] = i;
+    }
+    __syncthreads();
+    if (!x) return;
+    const int P = Hk * Wk, G = gridDim.x, per = (P + G - 1) / G;
+    const int lo = blockIdx.x * per, hi = min(lo + per, P);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    const LnFuse none = {nullptr, nullptr, 0.f, nullptr};
+    auto src_of = [&](int p) {
+        const int i = p / Wk, j = p - i * Wk;
+        return x + (((long long)b * H + kept[i]) * W + kept[kLineMax + j]) * row_vecs;
+    };
+    if (row_vecs <= 32) {
+        // short rows (up to 512 bytes): a warp takes 32 / rv positions side by side (rv = the row's
+        // 16-byte pieces rounded up to a power of two) and four such groups per step, so that every
+        // lane has four loads in flight
+        int rv = 1;
+        while (rv < row_vecs) rv <<= 1;
+        const int side = 32 / rv, sub = lane / rv, v = lane - sub * rv, step = side * 4;
+        for (int p0 = lo + warp * step; p0 < hi; p0 += nwarps * step) {
+            uint4 val[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int p = p0 + u * side + sub;
+                if (p < hi && v < row_vecs) val[u] = __ldg(src_of(p) + v);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int p = p0 + u * side + sub;
+                if (p < hi && v < row_vecs) x_out[((long long)b * P + p) * row_vecs + v] = val[u];
+            }
+        }
+        return;
+    }
+    for (int p = lo + warp; p < hi; p += nwarps)
+        copy_row<MAXV, void>(src_of(p), (long long)b * P + p, row_vecs, lane, x_out, none);
+}
+
+
 }  // namespace
 
 size_t select_smem_bytes(int N) { return (size_t)N * sizeof(uint32_t); }
@@ -417,6 +521,26 @@ cudaError_t launch_gather(rs_dtype dtype, const void* x, const int32_t* keep_idx
     if (!ln) return RS_G_CASE(void);
     return dtype == RS_BF16 ? RS_G_CASE(__nv_bfloat16) : RS_G_CASE(float);
 #undef RS_G_CASE
+}
+
+int linewise_max_lines() { return kLineMax; }
+
+cudaError_t launch_linewise(const float* scores, int B, int H, int W, int Hk, int Wk, int32_t* keep_rows,
+                            int32_t* keep_cols, rs_dtype dtype, const void* x, int D, void* x_out, int sm_count,
+                            cudaStream_t st) {
+    if (B == 0) return cudaSuccess;
+    const int row_vecs = x ? (int)((size_t)D * dtype_size(dtype) / 16) : 0;
+    // about eight CTAs per SM in all (measured best between six and twelve), at least 16 positions
+    // each; one CTA per sample for the indices alone
+    int G = 1;
+    if (x) {
+        G = (8 * sm_count + B - 1) / B;
+        const int cap = (Hk * Wk + 15) / 16;
+        if (G > cap) G = cap;
+        if (G < 1) G = 1;
+    }
+    return launch_pdl(linewise_kernel<4>, dim3(G, B), dim3(256), 0, st, scores, H, W, Hk, Wk, keep_rows, keep_cols,
+                      (const uint4*)x, row_vecs, (uint4*)x_out);
 }
 
 }  // namespace rs

@@ -148,6 +148,51 @@ def test_topk_indices_only_and_errors(ctx):
     ctx.async_status()                               # context still healthy
 
 
+# ------------------------------------------------------------------ rs_linewise_compact (Sec. 4, CNN variant L-W)
+@pytest.mark.parametrize("kind", ["normal", "ties", "special"])
+@pytest.mark.parametrize("B,H,W,D,dr,dc,dtype", [
+    (2, 56, 56, 64, 8, 8, "bf16"),        # ResNet stage 1 of a 224 x 224 image: 8 rows and 8 columns go
+    (3, 28, 28, 128, 4, 4, "bf16"),       # stage 2: 4 and 4
+    (2, 7, 13, 8, 6, 12, "f32"),          # one row and one column left
+    (1, 1, 1, 8, 0, 0, "f32"),
+    (2, 33, 5, 264, 0, 2, "bf16"),        # ragged channel count (33 pieces of 16 bytes), nothing from the rows
+    (1, 256, 256, 8, 100, 3, "bf16"),     # the largest grid
+])
+def test_linewise_compact_bit_exact(ctx, kind, B, H, W, D, dr, dc, dtype):
+    s = _scores(B, H * W, kind, H * 1000 + W).reshape(B, H, W)
+    x = _tok((B, H, W, D), DT[dtype], H + W)
+    xo, kr, kc = ctx.linewise_compact(torch.from_numpy(s).cuda(), x.cuda(), dr, dc)
+    want_r, want_c = orc.linewise(s.astype(np.float64), dr, dc)
+    np.testing.assert_array_equal(kr.cpu().numpy(), want_r)
+    np.testing.assert_array_equal(kc.cpu().numpy(), want_c)
+    want_x = orc.grid_gather(x.double().numpy(), want_r, want_c)
+    np.testing.assert_array_equal(xo.cpu().double().numpy(), want_x)
+
+
+def test_linewise_after_shift_score_and_errors(ctx):
+    # the whole step on a feature map: shift of every position across a stage, then the line-wise cut.
+    # The oracle ranks the same fp32 scores (the decision is taken on what the score kernel wrote).
+    B, H, W, D = 2, 28, 28, 128
+    before = _tok((B, H, W, D), torch.bfloat16, 5)
+    after = _tok((B, H, W, D), torch.bfloat16, 6)
+    sc = ctx.shift_score(after.cuda().view(B, H * W, D), before.cuda().view(B, H * W, D)).view(B, H, W)
+    _, kr, kc = ctx.linewise_compact(sc, None, 4, 4)
+    want_r, want_c = orc.linewise(sc.cpu().double().numpy(), 4, 4)
+    np.testing.assert_array_equal(kr.cpu().numpy(), want_r)
+    np.testing.assert_array_equal(kc.cpu().numpy(), want_c)
+    full = orc.shift_score(after.double().numpy().reshape(B, H * W, D), before.double().numpy().reshape(B, H * W, D))
+    np.testing.assert_allclose(sc.cpu().numpy().reshape(B, H * W).astype(np.float64), full, rtol=2e-6, atol=0)
+    import paper_2508_00367_b200 as rs
+    for bad in ((H, 0), (0, W), (-1, 0)):
+        with pytest.raises(rs.RsError):
+            ctx.linewise_compact(sc, None, *bad)
+    with pytest.raises(rs.RsError):
+        ctx.linewise_compact(torch.zeros(1, 257, 4, device="cuda"), None, 1, 1)       # more lines than supported
+    with pytest.raises(rs.RsError):
+        ctx.linewise_compact(sc, torch.zeros(B, H, W, 12, device="cuda"), 1, 1)      # D not a multiple of 8
+    ctx.async_status()
+
+
 # ------------------------------------------------------------------ rs_attn_fwd
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("B,N,H", [(2, 197, 6), (1, 1, 1), (1, 2, 2), (2, 17, 3), (1, 127, 2), (1, 128, 2),
