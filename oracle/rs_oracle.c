@@ -4,7 +4,8 @@
  * A plain, slow, fp64 CPU statement of what the Representation Shift hot path
  * computes: one pre-LN Vision-Transformer block (Eq. att, Eq. MLP), the
  * representation-shift score of Sec. 3.2 (s = D(F(x), x)), and the removal of
- * the r lowest-score tokens (Sec. 3.1, "reduced token set").  Only the tests,
+ * the r lowest-score tokens (Sec. 3.1, "reduced token set"), plus the line-wise
+ * pruning of a 2-D token grid (Sec. 4, CNN).  Only the tests,
  * the smoke check and the benchmark's cpu_baseline / reference arm may call
  * it.  It shares no code with the CUDA library and includes none of its
  * headers.
