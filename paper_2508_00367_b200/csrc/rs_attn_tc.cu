@@ -35,9 +35,10 @@ constexpr int kSoftmaxRegs = 208, kOtherRegs = 88;   // per-thread register budg
 constexpr int kTmemCols = 512;                  // S_A 0..127, S_B 128..255, P_A 256..319, P_B 320..383, O_A 384..447, O_B 448..511
 constexpr int kPCol = 256, kOCol = 384;
 constexpr float kRescaleGap = 8.f;              // log2 units the tile maximum may exceed the running one
-// shared memory: Q[2 buffers][A, B] | K[NS] | V[NS] | barriers
+// shared memory: Q[2 buffers][A, B] | K[NS] | V[NS] | output staging | barriers
 constexpr int OFF_Q = 0, OFF_K = 4 * TILE_BYTES, OFF_V = (4 + NS) * TILE_BYTES;
-constexpr int OFF_BAR = (4 + 2 * NS) * TILE_BYTES;
+constexpr int OFF_OST = (4 + 2 * NS) * TILE_BYTES;   // output staging: 8 softmax warps x 32 rows x 128 bytes
+constexpr int OFF_BAR = OFF_OST + 8 * 4096;
 constexpr size_t kSmem = (size_t)OFF_BAR + 256 + 1024 /*alignment slack*/;
 
 struct AttnArgs {
@@ -174,7 +175,7 @@ __device__ __forceinline__ float exp_pass(uint32_t (&r)[128], float sl, float mn
 template <bool FINE>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-               const __grid_constant__ CUtensorMap tmV, const AttnArgs args) {
+               const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO, const AttnArgs args) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + OFF_BAR);
@@ -195,7 +196,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     const int N = args.N;
 
     if (threadIdx.x == 0) {
-        prefetch_tmap(&tmQ); prefetch_tmap(&tmK); prefetch_tmap(&tmV);
+        prefetch_tmap(&tmQ); prefetch_tmap(&tmK); prefetch_tmap(&tmV); prefetch_tmap(&tmO);
         for (int i = 0; i < 2; ++i) { mbar_init(&q_full[i], 1); mbar_init(&q_empty[i], 1); }
         for (int s = 0; s < NS; ++s) { mbar_init(&k_full[s], 1); mbar_init(&v_full[s], 1); mbar_init(&kv_empty[s], 1); }
         for (int g = 0; g < 2; ++g) { mbar_init(&s_full[g], 1); mbar_init(&p_ready[g], 4); mbar_init(&o_done[g], 1); mbar_init(&s_free[g], 4); }
@@ -362,7 +363,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         for (int w = blockIdx.x; w < args.n_items && ok; w += gridDim.x, ++item_n) {
             const Item it = decode_item(args, w);
             if (g >= it.ng) continue;
-            const int row = (g ? it.q0[1] : it.q0[0]) + q * 32 + lane;
             float m_l2 = 0.f, l_run = 0.f;               // running maximum (times scale*log2 e) and sum
             for (int j = 0; j < it.nkv && ok; ++j, ++cnt) {
                 const int valid = min(BKV, N - j * BKV);
@@ -439,22 +439,34 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             if (!ok || !__all_sync(0xffffffffu, mbar_wait(&o_done[g], (cnt - 1) & 1u, abort_flag))) { ok = false; break; }
             tc_fence_after();
             const float inv = 1.f / l_run;
-            __nv_bfloat16* op = args.out + ((size_t)((size_t)it.b * N + row) * args.H + (g ? it.h[1] : it.h[0])) * DH;
             uint32_t o[64];
             tmem_ld_32x32(o_addr, o);
             tmem_ld_32x32(o_addr + 32, o + 32);
             tmem_wait_ld();
-            if (row < N) {
+            // The warp's 32 rows x 64 values go to its own slab of shared memory (128-byte rows,
+            // 16-byte pieces XOR-swizzled like the tensor map's box) and leave with one TMA store,
+            // which drops the rows past N.  Storing a row per lane straight to global memory cost
+            // about 200 cycles per 16-byte store instruction (32 lines touched by each).
+            if (lane == 0) tma_store_wait_read<0>();     // the slab's previous store has read it
+            __syncwarp();
+            uint8_t* slab = smem + OFF_OST + (g * 4 + q) * 4096 + (lane >> 3) * 1024 + (lane & 7) * 128;
 #pragma unroll
-                for (int g8 = 0; g8 < 8; ++g8) {
-                    uint32_t wv[4];
+            for (int g8 = 0; g8 < 8; ++g8) {
+                uint32_t wv[4];
 #pragma unroll
-                    for (int e = 0; e < 4; ++e)
-                        wv[e] = pack_bf16(__uint_as_float(o[8 * g8 + 2 * e]) * inv, __uint_as_float(o[8 * g8 + 2 * e + 1]) * inv);
-                    *reinterpret_cast<uint4*>(op + g8 * 8) = make_uint4(wv[0], wv[1], wv[2], wv[3]);
-                }
+                for (int e = 0; e < 4; ++e)
+                    wv[e] = pack_bf16(__uint_as_float(o[8 * g8 + 2 * e]) * inv, __uint_as_float(o[8 * g8 + 2 * e + 1]) * inv);
+                *reinterpret_cast<uint4*>(slab + ((g8 ^ (lane & 7)) << 4)) = make_uint4(wv[0], wv[1], wv[2], wv[3]);
+            }
+            fence_async_smem();
+            __syncwarp();
+            const int row0 = (g ? it.q0[1] : it.q0[0]) + q * 32;
+            if (lane == 0 && row0 < N) {
+                tma_store_4d(&tmO, smem + OFF_OST + (g * 4 + q) * 4096, 0, g ? it.h[1] : it.h[0], row0, it.b);
+                tma_store_commit();
             }
         }
+        if (lane == 0) tma_store_wait<0>();              // every output row written before the CTA exits
     }
     }
 
@@ -474,14 +486,14 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 
 // [B, N, H, 64] view with element strides; box = 128 rows of one head of one sample.
 bool make_tmap_qkv(void* encode_fn, CUtensorMap* out, const void* base, int B, int N, int H, long long bs,
-                   long long rs_, long long hs) {
+                   long long rs_, long long hs, int box_rows = 128) {
     EncodeTiledFn fn = reinterpret_cast<EncodeTiledFn>(encode_fn);
     const cuuint64_t dims[4] = {64, (cuuint64_t)H, (cuuint64_t)N, (cuuint64_t)B};
     // a dimension of extent 1 never uses its stride; give it a harmless valid one
     const cuuint64_t hs_b = (H > 1 ? (cuuint64_t)hs : 64) * 2, rs_b = (N > 1 ? (cuuint64_t)rs_ : 64) * 2,
                      bs_b = (B > 1 ? (cuuint64_t)bs : 64) * 2;
     const cuuint64_t strides[3] = {hs_b, rs_b, bs_b};
-    const cuuint32_t box[4] = {64, 1, 128, 1};
+    const cuuint32_t box[4] = {64, 1, (cuuint32_t)box_rows, 1};
     const cuuint32_t estr[4] = {1, 1, 1, 1};
     return fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -515,8 +527,10 @@ cudaError_t launch_attn_tc(rs_ctx* ctx, const rs_attn_desc& d, const void* q, co
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
-    CUtensorMap tmQ, tmK, tmV;
-    if (!make_tmap_qkv(ctx->encode_tiled, &tmQ, q, d.B, d.N, d.H, d.q_batch_stride, d.q_row_stride, d.q_head_stride) ||
+    CUtensorMap tmQ, tmK, tmV, tmO;
+    // out is [B, N, H, 64] contiguous; a softmax warp stores its 32 rows of one head at a time
+    if (!make_tmap_qkv(ctx->encode_tiled, &tmO, out, d.B, d.N, d.H, (long long)d.N * d.H * 64, (long long)d.H * 64, 64, 32) ||
+        !make_tmap_qkv(ctx->encode_tiled, &tmQ, q, d.B, d.N, d.H, d.q_batch_stride, d.q_row_stride, d.q_head_stride) ||
         !make_tmap_qkv(ctx->encode_tiled, &tmK, k, d.B, d.N, d.H, d.k_batch_stride, d.k_row_stride, d.k_head_stride) ||
         !make_tmap_qkv(ctx->encode_tiled, &tmV, v, d.B, d.N, d.H, d.v_batch_stride, d.v_row_stride, d.v_head_stride))
         return cudaErrorInvalidValue;
@@ -537,8 +551,8 @@ cudaError_t launch_attn_tc(rs_ctx* ctx, const rs_attn_desc& d, const void* q, co
     const int nkv = (d.N + BKV - 1) / BKV;
     const int grid = (nkv >= 16 || args.n_items < ctx->sm_count) ? args.n_items : ctx->sm_count;
     // a partial key tile is worth its own code when it is a good part of the sequence
-    if (nkv <= 12) return launch_pdl(attn_tc_kernel<true>, dim3(grid), dim3(kThreads), kSmem, st, tmQ, tmK, tmV, args);
-    return launch_pdl(attn_tc_kernel<false>, dim3(grid), dim3(kThreads), kSmem, st, tmQ, tmK, tmV, args);
+    if (nkv <= 12) return launch_pdl(attn_tc_kernel<true>, dim3(grid), dim3(kThreads), kSmem, st, tmQ, tmK, tmV, tmO, args);
+    return launch_pdl(attn_tc_kernel<false>, dim3(grid), dim3(kThreads), kSmem, st, tmQ, tmK, tmV, tmO, args);
 }
 
 }  // namespace rs
