@@ -36,16 +36,24 @@ constexpr int kThreads = 320;                 // warp 0: TMA, warp 1: MMA (leade
 constexpr int kEpiWarps = 8;
 constexpr int A_BYTES = BM * BK * 2;          // 16 KB
 constexpr int STG_BYTES = 32 * 128;           // one staged output block of a warp: its 32 rows of 128 bytes
-constexpr int kStgBufs = 2 * kEpiWarps;       // two per epilogue warp
+constexpr int RES_BOX_BYTES = 32 * 64;         // residual of one 32-column chunk of a warp: 32 rows of 32 bf16
 
-template <int BN> struct Cfg {
+// EPI_RESID brings the bf16 residual of a warp's rows in by TMA (a row per lane read straight from
+// global memory touches 32 lines per load instruction and cost a fifth of the projection's time):
+// one buffer per warp for a whole tile, loaded while the previous tile's main loop runs.  It pays
+// for the room with one staging buffer per warp instead of two and one operand stage less.
+template <int BN, int EPI> struct Cfg {
+    static constexpr bool RES_TMA = EPI == EPI_RESID;
     static constexpr int B_BYTES = (BN / 2) * BK * 2;              // this CTA's half of the W tile
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    static constexpr int STAGES = (BN == 128) ? 6 : 5;
+    static constexpr int STAGES = (BN == 128) ? 6 : RES_TMA ? 4 : 5;
     static constexpr int TMEM_COLS = (BN == 128) ? 256 : 512;      // two accumulators, a power of two
     static constexpr int SPLIT = (BN == 128) ? 64 : 128;           // epilogue warps 2-5 take columns [0, SPLIT)
+    static constexpr int STG_PER_WARP = RES_TMA ? 1 : 2;
+    static constexpr int RES_WARP_BYTES = RES_TMA ? (SPLIT / 32) * RES_BOX_BYTES : 0;   // the wider half's chunks
     static constexpr int OFF_STG = STAGES * STAGE_BYTES;
-    static constexpr int OFF_BAR = OFF_STG + kStgBufs * STG_BYTES;
+    static constexpr int OFF_RES = OFF_STG + kEpiWarps * STG_PER_WARP * STG_BYTES;
+    static constexpr int OFF_BAR = OFF_RES + kEpiWarps * RES_WARP_BYTES;
     static constexpr int OFF_BIAS = OFF_BAR + 256;                 // float [2 tile parities][2 halves][128]: bias slices
     static constexpr size_t SMEM = (size_t)OFF_BIAS + 2048;        // the window itself must be 1024-byte aligned
     static_assert(SMEM <= 227 * 1024, "shared memory of one CTA");
@@ -95,8 +103,9 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
 template <int BN, int EPI, typename OutT>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-               const __grid_constant__ CUtensorMap tmOut, const GemmArgs args) {
-    using C = Cfg<BN>;
+               const __grid_constant__ CUtensorMap tmOut, const __grid_constant__ CUtensorMap tmRes,
+               const GemmArgs args) {
+    using C = Cfg<BN, EPI>;
     // The 128-byte swizzle wants 1024-byte aligned stage and staging buffers, and the layout leaves no
     // room to round the base up: a window that is not aligned is reported, and nothing else is done.
     extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -113,6 +122,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * C::STAGES + 4);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     volatile int* half_fail = reinterpret_cast<volatile int*>(tmem_slot + 2);   // [2]
+    uint64_t* res_full = bars + 2 * C::STAGES + 6;   // [kEpiWarps] the warp's residual of a tile landed (EPI_RESID)
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();     // 0 = leader of the pair
@@ -126,6 +136,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         prefetch_tmap(&tmOut);
         for (int s = 0; s < C::STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
         for (int a = 0; a < 2; ++a) { mbar_init(&tfull[a], 1); mbar_init(&tempty[a], 2 * kEpiWarps); }
+        if (C::RES_TMA) {
+            prefetch_tmap(&tmRes);
+            for (int w = 0; w < kEpiWarps; ++w) mbar_init(&res_full[w], 1);
+        }
         *abort_flag = 0;
         half_fail[0] = 0;
         half_fail[1] = 0;
@@ -212,6 +226,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const int t128 = ((warp - 2) & 3) * 32 + lane;   // this thread's index among the 128 of its half
         const uint32_t lead_tempty[2] = {map_to_cta(smem_u32(&tempty[0]), 0), map_to_cta(smem_u32(&tempty[1]), 0)};
         uint32_t tl = 0, blk_ctr = 0;
+        // EPI_RESID: the residual of this warp's 32 rows x its half's columns of a tile, one 64-byte-
+        // swizzled box per 32-column chunk (rows past M arrive as zeros)
+        uint8_t* res_buf = smem + C::OFF_RES + (warp - 2) * C::RES_WARP_BYTES;
+        auto issue_res = [&](int tile) {
+            const int rm0 = (tile / num_n) * (2 * BM) + (int)rank * BM + q * 32, rn0 = (tile % num_n) * BN;
+            mbar_expect_tx(&res_full[warp - 2], (uint32_t)((c_end - c_begin) / 32) * RES_BOX_BYTES);
+            for (int c = c_begin; c < c_end; c += 32)
+                tma_load_2d(res_buf + ((c - c_begin) / 32) * RES_BOX_BYTES, &tmRes, &res_full[warp - 2], rn0 + c, rm0);
+        };
+        if (C::RES_TMA && lane == 0 && pair < tiles) issue_res(pair);
         constexpr int RES_VECS = EPI == EPI_RESID ? 4 : EPI == EPI_SCORE ? 8 : 1;   // 16-byte loads per 32 columns
         for (int tile = pair; tile < tiles; tile += npairs, ++tl) {
             const int m0 = (tile / num_n) * (2 * BM) + (int)rank * BM, nt = tile % num_n, n0 = nt * BN;
@@ -221,11 +245,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             // Residual values of 32 columns of this thread's row (zeros for rows past M).  They are
             // fetched one chunk ahead, the first chunk before the accumulator is even complete.
             auto load_res = [&](int c, uint4* dst) {
-                if (EPI == EPI_RESID || EPI == EPI_SCORE) {
+                if (EPI == EPI_SCORE) {
                     const size_t off = (size_t)row * args.N + n0 + c;
-                    const uint4* rp = EPI == EPI_RESID
-                        ? reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(args.residual) + off)
-                        : reinterpret_cast<const uint4*>(reinterpret_cast<const float*>(args.residual) + off);
+                    const uint4* rp = reinterpret_cast<const uint4*>(reinterpret_cast<const float*>(args.residual) + off);
 #pragma unroll
                     for (int j = 0; j < RES_VECS; ++j) dst[j] = valid ? __ldg(rp + j) : make_uint4(0u, 0u, 0u, 0u);
                 }
@@ -240,6 +262,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             float* bias_s = reinterpret_cast<float*>(smem + C::OFF_BIAS) + (tl & 1u) * 256 + half * 128;
             if (c_begin + t128 < c_end) bias_s[t128] = args.bias ? __ldg(args.bias + n0 + c_begin + t128) : 0.f;
             if (!__all_sync(0xffffffffu, mbar_wait(&tfull[a], aph, abort_flag))) half_fail[half] = 1;
+            if (C::RES_TMA && !__all_sync(0xffffffffu, mbar_wait(&res_full[warp - 2], tl & 1u, abort_flag))) half_fail[half] = 1;
             named_barrier(1 + half, 128);
             if (half_fail[half]) break;
             tc_fence_after();
@@ -248,16 +271,24 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll 1
             for (int c = c_begin; c < c_end; c += 32) {
                 const int cb = (c / 32) % CHUNKS_PER_BLK;            // chunk inside the staged block
-                uint8_t* stg = smem + C::OFF_STG + ((warp - 2) * 2 + (blk_ctr & 1u)) * STG_BYTES;
+                uint8_t* stg = smem + C::OFF_STG + ((warp - 2) * C::STG_PER_WARP + (C::STG_PER_WARP == 2 ? (blk_ctr & 1u) : 0u)) * STG_BYTES;
                 if (cb == 0) {
-                    // the store that last read this buffer (two blocks ago) must be done with it
-                    if (lane == 0) tma_store_wait_read<1>();
+                    // the store that last read this buffer (two blocks ago, or the last one) must be done with it
+                    if (lane == 0) tma_store_wait_read<C::STG_PER_WARP - 1>();
                     __syncwarp();
                 }
                 uint4 res[RES_VECS];
+                if (C::RES_TMA) {
+                    // this lane's row of the chunk's box: 64 bytes, 16-byte pieces XOR-ed with address bits 7-8
+                    const uint8_t* rrow = res_buf + ((c - c_begin) / 32) * RES_BOX_BYTES + lane * 64;
 #pragma unroll
-                for (int j = 0; j < RES_VECS; ++j) res[j] = res_next[j];
-                if (c + 32 < c_end) load_res(c + 32, res_next);
+                    for (int j = 0; j < RES_VECS; ++j)
+                        res[j] = *reinterpret_cast<const uint4*>(rrow + ((j ^ ((lane >> 1) & 3)) << 4));
+                } else {
+#pragma unroll
+                    for (int j = 0; j < RES_VECS; ++j) res[j] = res_next[j];
+                    if (c + 32 < c_end) load_res(c + 32, res_next);
+                }
                 uint32_t r[32];
                 __syncwarp();                            // tcgen05.ld is warp-collective
                 tmem_ld_32x32(taddr + c, r);
@@ -359,6 +390,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     ++blk_ctr;
                 }
             }
+            if (C::RES_TMA) {
+                __syncwarp();                            // every lane has read its residual rows
+                if (lane == 0 && tile + npairs < tiles) issue_res(tile + npairs);
+            }
             if ((EPI == EPI_SCORE || (EPI == EPI_RESID && args.partials)) && valid) {
                 const size_t pi = (size_t)row * (2 * num_n) + 2 * nt + half;
                 if (args.dist == RS_DIST_COS) {
@@ -401,10 +436,23 @@ bool make_tmap_2d(void* encode_fn, CUtensorMap* out, const void* base, int elem_
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Tensor map over the bf16 residual [rows, cols] of the projection: box [32 rows, 32 columns = 64 bytes],
+// 64-byte swizzle, zeros for rows past the matrix.
+bool make_tmap_res(void* encode_fn, CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols) {
+    EncodeTiledFn fn = reinterpret_cast<EncodeTiledFn>(encode_fn);
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {cols * 2};
+    const cuuint32_t box[2] = {32, 32};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 template <int BN, int EPI, typename OutT>
-cudaError_t launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmOut, const GemmArgs& args,
-                       int sm_count, cudaStream_t st) {
-    using C = Cfg<BN>;
+cudaError_t launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmOut, const CUtensorMap& tmRes,
+                       const GemmArgs& args, int sm_count, cudaStream_t st) {
+    using C = Cfg<BN, EPI>;
     static bool attr_done = false;   // per instantiation; the attribute is per function, set once
     if (!attr_done) {
         cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<BN, EPI, OutT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -428,7 +476,7 @@ cudaError_t launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUt
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<BN, EPI, OutT>, tmA, tmB, tmOut, args);
+    return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<BN, EPI, OutT>, tmA, tmB, tmOut, tmRes, args);
 }
 
 // Tile width (256, 192 or 128 columns per pair): the one whose waves over the SM pairs cost
@@ -474,19 +522,21 @@ cudaError_t launch_gemm_tc(rs_ctx* ctx, int epi, const void* A, const void* W, c
     if (!ctx->encode_tiled) return cudaErrorNotSupported;
     const int bn = pick_bn(M, N, ctx->sm_count);
     const int out_bytes = (epi == EPI_RESID || (epi == EPI_SCORE && out_dtype == RS_F32)) ? 4 : 2;
-    CUtensorMap tmA, tmB, tmOut;
+    CUtensorMap tmA, tmB, tmOut, tmRes;
+    if (epi == EPI_RESID && !make_tmap_res(ctx->encode_tiled, &tmRes, residual, (uint64_t)M, (uint64_t)N)) return cudaErrorInvalidValue;
     if (!make_tmap_2d(ctx->encode_tiled, &tmA, A, 2, (uint64_t)M, (uint64_t)K, BM) ||
         !make_tmap_2d(ctx->encode_tiled, &tmB, W, 2, (uint64_t)N, (uint64_t)K, (uint32_t)(bn / 2)) ||
         !make_tmap_2d(ctx->encode_tiled, &tmOut, out, out_bytes, (uint64_t)M, (uint64_t)N, 32))
         return cudaErrorInvalidValue;
+    if (epi != EPI_RESID) tmRes = tmOut;             // unused by the other epilogues
     GemmArgs args;
     args.M = (int)M; args.N = N; args.K = K; args.bias = bias; args.residual = residual;
     args.residual2 = residual2; args.partials = partials; args.score_kind = score_kind; args.dist = dist; args.status = ctx->d_status;
     const int sms = ctx->sm_count;
 #define RS_GEMM_CASE(E, T)                                                                       \
-    return bn == 256   ? launch_one<256, E, T>(tmA, tmB, tmOut, args, sms, st)                  \
-           : bn == 192 ? launch_one<192, E, T>(tmA, tmB, tmOut, args, sms, st)                  \
-                       : launch_one<128, E, T>(tmA, tmB, tmOut, args, sms, st)
+    return bn == 256   ? launch_one<256, E, T>(tmA, tmB, tmOut, tmRes, args, sms, st)           \
+           : bn == 192 ? launch_one<192, E, T>(tmA, tmB, tmOut, tmRes, args, sms, st)           \
+                       : launch_one<128, E, T>(tmA, tmB, tmOut, tmRes, args, sms, st)
     switch (epi) {
         case EPI_BIAS: RS_GEMM_CASE(EPI_BIAS, __nv_bfloat16);
         case EPI_BIAS_GELU: RS_GEMM_CASE(EPI_BIAS_GELU, __nv_bfloat16);
