@@ -316,6 +316,39 @@ class Context:
                                         _ptr(keep), _ptr(workspace), workspace.numel(), _stream(x.device)))
         return dict(x_out=x_out, scores=scores, keep_idx=keep)
 
+    def vit_fwd_taps(self, x: torch.Tensor, weights: Sequence["DeviceBlockWeights"], H: int, drops: Sequence[int],
+                     tap_blocks: Sequence[int], has_cls: bool = True, score_mode: str = "mlp",
+                     dist: str = "l2") -> Dict[int, Dict[str, torch.Tensor]]:
+        """rs_vit_fwd_taps with outputs requested for the blocks in `tap_blocks` only (the last block is
+        always included); the other blocks' tokens live in the call's workspace.  Returns
+        {block: dict(x_out, scores, keep_idx)}."""
+        assert x.is_cuda and x.is_contiguous() and len(weights) == len(drops)
+        B, N, D = x.shape
+        L = len(weights)
+        desc = VitDesc(_dt(x), B, N, D, H, weights[0].D_mlp, L, int(has_cls), 0.0, 0.0, SCORE_MODE[score_mode], DIST[dist])
+        cdrops = (ctypes.c_int * L)(*[int(r) for r in drops])
+        warr = (BlockWeights * L)(*[w.struct for w in weights])
+        need = int(self.lib.rs_vit_workspace_bytes(ctypes.byref(desc), cdrops))
+        if need == 0:
+            raise RsError(1, "rs_vit_fwd: bad descriptor or schedule")
+        workspace = torch.empty(need, dtype=torch.uint8, device=x.device)
+        want = set(int(b) for b in tap_blocks) | {L - 1}
+        outs, n = {}, N
+        arrs = {k: (ctypes.c_void_p * L)() for k in ("x_out", "scores", "keep_idx")}
+        for l, r in enumerate(drops):
+            k = n - int(r)
+            if l in want:
+                outs[l] = dict(x_out=torch.empty(B, k, D, dtype=x.dtype, device=x.device),
+                               scores=torch.empty(B, n, dtype=torch.float32, device=x.device),
+                               keep_idx=torch.empty(B, k, dtype=torch.int32, device=x.device))
+                for key in arrs:
+                    arrs[key][l] = outs[l][key].data_ptr()
+            n = k
+        taps = VitTaps(arrs["x_out"], arrs["scores"], arrs["keep_idx"])
+        self._check(self.lib.rs_vit_fwd_taps(self.handle, ctypes.byref(desc), warr, cdrops, _ptr(x), ctypes.byref(taps),
+                                             _ptr(workspace), workspace.numel(), _stream(x.device)))
+        return outs
+
     # ---- rs_block_fwd ----
     def block_desc(self, B, N, D, H, D_mlp, r, dtype, out_dtype=None, has_cls=True, ln_eps=0.0, scale=0.0,
                    score_mode="mlp", dist="l2") -> BlockDesc:
@@ -411,10 +444,10 @@ class PrunedViT:
     compacted output; `drops[l]` tokens are removed after block l."""
 
     def __init__(self, ctx: Context, blocks: Sequence[Dict[str, torch.Tensor]], H: int, drops: Sequence[int],
-                 dtype: torch.dtype, has_cls: bool = True, score_mode: str = "mlp"):
+                 dtype: torch.dtype, has_cls: bool = True, score_mode: str = "mlp", dist: str = "l2"):
         assert len(blocks) == len(drops)
         self.ctx, self.H, self.drops, self.dtype = ctx, H, list(drops), dtype
-        self.has_cls, self.score_mode = has_cls, score_mode
+        self.has_cls, self.score_mode, self.dist = has_cls, score_mode, dist
         self.weights: List[DeviceBlockWeights] = [DeviceBlockWeights(w, dtype, ctx.device) for w in blocks]
         self._plan = None
 
@@ -434,7 +467,7 @@ class PrunedViT:
             n = k
         code = RS_BF16 if self.dtype == torch.bfloat16 else RS_F32
         desc = VitDesc(code, B, N, D, self.H, self.weights[0].D_mlp, L, int(self.has_cls), 0.0, 0.0,
-                       SCORE_MODE[self.score_mode], DIST["l2"])
+                       SCORE_MODE[self.score_mode], DIST[self.dist])
         cdrops = (ctypes.c_int * L)(*[int(r) for r in self.drops])
         warr = (BlockWeights * L)(*[w.struct for w in self.weights])
         need = int(self.ctx.lib.rs_vit_workspace_bytes(ctypes.byref(desc), cdrops))

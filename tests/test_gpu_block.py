@@ -282,6 +282,14 @@ def test_vit_fwd_equals_the_block_loop(ctx, B, N, D, H, drops, dt):
         assert torch.equal(got_l["keep_idx"], want["keep_idx"])
         assert torch.equal(got_l["scores"], want["scores"])
         assert torch.equal(got_l["x_out"], want["x_out"])
+    # outputs requested for some blocks only: the others' tokens stay in the two workspace buffers
+    some = ctx.vit_fwd_taps(x, model.weights, H, drops, tap_blocks=[1])
+    torch.cuda.synchronize()
+    assert sorted(some) == sorted({1, len(drops) - 1})
+    for l, got_l in some.items():
+        assert torch.equal(got_l["keep_idx"], chain[l]["keep_idx"])
+        assert torch.equal(got_l["scores"], chain[l]["scores"])
+        assert torch.equal(got_l["x_out"], chain[l]["x_out"])
     want = chain[-1]
     got = ctx.vit_fwd(x, model.weights, H, drops)
     torch.cuda.synchronize()
