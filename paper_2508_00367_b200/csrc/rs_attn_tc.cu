@@ -188,8 +188,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     uint64_t* p_ready = s_full + 2;          // [2] P written (one arrival per softmax warp)
     uint64_t* o_done = s_full + 4;           // [2] O += P V retired
     uint64_t* s_free = s_full + 6;           // [2] S row in registers, columns reusable (one arrival per warp)
-    uint64_t* first_pass = s_full + 8;       // tile A's warps finished the first exponent pass of an item
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(s_full + 9);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(s_full + 8);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -200,7 +199,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         for (int i = 0; i < 2; ++i) { mbar_init(&q_full[i], 1); mbar_init(&q_empty[i], 1); }
         for (int s = 0; s < NS; ++s) { mbar_init(&k_full[s], 1); mbar_init(&v_full[s], 1); mbar_init(&kv_empty[s], 1); }
         for (int g = 0; g < 2; ++g) { mbar_init(&s_full[g], 1); mbar_init(&p_ready[g], 4); mbar_init(&o_done[g], 1); mbar_init(&s_free[g], 4); }
-        mbar_init(first_pass, 4);
         *abort_flag = 0;
         mbar_fence_init();
     }
@@ -410,17 +408,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     }
                     tmem_wait_st();
                 }
-                // Tile B's first pass of an item starts when tile A's has ended: the two groups then
-                // stay out of step, and one group's loads, stores and waits hide behind the other's pass.
-                // (Tile A cannot get two items ahead of this wait: its item n+2 needs the MMA thread past
-                // tile B's P V of item n, and tile B reaches its next wait about a pass sooner than tile A
-                // can arrive again; were that ever inverted, the wait is bounded and reports.)
-                if (j == 0 && g == 1 && !__all_sync(0xffffffffu, mbar_wait(first_pass, item_n & 1u, abort_flag))) { ok = false; break; }
                 if (valid == BKV) l_run += exp_pass<128, 0>(r, sl, -m_l2, valid);
                 else if (!FINE) l_run += ncol == 64 ? exp_pass<64, 2>(r, sl, -m_l2, valid) : exp_pass<128, 2>(r, sl, -m_l2, valid);
                 else l_run += ncol == 128 ? exp_pass<128, 1>(r, sl, -m_l2, valid) : ncol == 96 ? exp_pass<96, 1>(r, sl, -m_l2, valid)
                               : ncol == 64 ? exp_pass<64, 1>(r, sl, -m_l2, valid) : exp_pass<32, 1>(r, sl, -m_l2, valid);
-                if (j == 0 && g == 0 && lane == 0) mbar_arrive(first_pass);
                 if (cnt > 0) {
                     // P V of the previous key tile reads the P columns: it must have retired
                     if (!__all_sync(0xffffffffu, mbar_wait(&o_done[g], (cnt - 1) & 1u, abort_flag))) { ok = false; break; }
