@@ -31,7 +31,7 @@ constexpr int BQ = 128, BKV = 128, DH = 64;
 constexpr int TILE_BYTES = 128 * DH * 2;        // 16 KB: a [128, 64] bf16 tile
 constexpr int NS = 4;                           // K/V ring stages
 constexpr int kThreads = 384;                   // warps 0-3 / 4-7: softmax of tile A / B, warp 8: TMA, warp 9: MMA
-constexpr int kSoftmaxRegs = 208, kOtherRegs = 88;   // per-thread register budgets after the warpgroups re-split the pool
+constexpr int kSoftmaxRegs = 216, kOtherRegs = 72;   // per-thread register budgets after the warpgroups re-split the pool
 constexpr int kTmemCols = 512;                  // S_A 0..127, S_B 128..255, P_A 256..319, P_B 320..383, O_A 384..447, O_B 448..511
 constexpr int kPCol = 256, kOCol = 384;
 constexpr float kRescaleGap = 8.f;              // log2 units the tile maximum may exceed the running one
