@@ -1,6 +1,6 @@
 // sm_100a building blocks in inline PTX: mbarrier, TMA (cp.async.bulk.tensor),
 // tensor memory (tcgen05.alloc / ld / st) and tcgen05.mma with hand-encoded
-// shared-memory and instruction descriptors.  No multicast anywhere.
+// shared-memory and instruction descriptors.  No copy uses cluster multicast (only the commit of a CTA pair signals both CTAs).
 #pragma once
 #include <cuda.h>
 #include <cuda_runtime.h>
