@@ -29,7 +29,7 @@ def build(force: bool = False) -> str:
     """Compile the C oracle with gcc (OpenMP) if the shared object is stale."""
     if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
         subprocess.check_call(
-            ["gcc", "-O2", "-march=native", "-fopenmp", "-fPIC", "-shared", "-std=c99",
+            ["gcc", "-O3", "-march=native", "-fopenmp", "-fPIC", "-shared", "-std=c99",
              "-o", _LIB, _SRC, "-lm"])
     return _LIB
 
