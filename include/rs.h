@@ -73,24 +73,16 @@ RS_API void rs_destroy(rs_ctx* ctx);
 RS_API const char* rs_last_error(const rs_ctx* ctx);
 /* Synchronise `stream`, then return and clear the device status word. */
 RS_API rs_status rs_async_status(rs_ctx* ctx, void* stream);
-/* 1 if the tcgen05 tensor-core kernels are used for (dtype), else 0 (SIMT path). */
+/* 1 if the tcgen05 tensor-core kernels are available for (dtype) on this context, else 0.
+ * Whether a given shape runs on them is answered by the two queries below. */
 RS_API int rs_uses_tensor_cores(const rs_ctx* ctx, rs_dtype dtype);
-/* Number of kernels the library has launched through this context so far. */
-RS_API long long rs_launch_count(const rs_ctx* ctx);
-
-/* Per-kernel-class device timing, for benchmarks (the paper reports whole-model
- * throughput only; this has no counterpart there).  While enabled, every launch
- * is bracketed by CUDA events on the launch stream (up to 8192 launches between
- * reads; later ones are not recorded).  rs_timing_read synchronises `stream`,
- * adds up the elapsed milliseconds and launch counts per class into the two
- * host arrays of RS_K_COUNT entries, and clears the record. */
-typedef enum {
-    RS_K_LAYERNORM = 0, RS_K_GEMM = 1, RS_K_ATTN = 2, RS_K_SCORE = 3, RS_K_SELECT = 4, RS_K_GATHER = 5,
-    RS_K_COUNT = 6
-} rs_kernel_class;
-RS_API rs_status rs_timing_enable(rs_ctx* ctx, int on);
-RS_API rs_status rs_timing_read(rs_ctx* ctx, void* stream, double* ms /*host[RS_K_COUNT]*/,
-                                long long* launches /*host[RS_K_COUNT]*/);
+/* Which kernels a call would run, by shape (Eq. att / Eq. MLP contractions and Eq. sa): 1 = the
+ * tcgen05 kernels, 0 = the fp32-FMA kernels.  The tensor-core GEMM needs RS_BF16, N % 128 == 0 and
+ * K % 64 == 0; a block runs on the tensor cores only if all four of its projections qualify
+ * (D % 128 == 0, D_mlp % 128 == 0).  Every other valid shape still computes the same result on
+ * the fp32-FMA kernels, far slower.  With RS_REQUIRE_TC=1 in the environment at rs_create such a
+ * call returns RS_ERR_UNSUPPORTED instead of taking the slow kernels. */
+RS_API int rs_linear_uses_tensor_cores(const rs_ctx* ctx, rs_dtype dtype, long long M, int N, int K);
 
 /* ---- rs_attn_fwd: Eq. sa, out = Softmax(Q K^T * scale) V per (sample, head) ----------
  * q, k, v (dev): element [b, i, h, c] lives at  b*batch_stride + i*row_stride +
@@ -177,6 +169,10 @@ typedef struct {           /* all dev pointers */
     const float *b_qkv, *b_o, *b_fc1, *b_fc2;        /* fp32; may be NULL */
     const float *ln1_g, *ln1_b, *ln2_g, *ln2_b;      /* fp32 */
 } rs_block_weights;
+
+/* 1 if rs_block_fwd runs this descriptor on the tcgen05 kernels, 0 if on the fp32-FMA kernels
+ * (see rs_linear_uses_tensor_cores). */
+RS_API int rs_block_uses_tensor_cores(const rs_ctx* ctx, const rs_block_desc* desc /*host*/);
 
 /* Bytes of scratch rs_block_fwd needs for this descriptor (0 on a bad descriptor). */
 RS_API size_t rs_block_workspace_bytes(const rs_block_desc* desc /*host*/);
@@ -267,6 +263,13 @@ RS_API rs_status rs_block_fwd_static(const rs_block_desc* desc /*host*/,
                                      const rs_block_weights* weights /*host struct of dev pointers*/,
                                      const void* x, void* x_out, float* scores, int32_t* keep_idx,
                                      void* x_full, void* stream, char* err /*host*/, size_t err_len);
+/* rs_async_status for the calls above (they have no context to ask): synchronises `stream`,
+ * then returns and clears the status word that the kernels of rs_block_fwd_static write on the
+ * current device -- RS_ERR_TIMEOUT when a bounded device-side wait ran out, RS_ERR_CUDA when a
+ * kernel found its shared-memory window misaligned or a runtime call failed; in both cases the
+ * outputs of the calls since the last query are not to be used.  RS_OK before the first
+ * rs_block_fwd_static call on the device.  Allocates nothing (one 4-byte copy to the host). */
+RS_API rs_status rs_static_async_status(void* stream, char* err /*host*/, size_t err_len);
 
 #ifdef __cplusplus
 }

@@ -1,0 +1,34 @@
+/*
+ * rs_profile.h -- instrumentation of librs.so for benchmarks: launch counting and per-kernel-class
+ * device timing.  The paper reports whole-model throughput only (Sec. 4); nothing here has a
+ * counterpart there, and no entry point of rs.h depends on it.
+ */
+#ifndef RS_PROFILE_H_
+#define RS_PROFILE_H_
+
+#include "rs.h"
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Number of kernels the library has launched through this context so far. */
+RS_API long long rs_launch_count(const rs_ctx* ctx);
+
+/* While enabled, every launch through the context is bracketed by CUDA events on the launch
+ * stream (up to 8192 launches between reads; later ones are not recorded).  rs_timing_read
+ * synchronises `stream`, adds up the elapsed milliseconds and launch counts per class into the
+ * two host arrays of RS_K_COUNT entries, and clears the record.  Errors: RS_ERR_INVALID_ARG on a
+ * null argument, RS_ERR_CUDA when an event call fails. */
+typedef enum {
+    RS_K_LAYERNORM = 0, RS_K_GEMM = 1, RS_K_ATTN = 2, RS_K_SCORE = 3, RS_K_SELECT = 4, RS_K_GATHER = 5,
+    RS_K_COUNT = 6
+} rs_kernel_class;
+RS_API rs_status rs_timing_enable(rs_ctx* ctx, int on);
+RS_API rs_status rs_timing_read(rs_ctx* ctx, void* stream, double* ms /*host[RS_K_COUNT]*/,
+                                long long* launches /*host[RS_K_COUNT]*/);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RS_PROFILE_H_ */

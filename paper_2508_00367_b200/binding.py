@@ -27,7 +27,8 @@ EXPORTS = ("rs_create", "rs_destroy", "rs_last_error", "rs_async_status", "rs_us
            "rs_launch_count", "rs_attn_fwd", "rs_shift_score", "rs_topk_compact",
            "rs_block_workspace_bytes", "rs_block_fwd", "rs_timing_enable", "rs_timing_read",
            "rs_static_scratch_bytes", "rs_block_fwd_static", "rs_linear_fwd", "rs_vit_workspace_bytes", "rs_vit_fwd",
-           "rs_vit_fwd_taps", "rs_linewise_compact")
+           "rs_vit_fwd_taps", "rs_linewise_compact", "rs_static_async_status", "rs_linear_uses_tensor_cores",
+           "rs_block_uses_tensor_cores")
 LIN_EPILOGUE = {"bias": 0, "gelu": 1, "residual": 2}
 KERNEL_CLASSES = ("layernorm", "gemm", "attn", "score", "select", "gather")
 
@@ -124,6 +125,12 @@ def load_library() -> ctypes.CDLL:
     lib.rs_block_fwd_static.argtypes = [ctypes.POINTER(BlockDesc), ctypes.POINTER(BlockWeights), vp, vp, vp, vp, vp,
                                         vp, ctypes.c_char_p, ctypes.c_size_t]
     lib.rs_block_fwd_static.restype = ci
+    lib.rs_static_async_status.argtypes = [vp, ctypes.c_char_p, ctypes.c_size_t]
+    lib.rs_static_async_status.restype = ci
+    lib.rs_linear_uses_tensor_cores.argtypes = [vp, ci, ctypes.c_longlong, ci, ci]
+    lib.rs_linear_uses_tensor_cores.restype = ci
+    lib.rs_block_uses_tensor_cores.argtypes = [vp, ctypes.POINTER(BlockDesc)]
+    lib.rs_block_uses_tensor_cores.restype = ci
     lib.rs_vit_workspace_bytes.argtypes = [ctypes.POINTER(VitDesc), ctypes.POINTER(ci)]
     lib.rs_vit_workspace_bytes.restype = ctypes.c_size_t
     lib.rs_vit_fwd.argtypes = [vp, ctypes.POINTER(VitDesc), ctypes.POINTER(BlockWeights), ctypes.POINTER(ci), vp, vp, vp,
@@ -197,6 +204,12 @@ class Context:
 
     def uses_tensor_cores(self, dtype=torch.bfloat16) -> bool:
         return bool(self.lib.rs_uses_tensor_cores(self.handle, RS_BF16 if dtype == torch.bfloat16 else RS_F32))
+
+    def block_uses_tensor_cores(self, desc: "BlockDesc") -> bool:
+        return bool(self.lib.rs_block_uses_tensor_cores(self.handle, ctypes.byref(desc)))
+
+    def linear_uses_tensor_cores(self, dtype, M: int, N: int, K: int) -> bool:
+        return bool(self.lib.rs_linear_uses_tensor_cores(self.handle, RS_BF16 if dtype == torch.bfloat16 else RS_F32, M, N, K))
 
     def launch_count(self) -> int:
         return int(self.lib.rs_launch_count(self.handle))
@@ -419,6 +432,17 @@ def block_fwd_static(x: torch.Tensor, weights: "DeviceBlockWeights", H: int, r: 
     if want_full:
         res["x_full"] = x_full
     return res
+
+
+def static_async_status(device) -> None:
+    """rs_static_async_status: synchronise the current stream of `device` and raise if a kernel of an
+    earlier block_fwd_static call reported a device-side anomaly."""
+    lib = load_library()
+    err = ctypes.create_string_buffer(512)
+    with torch.cuda.device(device):
+        st = lib.rs_static_async_status(_stream(device), err, 512)
+    if st != RS_OK:
+        raise RsError(st, err.value.decode())
 
 
 class DeviceBlockWeights:

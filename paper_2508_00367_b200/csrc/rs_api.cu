@@ -100,6 +100,8 @@ rs_status rs_create(rs_ctx** out, int device) {
     const char* no_tc = getenv("RS_DISABLE_TC");
     ctx->encode_tiled = rs::tc_get_encode_fn();
     ctx->use_tc = (ctx->encode_tiled != nullptr) && !(no_tc && no_tc[0] == '1');
+    const char* req = getenv("RS_REQUIRE_TC");
+    ctx->require_tc = req && req[0] == '1';
     *out = ctx;
     return RS_OK;
 }
@@ -172,6 +174,17 @@ int rs_uses_tensor_cores(const rs_ctx* ctx, rs_dtype dtype) {
 
 long long rs_launch_count(const rs_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
+int rs_linear_uses_tensor_cores(const rs_ctx* ctx, rs_dtype dtype, long long M, int N, int K) {
+    return ctx && ctx->use_tc && dtype == RS_BF16 && rs::gemm_tc_supported(M, N, K);
+}
+
+int rs_block_uses_tensor_cores(const rs_ctx* ctx, const rs_block_desc* d) {
+    if (!ctx || !d || !ctx->use_tc || d->dtype != RS_BF16 || d->B < 1 || d->N < 1) return 0;
+    const long long T = (long long)d->B * d->N;
+    return rs::gemm_tc_supported(T, 3 * d->D, d->D) && rs::gemm_tc_supported(T, d->D, d->D) &&
+           rs::gemm_tc_supported(T, d->D_mlp, d->D) && rs::gemm_tc_supported(T, d->D, d->D_mlp);
+}
+
 rs_status rs_attn_fwd(rs_ctx* ctx, const rs_attn_desc* d, const void* q, const void* k, const void* v,
                       void* out, void* stream) {
     if (!ctx) return RS_ERR_INVALID_ARG;
@@ -209,6 +222,8 @@ rs_status rs_linear_fwd(rs_ctx* ctx, rs_dtype dtype, rs_linear_epilogue epi, lon
         return fail(ctx, RS_ERR_INVALID_ARG, "rs_linear_fwd: pointers must be 16-byte aligned");
     cudaStream_t st = (cudaStream_t)stream;
     const rs_dtype out_dtype = epi == RS_LIN_BIAS_RESIDUAL ? RS_F32 : dtype;
+    if (ctx->require_tc && dtype == RS_BF16 && !rs_linear_uses_tensor_cores(ctx, dtype, M, N, K))
+        return fail(ctx, RS_ERR_UNSUPPORTED, "rs_linear_fwd: shape outside the tensor-core kernel (N %% 128, K %% 64) and RS_REQUIRE_TC is set");
     if (ctx->use_tc && dtype == RS_BF16 && rs::gemm_tc_supported(M, N, K)) {
         const int e = epi == RS_LIN_BIAS ? rs::RS_EPI_BIAS : epi == RS_LIN_BIAS_GELU ? rs::RS_EPI_BIAS_GELU : rs::RS_EPI_RESID;
         RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_tc(ctx, e, A, W, bias, residual, nullptr, out, out_dtype, nullptr, 0, 0, M, N, K, st), "tensor-core GEMM");
@@ -353,9 +368,9 @@ static rs_status block_fwd_impl(rs_ctx* ctx, const rs_block_desc* d, const rs_bl
     // dropped, else to scratch.
     void* x_hat = x_full ? x_full : (d->r == 0 ? x_out : (void*)(base + ws.x_hat));
 
-    const bool tc = ctx->use_tc && d->dtype == RS_BF16 && rs::gemm_tc_supported(T, 3 * D, D) &&
-                    rs::gemm_tc_supported(T, D, D) && rs::gemm_tc_supported(T, Dm, D) &&
-                    rs::gemm_tc_supported(T, D, Dm);
+    const bool tc = rs_block_uses_tensor_cores(ctx, d) != 0;
+    if (ctx->require_tc && d->dtype == RS_BF16 && !tc)
+        return fail(ctx, RS_ERR_UNSUPPORTED, "rs_block_fwd: shape outside the tensor-core kernels (D, D_mlp multiples of 128) and RS_REQUIRE_TC is set");
     const size_t sz = rs::dtype_size(d->dtype);
     rs_attn_desc ad;
     ad.dtype = d->dtype; ad.B = d->B; ad.N = d->N; ad.H = d->H; ad.head_dim = 64; ad.scale = d->scale;

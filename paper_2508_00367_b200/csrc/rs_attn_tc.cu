@@ -19,6 +19,7 @@
 
 #include "rs_internal.h"
 #include "rs_device.cuh"
+#include "rs_once.h"
 #include "rs_tc.cuh"
 
 namespace rs {
@@ -510,14 +511,16 @@ bool attn_tc_supported(const rs_attn_desc& d) {
 cudaError_t launch_attn_tc(rs_ctx* ctx, const rs_attn_desc& d, const void* q, const void* k, const void* v,
                            void* out, cudaStream_t st) {
     if (!ctx->encode_tiled) return cudaErrorNotSupported;
-    static bool attr_done = false;
-    if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmem);
-        if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(attn_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmem);
-        if (e != cudaSuccess) return e;
-        attr_done = true;
-    }
+    static PerDeviceOnce attr_once;   // the attribute belongs to the device current at the call
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    e = (cudaError_t)attr_once.run(dev, [] {
+        cudaError_t a = cudaFuncSetAttribute(attn_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmem);
+        if (a == cudaSuccess) a = cudaFuncSetAttribute(attn_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmem);
+        return (int)a;
+    });
+    if (e != cudaSuccess) return e;
     CUtensorMap tmQ, tmK, tmV, tmO;
     // out is [B, N, H, 64] contiguous; a softmax warp stores its 32 rows of one head at a time
     if (!make_tmap_qkv(ctx->encode_tiled, &tmO, out, d.B, d.N, d.H, (long long)d.N * d.H * 64, (long long)d.H * 64, 64, 32) ||

@@ -20,6 +20,7 @@
 //                                                          -> bf16/fp32 (FC2 + residual + shift score)
 #include "rs_internal.h"
 #include "rs_device.cuh"
+#include "rs_once.h"
 #include "rs_tc.cuh"
 
 namespace rs {
@@ -453,13 +454,14 @@ template <int BN, int EPI, typename OutT>
 cudaError_t launch_one(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmOut, const CUtensorMap& tmRes,
                        const GemmArgs& args, int sm_count, cudaStream_t st) {
     using C = Cfg<BN, EPI>;
-    static bool attr_done = false;   // per instantiation; the attribute is per function, set once
-    if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<BN, EPI, OutT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)C::SMEM);
-        if (e != cudaSuccess) return e;
-        attr_done = true;
-    }
+    static PerDeviceOnce attr_once;   // per instantiation: the attribute is per function and per device
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    e = (cudaError_t)attr_once.run(dev, [] {
+        return (int)cudaFuncSetAttribute(gemm_tc_kernel<BN, EPI, OutT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM);
+    });
+    if (e != cudaSuccess) return e;
     const int tiles = ((args.M + 2 * BM - 1) / (2 * BM)) * (args.N / BN);
     const int pairs = tiles < sm_count / 2 ? tiles : sm_count / 2;
     cudaLaunchConfig_t cfg = {};

@@ -7,11 +7,13 @@
 #include <stddef.h>
 
 #include "rs.h"
+#include "rs_profile.h"
 
 struct rs_ctx {
     int device;
     int sm_count;
     int use_tc;            // tcgen05 kernels enabled for bf16
+    int require_tc;        // RS_REQUIRE_TC=1: a bf16 shape the tensor-core kernels cannot take is an error
     int* d_status;         // device status word (0 = ok)
     long long launches;    // kernels launched through this context
     void* encode_tiled;    // cuTensorMapEncodeTiled entry point (driver API), or null
@@ -90,7 +92,7 @@ cudaError_t launch_linewise(const float* scores, int B, int H, int W, int Hk, in
                             int32_t* keep_cols, rs_dtype dtype, const void* x, int D, void* x_out, int sm_count,
                             cudaStream_t st);
 size_t select_smem_bytes(int N);
-cudaError_t select_init();   // opt in to large dynamic shared memory once per process/device
+cudaError_t select_init();   // opt in to large dynamic shared memory, once per device (the current one)
 
 // ---- SIMT contraction path (rs_simt.cu): fp32 FMA, used for RS_F32 and as a cross-check ----
 // out[M, N] = act(A[M, K] * W[N, K]^T + bias) + residual.

@@ -121,4 +121,38 @@ rs_status rs_block_fwd_static(const rs_block_desc* desc, const rs_block_weights*
     return st;
 }
 
+rs_status rs_static_async_status(void* stream, char* err, size_t err_len) {
+    cudaError_t e = cudaStreamSynchronize((cudaStream_t)stream);
+    if (e != cudaSuccess) {
+        say(err, err_len, cudaGetErrorString(e));
+        return RS_ERR_CUDA;
+    }
+    int dev = -1;
+    e = cudaGetDevice(&dev);
+    if (e != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+        say(err, err_len, e != cudaSuccess ? cudaGetErrorString(e) : "device index out of range");
+        return RS_ERR_CUDA;
+    }
+    int* status = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_mu);
+        if (!g_ready[dev]) return RS_OK;          // no static call has run on this device yet
+        status = g_status[dev];
+    }
+    int word = 0;
+    e = cudaMemcpy(&word, status, sizeof(int), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) {
+        say(err, err_len, cudaGetErrorString(e));
+        return RS_ERR_CUDA;
+    }
+    if (word == RS_DEV_OK) return RS_OK;
+    cudaMemset(status, 0, sizeof(int));
+    if (word == RS_DEV_SMEM_ALIGN) {
+        say(err, err_len, "rs_block_fwd_static: a kernel's shared memory window was not 1024-byte aligned");
+        return RS_ERR_CUDA;
+    }
+    say(err, err_len, "rs_block_fwd_static: a bounded device-side wait expired");
+    return RS_ERR_TIMEOUT;
+}
+
 }  // extern "C"

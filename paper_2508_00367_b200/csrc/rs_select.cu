@@ -10,6 +10,7 @@
 // no sort.  Integer work only once the keys are formed, hence bit-exact.
 #include "rs_internal.h"
 #include "rs_device.cuh"
+#include "rs_once.h"
 #include <type_traits>
 
 namespace rs {
@@ -464,7 +465,13 @@ linewise_kernel(const float* __restrict__ scores, int H, int W, int Hk, int Wk, 
 size_t select_smem_bytes(int N) { return (size_t)N * sizeof(uint32_t); }
 
 cudaError_t select_init() {
-    return cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 32768 * 4);
+    static PerDeviceOnce once;
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    return (cudaError_t)once.run(dev, [] {
+        return (int)cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 32768 * 4);
+    });
 }
 
 cudaError_t launch_select(const float* scores, int nparts, float* scores_out, int B, int N, int K,

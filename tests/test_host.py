@@ -15,8 +15,11 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
 def _declared():
-    text = open(os.path.join(ROOT, "include", "rs.h")).read()
-    return sorted(set(re.findall(r"RS_API[^;(]*?\b(rs_[a-z_0-9]+)\s*\(", text)))
+    import glob
+    names = set()
+    for h in glob.glob(os.path.join(ROOT, "include", "*.h")):
+        names |= set(re.findall(r"RS_API[^;(]*?\b(rs_[a-z_0-9]+)\s*\(", open(h).read()))
+    return sorted(names)
 
 
 def test_library_builds_and_exports_every_declared_symbol():
@@ -115,6 +118,82 @@ def test_batch_sharding_two_ranks_gloo(tmp_path):
     for p, o in zip(procs, outs):
         assert p.returncode == 0, o
         assert "OK" in o
+
+
+def test_bench_spawns_its_own_ranks(tmp_path):
+    """`bench.py --gpus N` outside torchrun starts N ranks itself: spawn_ranks gives every child its
+    rank and one rendezvous; here two CPU ranks meet over gloo and shard a batch."""
+    sys.path.insert(0, ROOT)
+    import bench
+    script = tmp_path / "worker.py"
+    script.write_text(_WORKER)
+    marks = tmp_path / "ranks"
+    marks.mkdir()
+    wrapper = tmp_path / "wrap.py"
+    wrapper.write_text("import os, sys, runpy\n"
+                       f"open(os.path.join({str(marks)!r}, os.environ['RANK'] + '_' + os.environ['LOCAL_RANK'] + '_' + os.environ['WORLD_SIZE']), 'w').close()\n"
+                       f"sys.argv = [{str(script)!r}, {ROOT!r}]\n"
+                       f"runpy.run_path({str(script)!r}, run_name='__main__')\n")
+    rcs = bench.spawn_ranks(2, [sys.executable, str(wrapper)], timeout=120)
+    assert rcs == [0, 0]
+    assert sorted(os.listdir(marks)) == ["0_0_2", "1_1_2"]
+    # a WORLD_SIZE that contradicts --gpus is an error, not a silent one-rank run
+    env = dict(os.environ, WORLD_SIZE="2", RANK="0", LOCAL_RANK="0")
+    p = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "4", "--impl", "reference"],
+                       env=env, capture_output=True, text=True, timeout=120)
+    assert p.returncode == 2 and "WORLD_SIZE" in p.stderr
+
+
+def test_per_device_once_guard(tmp_path):
+    """Kernel attributes are per device: the guard that sets them runs the set-up once for every
+    device, again after a failure, and never caches an out-of-range device index."""
+    src = tmp_path / "once.cpp"
+    src.write_text(r"""
+#include "rs_once.h"
+#include <thread>
+#include <vector>
+#include <cstdio>
+int main() {
+    rs::PerDeviceOnce once;
+    int calls[3] = {0, 0, 0};
+    for (int rep = 0; rep < 3; ++rep)
+        for (int dev = 0; dev < 2; ++dev)
+            if (once.run(dev, [&] { ++calls[dev]; return 0; }) != 0) return 1;
+    if (calls[0] != 1 || calls[1] != 1) return 2;                 // once per device, not once per process
+    if (!once.done(0) || !once.done(1) || once.done(2)) return 3;
+    int fails = 0;
+    if (once.run(2, [&] { ++fails; return 7; }) != 7) return 4;   // a failed set-up is reported ...
+    if (once.done(2)) return 5;
+    if (once.run(2, [&] { ++calls[2]; return 0; }) != 0 || calls[2] != 1 || !once.done(2)) return 6;   // ... and retried
+    int n = 0;
+    once.run(-1, [&] { ++n; return 0; });
+    once.run(1000, [&] { ++n; return 0; });
+    once.run(1000, [&] { ++n; return 0; });
+    if (n != 3) return 7;                                          // never cached outside the table
+    rs::PerDeviceOnce shared;
+    int hits = 0;
+    std::vector<std::thread> th;
+    for (int t = 0; t < 8; ++t) th.emplace_back([&] { for (int i = 0; i < 1000; ++i) shared.run(5, [&] { ++hits; return 0; }); });
+    for (auto& t : th) t.join();
+    if (hits != 1) return 8;
+    std::puts("ok");
+    return 0;
+}
+""")
+    exe = tmp_path / "once"
+    csrc = os.path.join(ROOT, "paper_2508_00367_b200", "csrc")
+    subprocess.check_call(["g++", "-std=c++17", "-O1", "-pthread", "-I", csrc, "-o", str(exe), str(src)])
+    p = subprocess.run([str(exe)], capture_output=True, text=True)
+    assert p.returncode == 0 and p.stdout.strip() == "ok", (p.returncode, p.stdout)
+
+
+def test_static_status_before_any_static_call_needs_no_gpu_work():
+    """Header contract: arguments are validated on the host; a null descriptor is refused."""
+    from paper_2508_00367_b200 import binding
+    lib = binding.load_library()
+    err = ctypes.create_string_buffer(128)
+    st = lib.rs_block_fwd_static(None, None, None, None, None, None, None, None, err, 128)
+    assert st == 1 and b"null" in err.value
 
 
 def test_gelu_polynomial_matches_exact_erf_gelu():

@@ -39,7 +39,7 @@ def test_static_scratch_block_matches_workspace_block(dtype, B, N, D, H, r):
     want = [ctx.block_fwd(x, dw, H, r, want_full=True) for x in xs]
     got = [rs.block_fwd_static(x, dw, H, r, want_full=True) for x in xs]     # two calls in a row
     got.append(rs.block_fwd_static(xs[0], dw, H, r, want_full=True))         # stale scratch from call 2
-    torch.cuda.synchronize()
+    rs.static_async_status(ctx.device)       # the static kernels' own status word: no bounded wait ran out
     ctx.async_status()
     for g, wnt in zip(got, want + [want[0]]):
         for k in ("x_out", "scores", "keep_idx", "x_full"):
@@ -48,4 +48,28 @@ def test_static_scratch_block_matches_workspace_block(dtype, B, N, D, H, r):
         big = torch.zeros(64, N, D, dtype=tdt, device="cuda")
         rs.block_fwd_static(big, dw, H, r)
     assert e.value.status == 3
+    del big
+    # The property the entry point exists for: the call itself takes no device memory.  Straight
+    # through the C ABI with buffers made beforehand, neither the driver's free-memory figure nor
+    # torch's allocator moves across the call.
+    from paper_2508_00367_b200 import binding
+    lib = binding.load_library()
+    x = xs[1]
+    K = N - r
+    code = binding.RS_BF16 if tdt == torch.bfloat16 else binding.RS_F32
+    desc = binding.BlockDesc(code, code, B, N, D, H, dw.D_mlp, r, 1, 0.0, 0.0, 0, 0)
+    x_out = torch.empty(B, K, D, dtype=tdt, device="cuda")
+    scores = torch.empty(B, N, dtype=torch.float32, device="cuda")
+    keep = torch.empty(B, K, dtype=torch.int32, device="cuda")
+    err = ctypes.create_string_buffer(256)
+    stream = ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    free0, alloc0, reserved0 = torch.cuda.mem_get_info()[0], torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
+    st = lib.rs_block_fwd_static(ctypes.byref(desc), ctypes.byref(dw.struct), x.data_ptr(), x_out.data_ptr(),
+                                 scores.data_ptr(), keep.data_ptr(), None, stream, err, 256)
+    assert st == 0, err.value
+    assert lib.rs_static_async_status(stream, err, 256) == 0, err.value
+    assert torch.cuda.mem_get_info()[0] == free0
+    assert torch.cuda.memory_allocated() == alloc0 and torch.cuda.memory_reserved() == reserved0
+    assert torch.equal(x_out, want[1]["x_out"]) and torch.equal(keep, want[1]["keep_idx"]) and torch.equal(scores, want[1]["scores"])
     ctx.close()
