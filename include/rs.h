@@ -196,8 +196,8 @@ RS_API rs_status rs_block_fwd(rs_ctx* ctx, const rs_block_desc* desc /*host*/,
  * [0, N_l - 1].  x (dev): [B, N, D].  x_out (dev): [B, N_L, D] with N_L = N - sum(drops).
  * scores_last / keep_last (dev, optional): the last block's scores [B, N_{L-1}] and kept
  * indices [B, N_L].  workspace (dev): at least rs_vit_workspace_bytes() bytes, 256-byte
- * aligned; it holds one block's scratch, two token buffers the blocks alternate between and
- * one buffer for the normalised input of the next block. */
+ * aligned; it holds one block's scratch, two token buffers the blocks alternate between, one
+ * buffer for the normalised input of the next block and two row-index lists. */
 typedef struct {
     rs_dtype dtype;
     int B, N, D, H, D_mlp, L;
@@ -219,8 +219,13 @@ typedef struct {
 
 RS_API size_t rs_vit_workspace_bytes(const rs_vit_desc* desc /*host*/, const int* drops /*host[L]*/);
 /* The layer loop with every block's outputs available.  Same computation as rs_vit_fwd.  In both,
- * the compaction kernel of a block that drops tokens also writes LN1 of the next block's input
- * (the kept row is in its registers), so a block after a pruning block launches no LN1 kernel. */
+ * the pruning kernel of a block that drops tokens also writes LN1 of the next block's input
+ * (the kept row is in its registers), so a block after a pruning block launches no LN1 kernel.
+ * The reduced token set of Sec. 3.1 is materialised as a dense [B, N_{l+1}, D] buffer only where a
+ * caller asks for it (taps->x_out[l] non-NULL, and always for the last block): otherwise the
+ * un-pruned output stays where the block wrote it and the next block reads the kept rows in place
+ * through the index list (its LN1 and the residual of its projection), so the copy's
+ * B * N_{l+1} * D elements are never written.  The results are the same bits either way. */
 RS_API rs_status rs_vit_fwd_taps(rs_ctx* ctx, const rs_vit_desc* desc /*host*/,
                                  const rs_block_weights* weights /*host[L]*/, const int* drops /*host[L]*/,
                                  const void* x, const rs_vit_taps* taps /*host*/, void* workspace,

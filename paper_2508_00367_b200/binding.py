@@ -468,9 +468,16 @@ class PrunedViT:
     compacted output; `drops[l]` tokens are removed after block l."""
 
     def __init__(self, ctx: Context, blocks: Sequence[Dict[str, torch.Tensor]], H: int, drops: Sequence[int],
-                 dtype: torch.dtype, has_cls: bool = True, score_mode: str = "mlp", dist: str = "l2"):
+                 dtype: torch.dtype, has_cls: bool = True, score_mode: str = "mlp", dist: str = "l2",
+                 tap_blocks: Optional[Sequence[int]] = None):
+        """tap_blocks: the blocks whose compacted tokens x_out the caller wants (the last block always);
+        None = every block.  A pruning block that is not tapped writes no dense copy of its kept
+        tokens: the next block reads them in place through the index list.  Scores and kept indices
+        are returned for every tapped block and for every block that drops tokens."""
         assert len(blocks) == len(drops)
         self.ctx, self.H, self.drops, self.dtype = ctx, H, list(drops), dtype
+        L = len(self.drops)
+        self.tapped = set(range(L)) if tap_blocks is None else (set(int(b) for b in tap_blocks) | {L - 1})
         self.has_cls, self.score_mode, self.dist = has_cls, score_mode, dist
         self.weights: List[DeviceBlockWeights] = [DeviceBlockWeights(w, dtype, ctx.device) for w in blocks]
         self._plan = None
@@ -483,11 +490,15 @@ class PrunedViT:
         dev = self.ctx.device
         L = len(self.drops)
         outs, n = [], N
-        for r in self.drops:
+        for l, r in enumerate(self.drops):
             k = n - r
-            outs.append(dict(x_out=torch.empty(B, k, D, dtype=self.dtype, device=dev),
-                             scores=torch.empty(B, n, dtype=torch.float32, device=dev),
-                             keep_idx=torch.empty(B, k, dtype=torch.int32, device=dev)))
+            o = {}
+            if l in self.tapped or r > 0:
+                o = dict(scores=torch.empty(B, n, dtype=torch.float32, device=dev),
+                         keep_idx=torch.empty(B, k, dtype=torch.int32, device=dev))
+            if l in self.tapped:
+                o["x_out"] = torch.empty(B, k, D, dtype=self.dtype, device=dev)
+            outs.append(o)
             n = k
         code = RS_BF16 if self.dtype == torch.bfloat16 else RS_F32
         desc = VitDesc(code, B, N, D, self.H, self.weights[0].D_mlp, L, int(self.has_cls), 0.0, 0.0,
@@ -497,7 +508,8 @@ class PrunedViT:
         need = int(self.ctx.lib.rs_vit_workspace_bytes(ctypes.byref(desc), cdrops))
         if need == 0:
             raise RsError(1, "rs_vit_fwd: bad descriptor or schedule")
-        arrs = {k: (ctypes.c_void_p * L)(*[o[k].data_ptr() for o in outs]) for k in ("x_out", "scores", "keep_idx")}
+        arrs = {k: (ctypes.c_void_p * L)(*[(o[k].data_ptr() if k in o else None) for o in outs])
+                for k in ("x_out", "scores", "keep_idx")}
         taps = VitTaps(arrs["x_out"], arrs["scores"], arrs["keep_idx"])
         ws = torch.empty(need, dtype=torch.uint8, device=dev)
         self._plan = dict(key=key, desc=desc, drops=cdrops, warr=warr, arrs=arrs, taps=taps, outs=outs, ws=ws)

@@ -44,7 +44,7 @@ bool valid_dtype(int t) { return t == RS_F32 || t == RS_BF16; }
 
 // Scratch layout of one block.  Every buffer starts on a 256-byte boundary.
 struct BlockWs {
-    size_t u, qkv, o, x_prime, h, m, x_hat, scores, keep, total;
+    size_t u, qkv, o, x_prime, h, m, x_hat, scores, keep, flags, total;
 };
 
 bool block_layout(const rs_block_desc& d, BlockWs* ws) {
@@ -63,6 +63,7 @@ bool block_layout(const rs_block_desc& d, BlockWs* ws) {
     ws->x_hat = take(T * D * osz);       // un-pruned block output when the caller gives no x_full
     ws->scores = take(T * 4);            // when the caller gives no scores buffer
     ws->keep = take((size_t)d.B * (size_t)(d.N) * 4);
+    ws->flags = take(T);                 // keep flags between the ranking kernel and the mover
     ws->total = off;
     return true;
 }
@@ -90,12 +91,13 @@ rs_status rs_create(rs_ctx** out, int device) {
         return RS_ERR_UNSUPPORTED;
     }
     ctx->sm_count = prop.multiProcessorCount;
-    if (cudaMalloc(&ctx->d_status, 256) != cudaSuccess || cudaMemset(ctx->d_status, 0, 256) != cudaSuccess ||
+    if (cudaMalloc(&ctx->d_status, 256 + kFlagScratch) != cudaSuccess || cudaMemset(ctx->d_status, 0, 256) != cudaSuccess ||
         rs::select_init() != cudaSuccess) {
         if (ctx->d_status) cudaFree(ctx->d_status);
         free(ctx);
         return RS_ERR_CUDA;
     }
+    ctx->d_flags = (unsigned char*)ctx->d_status + 256;
     // RS_DISABLE_TC=1 routes bf16 through the fp32-FMA kernels (cross-check of the tcgen05 path).
     const char* no_tc = getenv("RS_DISABLE_TC");
     ctx->encode_tiled = rs::tc_get_encode_fn();
@@ -226,7 +228,7 @@ rs_status rs_linear_fwd(rs_ctx* ctx, rs_dtype dtype, rs_linear_epilogue epi, lon
         return fail(ctx, RS_ERR_UNSUPPORTED, "rs_linear_fwd: shape outside the tensor-core kernel (N %% 128, K %% 64) and RS_REQUIRE_TC is set");
     if (ctx->use_tc && dtype == RS_BF16 && rs::gemm_tc_supported(M, N, K)) {
         const int e = epi == RS_LIN_BIAS ? rs::RS_EPI_BIAS : epi == RS_LIN_BIAS_GELU ? rs::RS_EPI_BIAS_GELU : rs::RS_EPI_RESID;
-        RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_tc(ctx, e, A, W, bias, residual, nullptr, out, out_dtype, nullptr, 0, 0, M, N, K, st), "tensor-core GEMM");
+        RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_tc(ctx, e, A, W, bias, residual, nullptr, nullptr, out, out_dtype, nullptr, 0, 0, M, N, K, st), "tensor-core GEMM");
     } else {
         RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_simt(dtype, A, W, bias, epi == RS_LIN_BIAS_GELU, epi == RS_LIN_BIAS_RESIDUAL ? residual : nullptr, dtype, out, out_dtype, M, N, K, st), "GEMM");
     }
@@ -269,11 +271,14 @@ rs_status rs_topk_compact(rs_ctx* ctx, rs_dtype dtype, int B, int N, int D, int 
         const size_t xbytes = (size_t)B * N * D * sz, obytes = (size_t)B * K * D * sz;
         if (xa < xo + obytes && xo < xa + xbytes) return fail(ctx, RS_ERR_INVALID_ARG, "rs_topk_compact: x_out overlaps x");
     }
-    if (x && rs::select_gather_fusable(N, K)) {
-        RS_CHECK_LAUNCH(ctx, RS_K_GATHER, st, rs::launch_select_gather(scores, 0, nullptr, B, N, K, has_cls ? 1 : 0, keep_idx, dtype, x, D, x_out, nullptr, ctx->sm_count, st), "select+gather launch");
+    int nl = 1;
+    if (x && rs::prune_fusable(N, K, kFlagScratch)) {
+        RS_CHECK_LAUNCH(ctx, RS_K_GATHER, st, rs::launch_prune(scores, 0, nullptr, B, N, K, has_cls ? 1 : 0, keep_idx, nullptr, dtype, x, D, x_out, nullptr, ctx->d_flags, kFlagScratch, ctx->sm_count, st, &nl), "select+gather launch");
+        ctx->launches += nl - 1;
         return RS_OK;
     }
-    RS_CHECK_LAUNCH(ctx, RS_K_SELECT, st, rs::launch_select(scores, 0, nullptr, B, N, K, has_cls ? 1 : 0, keep_idx, st), "select launch");
+    RS_CHECK_LAUNCH(ctx, RS_K_SELECT, st, rs::launch_select(scores, 0, nullptr, B, N, K, has_cls ? 1 : 0, keep_idx, nullptr, ctx->d_flags, kFlagScratch, ctx->sm_count, st, &nl), "select launch");
+    ctx->launches += nl - 1;
     if (x) RS_CHECK_LAUNCH(ctx, RS_K_GATHER, st, rs::launch_gather(dtype, x, keep_idx, B, N, K, D, x_out, nullptr, st), "gather launch");
     return RS_OK;
 }
@@ -314,18 +319,31 @@ rs_status rs_linewise_compact(rs_ctx* ctx, rs_dtype dtype, int B, int H, int W, 
     return RS_OK;
 }
 
-// The block, with the two hooks the layer loop uses to save one kernel per block: `x_ln`, when
-// non-null, is LN1(x) already computed (by the previous block's compaction); `next_ln`, when
-// non-null, asks for LN(x_out) with the next block's LN1 parameters in next_ln->out, written by the
-// compaction kernel.  *ln_done tells whether that happened (it cannot when nothing is dropped, or
-// when a row does not fit one warp's registers): if not, the next block normalises its input itself.
+// What the layer loop adds to a block call.
+//   in_map:  the block input is read in place from the previous block's un-pruned output: row t of
+//            the input is row in_map[t] of `x` ([B, N_prev, D]); null: `x` is the dense [B, N, D] input.
+//   x_ln:    LN1 of the input, already computed by the previous block's pruning kernel; null: not.
+//   next_ln: asks that kernel for LN of this block's kept rows with the next block's LN1 parameters
+//            (it cannot when nothing is dropped or a row does not fit one warp's registers; *ln_done tells).
+//   out_map: where to leave this block's row map (b * N + kept token) for the next block; with it and
+//            dense_out == false the dense copy x_out is not written at all: the next block reads x^
+//            through the map (Sec. 3.1: the reduced token set as an index list).
+struct LoopHooks {
+    const int32_t* in_map;
+    const void* x_ln;
+    const rs::LnFuse* next_ln;
+    int32_t* out_map;
+    bool dense_out;
+    bool* ln_done;
+};
+
 static rs_status block_fwd_impl(rs_ctx* ctx, const rs_block_desc* d, const rs_block_weights* w, const void* x,
-                                const void* x_ln, void* x_out, float* scores, int32_t* keep_idx, void* x_full,
-                                void* workspace, size_t workspace_bytes, void* stream, const rs::LnFuse* next_ln,
-                                bool* ln_done) {
-    if (ln_done) *ln_done = false;
+                                void* x_out, float* scores, int32_t* keep_idx, void* x_full, void* workspace,
+                                size_t workspace_bytes, void* stream, const LoopHooks* hk) {
+    if (hk && hk->ln_done) *hk->ln_done = false;
     if (!ctx) return RS_ERR_INVALID_ARG;
-    if (!d || !w || !x || !x_out) return fail(ctx, RS_ERR_INVALID_ARG, "rs_block_fwd: null argument");
+    const bool dense_out = !hk || hk->dense_out;
+    if (!d || !w || !x || (dense_out && !x_out)) return fail(ctx, RS_ERR_INVALID_ARG, "rs_block_fwd: null argument");
     BlockWs ws;
     if (!block_layout(*d, &ws)) return fail(ctx, RS_ERR_INVALID_ARG, "rs_block_fwd: bad descriptor");
     if (d->H * 64 != d->D) return fail(ctx, RS_ERR_UNSUPPORTED, "rs_block_fwd: D must equal 64 * H");
@@ -371,6 +389,8 @@ static rs_status block_fwd_impl(rs_ctx* ctx, const rs_block_desc* d, const rs_bl
     const bool tc = rs_block_uses_tensor_cores(ctx, d) != 0;
     if (ctx->require_tc && d->dtype == RS_BF16 && !tc)
         return fail(ctx, RS_ERR_UNSUPPORTED, "rs_block_fwd: shape outside the tensor-core kernels (D, D_mlp multiples of 128) and RS_REQUIRE_TC is set");
+    const int32_t* in_map = hk ? hk->in_map : nullptr;
+    if (in_map && !tc) return fail(ctx, RS_ERR_UNSUPPORTED, "rs_block_fwd: a row-mapped input needs the tensor-core kernels");
     const size_t sz = rs::dtype_size(d->dtype);
     rs_attn_desc ad;
     ad.dtype = d->dtype; ad.B = d->B; ad.N = d->N; ad.H = d->H; ad.head_dim = 64; ad.scale = d->scale;
@@ -382,32 +402,33 @@ static rs_status block_fwd_impl(rs_ctx* ctx, const rs_block_desc* d, const rs_bl
     int nparts = 0;
 
     // x' = SA(LN(x)) + x                                                  (Eq. att)
+    const void* x_ln = hk ? hk->x_ln : nullptr;
     if (!x_ln) {
-        RS_CHECK_LAUNCH(ctx, RS_K_LAYERNORM, st, rs::launch_layernorm(d->dtype, d->dtype, x, w->ln1_g, w->ln1_b, eps, T, D, u, st), "LN1");
+        RS_CHECK_LAUNCH(ctx, RS_K_LAYERNORM, st, rs::launch_layernorm(d->dtype, d->dtype, x, w->ln1_g, w->ln1_b, eps, T, D, u, in_map, st), "LN1");
         x_ln = u;
     }
     if (tc) {
-        RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_tc(ctx, rs::RS_EPI_BIAS, x_ln, w->w_qkv, w->b_qkv, nullptr, nullptr, qkv, RS_BF16, nullptr, 0, 0, T, 3 * D, D, st), "QKV");
+        RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_tc(ctx, rs::RS_EPI_BIAS, x_ln, w->w_qkv, w->b_qkv, nullptr, nullptr, nullptr, qkv, RS_BF16, nullptr, 0, 0, T, 3 * D, D, st), "QKV");
         RS_CHECK_LAUNCH(ctx, RS_K_ATTN, st, rs::launch_attn_tc(ctx, ad, qkv, kp, vp, o, st), "attention");
         // shift through attention (operation choice (i)): partial sums of (SA(LN(x)) - x)^2 from this epilogue
         nparts = rs::gemm_tc_score_parts(ctx, T, D);
         float* attn_parts = d->score_mode == RS_SCORE_ATTN ? m : nullptr;
-        RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_tc(ctx, rs::RS_EPI_RESID, o, w->w_o, w->b_o, x, nullptr, x_prime, RS_F32, attn_parts, 0, (int)d->dist, T, D, D, st), "proj");
+        RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_tc(ctx, rs::RS_EPI_RESID, o, w->w_o, w->b_o, x, nullptr, in_map, x_prime, RS_F32, attn_parts, 0, (int)d->dist, T, D, D, st), "proj");
     } else {
         RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_simt(d->dtype, x_ln, w->w_qkv, w->b_qkv, 0, nullptr, RS_F32, qkv, d->dtype, T, 3 * D, D, st), "QKV");
         RS_CHECK_LAUNCH(ctx, RS_K_ATTN, st, rs::launch_attn_simt(ad, qkv, kp, vp, o, st), "attention");
         RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_simt(d->dtype, o, w->w_o, w->b_o, 0, x, d->dtype, x_prime, RS_F32, T, D, D, st), "proj");
     }
     // x^ = MLP(LN(x')) + x',  s = |MLP(LN(x')) - x'|                      (Eq. MLP, Sec. 3.2)
-    RS_CHECK_LAUNCH(ctx, RS_K_LAYERNORM, st, rs::launch_layernorm(RS_F32, d->dtype, x_prime, w->ln2_g, w->ln2_b, eps, T, D, u, st), "LN2");
+    RS_CHECK_LAUNCH(ctx, RS_K_LAYERNORM, st, rs::launch_layernorm(RS_F32, d->dtype, x_prime, w->ln2_g, w->ln2_b, eps, T, D, u, nullptr, st), "LN2");
     if (tc) {
         // The FC2 epilogue adds the residual and leaves per-tile partial sums of squares of the
         // shift in `m`; the selection kernel adds them up in a fixed order.
         // (when the score came from the projection, this epilogue's partial sums go to a second array)
         float* fc2_parts = d->score_mode == RS_SCORE_ATTN ? m + (size_t)T * nparts * 3 : m;
         const int kind = d->score_mode == RS_SCORE_MLP_DELTA ? 1 : d->score_mode == RS_SCORE_BLOCK ? 2 : 0;
-        RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_tc(ctx, rs::RS_EPI_BIAS_GELU, u, w->w_fc1, w->b_fc1, nullptr, nullptr, h, RS_BF16, nullptr, 0, 0, T, Dm, D, st), "FC1");
-        RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_tc(ctx, rs::RS_EPI_SCORE, h, w->w_fc2, w->b_fc2, x_prime, x, x_hat, d->out_dtype, fc2_parts, kind, (int)d->dist, T, D, Dm, st), "FC2+residual+score");
+        RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_tc(ctx, rs::RS_EPI_BIAS_GELU, u, w->w_fc1, w->b_fc1, nullptr, nullptr, nullptr, h, RS_BF16, nullptr, 0, 0, T, Dm, D, st), "FC1");
+        RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_tc(ctx, rs::RS_EPI_SCORE, h, w->w_fc2, w->b_fc2, x_prime, x, in_map, x_hat, d->out_dtype, fc2_parts, kind, (int)d->dist, T, D, Dm, st), "FC2+residual+score");
     } else {
         RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_simt(d->dtype, u, w->w_fc1, w->b_fc1, 1, nullptr, RS_F32, h, d->dtype, T, Dm, D, st), "FC1");
         RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_simt(d->dtype, h, w->w_fc2, w->b_fc2, 0, nullptr, RS_F32, m, RS_F32, T, D, Dm, st), "FC2");
@@ -417,23 +438,32 @@ static rs_status block_fwd_impl(rs_ctx* ctx, const rs_block_desc* d, const rs_bl
     const float* sel_in = nparts > 0 ? m : s;
     const int sel_enc = nparts > 0 ? (nparts | ((int)d->dist << 16)) : 0;
     float* sel_out = nparts > 0 ? s : nullptr;
-    const rs::LnFuse* ln = (next_ln && x_hat != x_out && rs::ln_fusable(d->out_dtype, D)) ? next_ln : nullptr;
-    if (ln && ln_done) *ln_done = true;
-    if (x_hat != x_out && rs::select_gather_fusable(d->N, K)) {
-        RS_CHECK_LAUNCH(ctx, RS_K_GATHER, st, rs::launch_select_gather(sel_in, sel_enc, sel_out, d->B, d->N, K, d->has_cls ? 1 : 0, keep, d->out_dtype, x_hat, D, x_out, ln, ctx->sm_count, st), "select+gather");
+    const bool moves = x_hat != x_out;      // something is dropped: the kept rows are moved (or normalised) here
+    const rs::LnFuse* ln = (hk && hk->next_ln && moves && rs::ln_fusable(d->out_dtype, D)) ? hk->next_ln : nullptr;
+    if (ln && hk->ln_done) *hk->ln_done = true;
+    int32_t* out_map = (hk && moves) ? hk->out_map : nullptr;
+    void* dense = dense_out ? x_out : nullptr;
+    const int cls = d->has_cls ? 1 : 0;
+    uint8_t* flags = (uint8_t*)(base + ws.flags);
+    int nl = 1;
+    if (moves && rs::prune_fusable(d->N, K, (size_t)T) && (dense || ln)) {
+        RS_CHECK_LAUNCH(ctx, RS_K_GATHER, st, rs::launch_prune(sel_in, sel_enc, sel_out, d->B, d->N, K, cls, keep, out_map, d->out_dtype, x_hat, D, dense, ln, flags, (size_t)T, ctx->sm_count, st, &nl), "select+gather");
+        ctx->launches += nl - 1;
         return RS_OK;
     }
-    RS_CHECK_LAUNCH(ctx, RS_K_SELECT, st, rs::launch_select(sel_in, sel_enc, sel_out, d->B, d->N, K, d->has_cls ? 1 : 0, keep, st), "select");
-    if (x_hat != x_out)
-        RS_CHECK_LAUNCH(ctx, RS_K_GATHER, st, rs::launch_gather(d->out_dtype, x_hat, keep, d->B, d->N, K, D, x_out, ln, st), "gather");
+    // nothing dropped and neither the scores nor the (identity) index list asked for: nothing left to do
+    if (!moves && hk && !scores && !keep_idx) return RS_OK;
+    RS_CHECK_LAUNCH(ctx, RS_K_SELECT, st, rs::launch_select(sel_in, sel_enc, sel_out, d->B, d->N, K, cls, keep, out_map, flags, (size_t)T, ctx->sm_count, st, &nl), "select");
+    ctx->launches += nl - 1;
+    if (moves && (dense || ln))
+        RS_CHECK_LAUNCH(ctx, RS_K_GATHER, st, rs::launch_gather(d->out_dtype, x_hat, keep, d->B, d->N, K, D, dense, ln, st), "gather");
     return RS_OK;
 }
 
 rs_status rs_block_fwd(rs_ctx* ctx, const rs_block_desc* d, const rs_block_weights* w, const void* x,
                        void* x_out, float* scores, int32_t* keep_idx, void* x_full, void* workspace,
                        size_t workspace_bytes, void* stream) {
-    return block_fwd_impl(ctx, d, w, x, nullptr, x_out, scores, keep_idx, x_full, workspace, workspace_bytes, stream,
-                          nullptr, nullptr);
+    return block_fwd_impl(ctx, d, w, x, x_out, scores, keep_idx, x_full, workspace, workspace_bytes, stream, nullptr);
 }
 
 }  // extern "C"
@@ -442,7 +472,7 @@ namespace {
 
 // Plan of the layer loop: per-block descriptors, the largest block scratch and the size of one
 // of the two token buffers the blocks alternate between.  False on a bad descriptor / schedule.
-struct VitPlan { size_t block_ws, act_bytes, total; int n_final; };
+struct VitPlan { size_t block_ws, act_bytes, map_bytes, total; int n_final; };
 
 bool vit_plan(const rs_vit_desc& d, const int* drops, VitPlan* p) {
     if (!drops || d.L < 1 || d.B < 1 || d.N < 1) return false;
@@ -458,7 +488,9 @@ bool vit_plan(const rs_vit_desc& d, const int* drops, VitPlan* p) {
     }
     p->block_ws = rs::align_up(block_ws, 256);
     p->act_bytes = rs::align_up((size_t)d.B * d.N * d.D * rs::dtype_size(d.dtype), 256);
-    p->total = p->block_ws + 3 * p->act_bytes;   // block scratch, two token buffers, one LN buffer
+    p->map_bytes = rs::align_up((size_t)d.B * d.N * sizeof(int32_t), 256);
+    // block scratch, two token buffers, one LN buffer, two row maps
+    p->total = p->block_ws + 3 * p->act_bytes + 2 * p->map_bytes;
     p->n_final = n;
     return true;
 }
@@ -488,24 +520,33 @@ rs_status rs_vit_fwd_taps(rs_ctx* ctx, const rs_vit_desc* d, const rs_block_weig
         return fail(ctx, RS_ERR_INVALID_ARG, "rs_vit_fwd: workspace must be 256-byte aligned");
     char* base = (char*)workspace;
     void* act[2] = {base + p.block_ws, base + p.block_ws + p.act_bytes};
-    void* ln_buf = base + p.block_ws + 2 * p.act_bytes;   // LN1 of the next block's input, from the compaction
+    void* ln_buf = base + p.block_ws + 2 * p.act_bytes;   // LN1 of the next block's input, from the pruning kernel
+    int32_t* maps[2] = {(int32_t*)(base + p.block_ws + 3 * p.act_bytes), (int32_t*)(base + p.block_ws + 3 * p.act_bytes + p.map_bytes)};
     const float eps = d->ln_eps > 0.f ? d->ln_eps : 1e-6f;
-    const void* cur = x;
+    const void* cur = x;                 // the block input: dense [B, n, D], or, with cur_map, the previous
+    const int32_t* cur_map = nullptr;    // block's un-pruned x^ read through the row map
     const void* cur_ln = nullptr;
     int n = d->N;
     for (int l = 0; l < d->L; ++l) {
         const bool last = l == d->L - 1;
         rs_block_desc bd = {d->dtype, d->dtype, d->B, n, d->D, d->H, d->D_mlp, drops[l], d->has_cls, d->ln_eps, d->scale,
                             d->score_mode, d->dist};
-        void* out = taps->x_out[l] ? taps->x_out[l] : act[l & 1];
-        // LN1 of block l+1 rides in this block's compaction: one kernel less per block
+        // A block that drops tokens and whose compacted output nobody asked for writes no dense copy:
+        // its un-pruned x^ stays in a token buffer and the next block reads the kept rows in place
+        // (LN1 in the pruning kernel or through the map, the projection's residual through the map).
+        const bool in_place = !last && drops[l] > 0 && !taps->x_out[l] && rs_block_uses_tensor_cores(ctx, &bd);
+        void* out = in_place ? nullptr : (taps->x_out[l] ? taps->x_out[l] : act[l & 1]);
+        // LN1 of block l+1 rides in this block's pruning kernel: one kernel less per block
         const rs::LnFuse next = {last ? nullptr : weights[l + 1].ln1_g, last ? nullptr : weights[l + 1].ln1_b, eps, ln_buf};
         bool ln_done = false;
-        rs_status st = block_fwd_impl(ctx, &bd, &weights[l], cur, cur_ln, out, taps->scores ? taps->scores[l] : nullptr,
-                                      taps->keep_idx ? taps->keep_idx[l] : nullptr, nullptr, base, p.block_ws, stream,
-                                      (last || !next.gamma || !next.beta) ? nullptr : &next, &ln_done);
+        const LoopHooks hk = {cur_map, cur_ln, (last || !next.gamma || !next.beta) ? nullptr : &next,
+                              in_place ? maps[l & 1] : nullptr, !in_place, &ln_done};
+        rs_status st = block_fwd_impl(ctx, &bd, &weights[l], cur, out, taps->scores ? taps->scores[l] : nullptr,
+                                      taps->keep_idx ? taps->keep_idx[l] : nullptr, in_place ? act[l & 1] : nullptr, base,
+                                      p.block_ws, stream, &hk);
         if (st != RS_OK) return st;
-        cur = out;
+        cur = in_place ? act[l & 1] : out;
+        cur_map = in_place ? maps[l & 1] : nullptr;
         cur_ln = ln_done ? ln_buf : nullptr;
         n -= drops[l];
     }

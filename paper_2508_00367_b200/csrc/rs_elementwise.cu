@@ -17,7 +17,8 @@ constexpr int kWarpsPerCta = 8;
 template <typename TI, typename TO, int MAXV>
 __global__ void __launch_bounds__(kWarpsPerCta * 32, MAXV <= 4 ? 5 : 4)
 layernorm_kernel(const TI* __restrict__ x, const float* __restrict__ gamma,
-                 const float* __restrict__ beta, float eps, long long T, int D, TO* __restrict__ out) {
+                 const float* __restrict__ beta, float eps, long long T, int D, TO* __restrict__ out,
+                 const int32_t* __restrict__ row_map) {
     constexpr int VN = Vec16<TI>::N;
     grid_dep_launch();
     grid_dep_wait();
@@ -25,7 +26,8 @@ layernorm_kernel(const TI* __restrict__ x, const float* __restrict__ gamma,
     const long long row = (long long)blockIdx.x * kWarpsPerCta + (threadIdx.x >> 5);
     if (row >= T) return;
     const int nvec = D / VN;
-    const uint4* xr = reinterpret_cast<const uint4*>(x + row * D);
+    const long long src = row_map ? (long long)row_map[row] : row;
+    const uint4* xr = reinterpret_cast<const uint4*>(x + src * D);
     uint4 raw[MAXV];
 #pragma unroll
     for (int j = 0; j < MAXV; ++j) {
@@ -141,13 +143,13 @@ inline unsigned row_grid(long long rows) { return (unsigned)((rows + kWarpsPerCt
 
 template <typename TI, typename TO>
 cudaError_t ln_dispatch(const void* x, const float* g, const float* b, float eps, long long T, int D,
-                        void* out, cudaStream_t st) {
+                        void* out, const int32_t* row_map, cudaStream_t st) {
     const int nvec = D / Vec16<TI>::N;
     const dim3 grid(row_grid(T)), block(kWarpsPerCta * 32);
     if (nvec <= 32 * 4)
-        return launch_pdl(layernorm_kernel<TI, TO, 4>, grid, block, 0, st, (const TI*)x, g, b, eps, T, D, (TO*)out);
+        return launch_pdl(layernorm_kernel<TI, TO, 4>, grid, block, 0, st, (const TI*)x, g, b, eps, T, D, (TO*)out, row_map);
     else if (nvec <= 32 * 8)
-        return launch_pdl(layernorm_kernel<TI, TO, 8>, grid, block, 0, st, (const TI*)x, g, b, eps, T, D, (TO*)out);
+        return launch_pdl(layernorm_kernel<TI, TO, 8>, grid, block, 0, st, (const TI*)x, g, b, eps, T, D, (TO*)out, row_map);
     return cudaErrorInvalidValue;
 }
 
@@ -155,12 +157,12 @@ cudaError_t ln_dispatch(const void* x, const float* g, const float* b, float eps
 
 cudaError_t launch_layernorm(rs_dtype in_dtype, rs_dtype out_dtype, const void* x, const float* gamma,
                              const float* beta, float eps, long long T, int D, void* out,
-                             cudaStream_t st) {
+                             const int32_t* row_map, cudaStream_t st) {
     if (T == 0) return cudaSuccess;
-    if (in_dtype == RS_F32 && out_dtype == RS_F32) return ln_dispatch<float, float>(x, gamma, beta, eps, T, D, out, st);
-    if (in_dtype == RS_F32 && out_dtype == RS_BF16) return ln_dispatch<float, __nv_bfloat16>(x, gamma, beta, eps, T, D, out, st);
-    if (in_dtype == RS_BF16 && out_dtype == RS_BF16) return ln_dispatch<__nv_bfloat16, __nv_bfloat16>(x, gamma, beta, eps, T, D, out, st);
-    return ln_dispatch<__nv_bfloat16, float>(x, gamma, beta, eps, T, D, out, st);
+    if (in_dtype == RS_F32 && out_dtype == RS_F32) return ln_dispatch<float, float>(x, gamma, beta, eps, T, D, out, row_map, st);
+    if (in_dtype == RS_F32 && out_dtype == RS_BF16) return ln_dispatch<float, __nv_bfloat16>(x, gamma, beta, eps, T, D, out, row_map, st);
+    if (in_dtype == RS_BF16 && out_dtype == RS_BF16) return ln_dispatch<__nv_bfloat16, __nv_bfloat16>(x, gamma, beta, eps, T, D, out, row_map, st);
+    return ln_dispatch<__nv_bfloat16, float>(x, gamma, beta, eps, T, D, out, row_map, st);
 }
 
 cudaError_t launch_shift_score(rs_dtype dtype, rs_dist dist, long long T, int D, const void* after,

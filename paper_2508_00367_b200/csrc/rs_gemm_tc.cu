@@ -65,6 +65,8 @@ struct GemmArgs {
     const float* bias;        // [N] or null
     const void* residual;     // EPI_RESID: bf16 [M, N];  EPI_SCORE: fp32 [M, N]
     const void* residual2;    // EPI_SCORE, score_kind 2: bf16 [M, N] block input x
+    const int* row_map;       // optional [M]: row t of the block input (EPI_RESID's residual, EPI_SCORE's residual2)
+                              // is row row_map[t] of that matrix (the previous block's un-pruned output, read in place)
     float* partials;          // EPI_SCORE (and EPI_RESID when non-null): [M, 2 * N / BN] sums of squares
     int score_kind;           // EPI_SCORE: scored pair (u, v) = 0: (m, x'), 1: (x^, x'), 2: (x^, x)
     int dist;                 // rs_dist of the score: L2 / L1 sums of (u - v)^2 / |u - v|, cosine sums of u.v, u.u, v.v
@@ -139,7 +141,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         for (int a = 0; a < 2; ++a) { mbar_init(&tfull[a], 1); mbar_init(&tempty[a], 2 * kEpiWarps); }
         if (C::RES_TMA) {
             prefetch_tmap(&tmRes);
-            for (int w = 0; w < kEpiWarps; ++w) mbar_init(&res_full[w], 1);
+            // one arrival by the lane that starts the TMA copies, or one by each lane's own indexed copies
+            for (int w = 0; w < kEpiWarps; ++w) mbar_init(&res_full[w], args.row_map ? 32 : 1);
         }
         *abort_flag = 0;
         half_fail[0] = 0;
@@ -236,13 +239,35 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             for (int c = c_begin; c < c_end; c += 32)
                 tma_load_2d(res_buf + ((c - c_begin) / 32) * RES_BOX_BYTES, &tmRes, &res_full[warp - 2], rn0 + c, rm0);
         };
-        if (C::RES_TMA && lane == 0 && pair < tiles) issue_res(pair);
+        // The same boxes filled row by row through the row map: lane l looks up the source row of the
+        // warp's row l; 16-byte asynchronous copies, a row's pieces by neighbouring lanes, land in the
+        // layout the tensor map's 64-byte swizzle would give; rows past M are zero-filled.
+        auto issue_res_mapped = [&](int tile) {      // whole warp
+            const int rm0 = (tile / num_n) * (2 * BM) + (int)rank * BM + q * 32, rn0 = (tile % num_n) * BN;
+            const int src_row = rm0 + lane < args.M ? __ldg(args.row_map + rm0 + lane) : -1;
+            const int ppr = (c_end - c_begin) / 8, total = 32 * ppr;          // 16-byte pieces per row
+            const __nv_bfloat16* base = reinterpret_cast<const __nv_bfloat16*>(args.residual) + rn0 + c_begin;
+            for (int idx = lane; idx < total; idx += 32) {
+                const int r = idx / ppr, piece = idx - r * ppr;
+                const int sr = __shfl_sync(0xffffffffu, src_row, r);
+                const uint32_t dst = smem_u32(res_buf + (piece >> 2) * RES_BOX_BYTES + r * 64 + (((piece & 3) ^ ((r >> 1) & 3)) << 4));
+                const __nv_bfloat16* src = base + (size_t)(sr < 0 ? 0 : sr) * args.N + piece * 8;
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(sr < 0 ? 0 : 16) : "memory");
+            }
+            asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(&res_full[warp - 2])) : "memory");
+        };
+        if (C::RES_TMA && pair < tiles) {
+            if (args.row_map) issue_res_mapped(pair);
+            else if (lane == 0) issue_res(pair);
+        }
         constexpr int RES_VECS = EPI == EPI_RESID ? 4 : EPI == EPI_SCORE ? 8 : 1;   // 16-byte loads per 32 columns
         for (int tile = pair; tile < tiles; tile += npairs, ++tl) {
             const int m0 = (tile / num_n) * (2 * BM) + (int)rank * BM, nt = tile % num_n, n0 = nt * BN;
             const uint32_t a = tl & 1u, aph = (tl >> 1) & 1u;
             const int row = m0 + trow;
             const bool valid = row < args.M;
+            // row of the block input x (EPI_SCORE, whole-block shift), possibly through the row map
+            const int xrow = (EPI == EPI_SCORE && args.score_kind == 2 && args.row_map && valid) ? __ldg(args.row_map + row) : row;
             // Residual values of 32 columns of this thread's row (zeros for rows past M).  They are
             // fetched one chunk ahead, the first chunk before the accumulator is even complete.
             auto load_res = [&](int c, uint4* dst) {
@@ -331,7 +356,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     if (args.score_kind == 2) {
                         // whole-block shift: x^ - x, with the block input x read here (rows past M: zeros)
                         const uint4* x0p = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(args.residual2) +
-                                                                          (size_t)row * args.N + col);
+                                                                          (size_t)xrow * args.N + col);
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
                             const uint4 xv = valid ? __ldg(x0p + j) : make_uint4(0u, 0u, 0u, 0u);
@@ -393,7 +418,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             }
             if (C::RES_TMA) {
                 __syncwarp();                            // every lane has read its residual rows
-                if (lane == 0 && tile + npairs < tiles) issue_res(tile + npairs);
+                if (tile + npairs < tiles) {
+                    if (args.row_map) issue_res_mapped(tile + npairs);
+                    else if (lane == 0) issue_res(tile + npairs);
+                }
             }
             if ((EPI == EPI_SCORE || (EPI == EPI_RESID && args.partials)) && valid) {
                 const size_t pi = (size_t)row * (2 * num_n) + 2 * nt + half;
@@ -519,21 +547,21 @@ int gemm_tc_score_parts(const rs_ctx* ctx, long long M, int N) {
 }
 
 cudaError_t launch_gemm_tc(rs_ctx* ctx, int epi, const void* A, const void* W, const float* bias,
-                           const void* residual, const void* residual2, void* out, rs_dtype out_dtype, float* partials, int score_kind, int dist,
-                           long long M, int N, int K, cudaStream_t st) {
+                           const void* residual, const void* residual2, const int32_t* row_map, void* out, rs_dtype out_dtype,
+                           float* partials, int score_kind, int dist, long long M, int N, int K, cudaStream_t st) {
     if (!ctx->encode_tiled) return cudaErrorNotSupported;
     const int bn = pick_bn(M, N, ctx->sm_count);
     const int out_bytes = (epi == EPI_RESID || (epi == EPI_SCORE && out_dtype == RS_F32)) ? 4 : 2;
     CUtensorMap tmA, tmB, tmOut, tmRes;
-    if (epi == EPI_RESID && !make_tmap_res(ctx->encode_tiled, &tmRes, residual, (uint64_t)M, (uint64_t)N)) return cudaErrorInvalidValue;
+    if (epi == EPI_RESID && !row_map && !make_tmap_res(ctx->encode_tiled, &tmRes, residual, (uint64_t)M, (uint64_t)N)) return cudaErrorInvalidValue;
     if (!make_tmap_2d(ctx->encode_tiled, &tmA, A, 2, (uint64_t)M, (uint64_t)K, BM) ||
         !make_tmap_2d(ctx->encode_tiled, &tmB, W, 2, (uint64_t)N, (uint64_t)K, (uint32_t)(bn / 2)) ||
         !make_tmap_2d(ctx->encode_tiled, &tmOut, out, out_bytes, (uint64_t)M, (uint64_t)N, 32))
         return cudaErrorInvalidValue;
-    if (epi != EPI_RESID) tmRes = tmOut;             // unused by the other epilogues
+    if (epi != EPI_RESID || row_map) tmRes = tmOut;  // unused by the other epilogues and by the mapped residual
     GemmArgs args;
     args.M = (int)M; args.N = N; args.K = K; args.bias = bias; args.residual = residual;
-    args.residual2 = residual2; args.partials = partials; args.score_kind = score_kind; args.dist = dist; args.status = ctx->d_status;
+    args.residual2 = residual2; args.row_map = row_map; args.partials = partials; args.score_kind = score_kind; args.dist = dist; args.status = ctx->d_status;
     const int sms = ctx->sm_count;
 #define RS_GEMM_CASE(E, T)                                                                       \
     return bn == 256   ? launch_one<256, E, T>(tmA, tmB, tmOut, tmRes, args, sms, st)           \

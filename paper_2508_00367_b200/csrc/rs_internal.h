@@ -14,7 +14,8 @@ struct rs_ctx {
     int sm_count;
     int use_tc;            // tcgen05 kernels enabled for bf16
     int require_tc;        // RS_REQUIRE_TC=1: a bf16 shape the tensor-core kernels cannot take is an error
-    int* d_status;         // device status word (0 = ok)
+    int* d_status;         // device status word (0 = ok), first bytes of a small allocation made by rs_create
+    unsigned char* d_flags; // keep-flag scratch of rs_topk_compact (kFlagScratch bytes, same allocation)
     long long launches;    // kernels launched through this context
     void* encode_tiled;    // cuTensorMapEncodeTiled entry point (driver API), or null
     int timing;            // bracket launches with events
@@ -25,6 +26,7 @@ struct rs_ctx {
 };
 
 enum { kMaxTimed = 8192 };
+enum { kFlagScratch = 1 << 20 };
 
 // Device status word values.
 enum { RS_DEV_OK = 0, RS_DEV_TIMEOUT = 1, RS_DEV_SMEM_ALIGN = 2 };
@@ -55,9 +57,10 @@ inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 // ---- memory-bound kernels (rs_elementwise.cu) ----
 // LayerNorm over the last dimension: x [T, D] (in_dtype) -> out [T, D] (out_dtype); fp32 math.
+// row_map (optional, [T] int32): output row t normalises input row row_map[t] instead of row t.
 cudaError_t launch_layernorm(rs_dtype in_dtype, rs_dtype out_dtype, const void* x, const float* gamma,
                              const float* beta, float eps, long long T, int D, void* out,
-                             cudaStream_t st);
+                             const int32_t* row_map, cudaStream_t st);
 // s[t] = D(after[t,:], before[t,:]).
 cudaError_t launch_shift_score(rs_dtype dtype, rs_dist dist, long long T, int D, const void* after,
                                const void* before, float* scores, cudaStream_t st);
@@ -72,19 +75,29 @@ cudaError_t launch_residual_score(const float* m, const float* x_prime, const vo
 // scores: [B, N] fp32; or, if nparts > 0, the per-tile partial sums a GEMM epilogue left
 // (nparts = tiles | rs_dist << 16; [B*N, tiles] sums, three per tile for the cosine distance),
 // from which the score is finished here (and written to scores_out when non-null).
+// row_map (optional, [B, K] int32): flat source row b * N + keep_idx[b, j] of every kept token, with
+// which the next block reads the un-pruned rows in place.
+// flags / flags_bytes: scratch for the keep flags of sequences longer than 256 tokens (N bytes per
+// sample; with less than B * N the batch is processed in several passes, with less than N the radix
+// kernel runs instead).  *launches (optional) receives the number of kernels launched.
 cudaError_t launch_select(const float* scores, int nparts, float* scores_out, int B, int N, int K,
-                          int has_cls, int32_t* keep_idx, cudaStream_t st);
+                          int has_cls, int32_t* keep_idx, int32_t* row_map, uint8_t* flags, size_t flags_bytes,
+                          int sm_count, cudaStream_t st, int* launches);
 // The compaction kernels can also write LN(x_out) for the block that follows (its LN1 of Eq. att):
 // the warp that copies a kept row has it in registers.  out: [B, K, D] of the rows' dtype.
 struct LnFuse { const float* gamma; const float* beta; float eps; void* out; };
 bool ln_fusable(rs_dtype dtype, int D);   // the row fits the registers of one warp
+// x_out may be null when ln is given: only the normalised rows are written (no dense copy).
 cudaError_t launch_gather(rs_dtype dtype, const void* x, const int32_t* keep_idx, int B, int N, int K,
                           int D, void* x_out, const LnFuse* ln /*null: none*/, cudaStream_t st);
-// Selection and compaction in one kernel (N <= 1024 and something is dropped).
-bool select_gather_fusable(int N, int K);
-cudaError_t launch_select_gather(const float* scores, int nparts, float* scores_out, int B, int N, int K, int has_cls,
-                                 int32_t* keep_idx, rs_dtype dtype, const void* x, int D, void* x_out,
-                                 const LnFuse* ln /*null: none*/, int sm_count, cudaStream_t st);
+// Selection, index lists and the rows' move (N <= 4608 and something is dropped): one kernel up to
+// 256 tokens, a ranking kernel spread over the grid plus the mover beyond.
+// x null: indices only.  x given: x_out (dense copy) and / or ln (normalised rows) must be given.
+bool prune_fusable(int N, int K, size_t flags_bytes);
+cudaError_t launch_prune(const float* scores, int nparts, float* scores_out, int B, int N, int K, int has_cls,
+                         int32_t* keep_idx, int32_t* row_map, rs_dtype dtype, const void* x, int D, void* x_out,
+                         const LnFuse* ln /*null: none*/, uint8_t* flags, size_t flags_bytes, int sm_count,
+                         cudaStream_t st, int* launches);
 // Line-wise pruning of a 2-D token grid: keep_rows [B, Hk], keep_cols [B, Wk] and, when x is given,
 // x_out[b, i, j, :] = x[b, keep_rows[b, i], keep_cols[b, j], :].  H, W <= linewise_max_lines().
 int linewise_max_lines();
@@ -108,9 +121,12 @@ void* tc_get_encode_fn();                       // cuTensorMapEncodeTiled via th
 bool gemm_tc_supported(long long M, int N, int K);
 int gemm_tc_score_parts(const rs_ctx* ctx, long long M, int N);   // partial sums per row written by RS_EPI_SCORE
 // out[M, N] = epilogue(A[M, K] . W[N, K]^T); see rs_gemm_tc.cu for the epilogues.
+// row_map (optional, [M] int32): row t of the block input (the bf16 residual of RS_EPI_RESID, residual2
+// of RS_EPI_SCORE) is row row_map[t] of the given matrix -- the un-pruned output of the previous block.
 cudaError_t launch_gemm_tc(rs_ctx* ctx, int epi, const void* A, const void* W, const float* bias,
-                           const void* residual, const void* residual2, void* out, rs_dtype out_dtype,
-                           float* partials, int score_kind, int dist, long long M, int N, int K, cudaStream_t st);
+                           const void* residual, const void* residual2, const int32_t* row_map, void* out,
+                           rs_dtype out_dtype, float* partials, int score_kind, int dist, long long M, int N, int K,
+                           cudaStream_t st);
 
 // ---- tcgen05 attention (rs_attn_tc.cu): bf16, head dimension 64 ----
 bool attn_tc_supported(const rs_attn_desc& d);

@@ -1,6 +1,6 @@
 // Per-sample selection of the K = N - r highest-score tokens and compaction of
-// the kept rows (Sec. 3.1 reduced token set; Sec. 3.2 "dropped the tokens
-// having the lowest k scores").
+// the kept rows (Sec. 3.1: the reduced token set; Sec. 3.2: the r lowest-score
+// tokens are removed).
 //
 // Selection is exact and order-stable.  fp32 scores are mapped to uint32 keys
 // that sort like the floats (NaN lowest).  A 4-pass, 8-bit radix select finds
@@ -74,7 +74,7 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int* wsum, int* total
 
 __global__ void __launch_bounds__(kSelThreads)
 select_kernel(const float* __restrict__ scores, int nparts, float* __restrict__ scores_out, int N,
-              int K, int has_cls, int32_t* __restrict__ keep_idx) {
+              int K, int has_cls, int32_t* __restrict__ keep_idx, int32_t* __restrict__ row_map) {
     extern __shared__ uint32_t keys[];     // [N]
     __shared__ int hist[256];
     __shared__ int wsum[32];
@@ -167,69 +167,23 @@ select_kernel(const float* __restrict__ scores, int nparts, float* __restrict__ 
     int pos = block_exclusive_scan(kept, wsum, &sh_total);
     int32_t* out = keep_idx + (long long)b * K;
     for (int i = lo; i < hi; ++i)
-        if (keys[i]) { if (pos < K) out[pos] = i; ++pos; }
+        if (keys[i]) {
+            if (pos < K) {
+                out[pos] = i;
+                if (row_map) row_map[(long long)b * K + pos] = b * N + i;
+            }
+            ++pos;
+        }
 }
 
-// Selection for N <= 1024: one token per thread, rank by counting.  Token i outranks token j
-// iff key_i > key_j, or the keys are equal and i < j (the same order the radix path realises),
-// so rank_i = #{j : j outranks i} and the K - first best-ranked candidates are kept.  N broadcast
-// reads of shared memory per thread replace the four histogram passes and their barriers: at
-// ViT token counts this is latency, not work.
-__global__ void __launch_bounds__(1024)
-select_small_kernel(const float* __restrict__ scores, int nparts, float* __restrict__ scores_out, int N,
-                    int K, int has_cls, int32_t* __restrict__ keep_idx) {
-    __shared__ uint32_t keys[1024];
-    __shared__ int wsum[32];
-    __shared__ int sh_total;
-    grid_dep_launch();
-    grid_dep_wait();
-    const int b = blockIdx.x, i = threadIdx.x;
-    const int first = has_cls ? 1 : 0, want = K - first;
-    uint32_t key = 0;
-    if (i < N) {
-        float s;
-        if (nparts > 0) {                  // per-tile partial sums from the GEMM epilogue
-            s = finish_score(scores + ((long long)b * N + i) * partial_stride(nparts), nparts);
-            if (scores_out) scores_out[(long long)b * N + i] = s;
-        } else {
-            s = scores[(long long)b * N + i];
-        }
-        key = score_key(s);
-        keys[i] = key;
-    }
-    __syncthreads();
-    int keep = 0;
-    if (i < N) {
-        if (i < first) {
-            keep = 1;
-        } else if (want > 0) {
-            int rank = 0;
-            int j = first;
-            for (; j + 4 <= N; j += 4) {   // keys[j] is a broadcast read: every thread reads the same word
-                const uint32_t k0 = keys[j], k1 = keys[j + 1], k2 = keys[j + 2], k3 = keys[j + 3];
-                rank += (k0 > key) || (k0 == key && j < i);
-                rank += (k1 > key) || (k1 == key && j + 1 < i);
-                rank += (k2 > key) || (k2 == key && j + 2 < i);
-                rank += (k3 > key) || (k3 == key && j + 3 < i);
-            }
-            for (; j < N; ++j) {
-                const uint32_t k0 = keys[j];
-                rank += (k0 > key) || (k0 == key && j < i);
-            }
-            keep = rank < want;
-        }
-    }
-    const int pos = block_exclusive_scan(keep, wsum, &sh_total);
-    if (keep && pos < K) keep_idx[(long long)b * K + pos] = i;
-}
-
-// One warp copies one kept row (16-byte pieces, all loads of a pass issued before its first store)
-// to row `orow` of x_out and, with LT given, writes LN of the row to the same row of ln.out.
+// One warp moves one kept row (16-byte pieces, all loads of a pass issued before its first store):
+// to row `orow` of x_out when x_out is given, and, with LT given, LN of the row to the same row of
+// ln.out.
 template <int MAXV, typename LT>
 __device__ __forceinline__ void copy_row(const uint4* __restrict__ src, long long orow, int row_vecs, int lane,
                                          uint4* __restrict__ x_out, const LnFuse& ln) {
-    uint4* dst = x_out + orow * row_vecs;
     if constexpr (std::is_void<LT>::value) {
+        uint4* dst = x_out + orow * row_vecs;
         for (int base = 0; base < row_vecs; base += 32 * MAXV) {
             uint4 v[MAXV];
 #pragma unroll
@@ -250,81 +204,143 @@ __device__ __forceinline__ void copy_row(const uint4* __restrict__ src, long lon
             const int iv = j * 32 + lane;
             if (iv < row_vecs) v[j] = __ldg(src + iv);
         }
+        if (x_out) {
+            uint4* dst = x_out + orow * row_vecs;
 #pragma unroll
-        for (int j = 0; j < MAXV; ++j) {
-            const int iv = j * 32 + lane;
-            if (iv < row_vecs) dst[iv] = v[j];
+            for (int j = 0; j < MAXV; ++j) {
+                const int iv = j * 32 + lane;
+                if (iv < row_vecs) dst[iv] = v[j];
+            }
         }
         const int D = row_vecs * Vec16<LT>::N;
         layernorm_row<LT, LT, MAXV>(v, row_vecs, lane, ln.gamma, ln.beta, ln.eps, D, reinterpret_cast<LT*>(ln.out) + orow * D);
     }
 }
 
-// Selection and compaction in one launch for N <= 1024.  Grid (G, B): every CTA of sample b
-// repeats the (cheap) counting selection of select_small_kernel, so no CTA waits for another;
-// CTA 0 of the sample writes the index list (and the finished scores), and each CTA copies its
-// share of the kept rows, a warp per row, all 16-byte loads of a row before its stores.
-// LT: void, or the rows' element type when LN of every written row goes to ln.out as well (the
-// whole row then sits in one warp's registers: row_vecs <= 32 * MAXV).
-template <int MAXV, typename LT>
+// Selection by counting, and what follows it, for N <= kPruneMaxN tokens.  Token i outranks j iff
+// key_i > key_j, or the keys are equal and i < j (the order the radix path realises too); its rank
+// is the number of tokens that outrank it, and the K - first best-ranked candidates are kept.
+// Integer work only once the keys are formed, hence bit-exact.
+constexpr int kPruneMaxN = 4608;
+constexpr int kFusedMaxN = 256;      // up to here every mover CTA repeats the (short) ranking itself
+
+struct PruneArgs {
+    const float* scores; int nparts; float* scores_out;
+    int N, K, has_cls, b0;            // b0: index of the grid's first sample in the whole batch (row_map is global)
+    const uint8_t* flags_in;         // keep flags from rank_kernel ([B, N]), or null: rank here
+    int32_t* keep_idx; int32_t* row_map;
+    const uint4* x; int row_vecs; uint4* x_out;
+    LnFuse ln;
+};
+
+// Forms the N orderable keys of sample b in shared memory (finishing the scores from the GEMM's
+// partial sums when they arrive that way); the scores of tokens [w0, w1) are also written out.
+__device__ __forceinline__ void load_keys(const float* scores, int nparts, float* scores_out, int b, int N, int w0, int w1,
+                                          uint32_t* keys) {
+    for (int i = threadIdx.x; i < N; i += blockDim.x) {
+        float s;
+        if (nparts > 0) {
+            s = finish_score(scores + ((long long)b * N + i) * partial_stride(nparts), nparts);
+            if (scores_out && i >= w0 && i < w1) scores_out[(long long)b * N + i] = s;
+        } else {
+            s = scores[(long long)b * N + i];
+        }
+        keys[i] = score_key(s);
+    }
+}
+
+// Keep flag of tokens [i0, i0 + P) of a sample whose keys are in shared memory: S threads (a power
+// of two, a group inside a warp) per token, each counting over a strided share of the N keys.
+template <typename Put>
+__device__ __forceinline__ void rank_slice(const uint32_t* keys, int N, int K, int first, int i0, int P, Put put) {
+    const int nt = blockDim.x, tid = threadIdx.x, want = K - first;
+    int S = 1;
+    while (S < 32 && 2 * S * P <= nt) S <<= 1;
+    const int sub = tid & (S - 1), per_pass = nt / S;
+    for (int base = 0; base < P; base += per_pass) {
+        const int t = base + tid / S, i = i0 + t;
+        const bool act = t < P && i < N;
+        int rank = 0;
+        if (act && i >= first && want > 0) {
+            const uint32_t key = keys[i];
+            for (int j = first + sub; j < N; j += S) {
+                const uint32_t k = keys[j];
+                rank += (k > key) || (k == key && j < i);
+            }
+        }
+        for (int o = S >> 1; o > 0; o >>= 1) rank += __shfl_xor_sync(0xffffffffu, rank, o);
+        if (act && sub == 0) put(i, (uint8_t)(i < first ? 1 : (want > 0 && rank < want) ? 1 : 0));
+    }
+}
+
+// Ranking spread over the grid: CTA (g, b) ranks tokens [g P, (g+1) P) of sample b against all N
+// and leaves their keep flags in global memory; N^2 / P comparisons per CTA instead of N^2.
 __global__ void __launch_bounds__(1024)
-select_gather_small_kernel(const float* __restrict__ scores, int nparts, float* __restrict__ scores_out, int N,
-                           int K, int has_cls, int32_t* __restrict__ keep_idx, const uint4* __restrict__ x,
-                           int row_vecs, uint4* __restrict__ x_out, const LnFuse ln) {
-    __shared__ uint32_t keys[1024];
-    __shared__ int32_t kept[1024];
+rank_kernel(const float* __restrict__ scores, int nparts, float* __restrict__ scores_out, int N, int K, int has_cls,
+            int P, uint8_t* __restrict__ flags) {
+    __shared__ uint32_t keys[kPruneMaxN];
+    grid_dep_launch();
+    grid_dep_wait();
+    const int b = blockIdx.y, i0 = blockIdx.x * P;
+    load_keys(scores, nparts, scores_out, b, N, i0, i0 + P, keys);
+    __syncthreads();
+    uint8_t* fb = flags + (long long)b * N;
+    rank_slice(keys, N, K, has_cls ? 1 : 0, i0, P, [&](int i, uint8_t f) { fb[i] = f; });
+}
+
+// The kept tokens' index lists and rows.  Grid (G, B).  Every CTA of sample b gets the sample's N
+// keep flags -- from rank_kernel, or, for short sequences, by ranking all tokens itself (cheaper
+// than a second launch up to kFusedMaxN tokens) -- and scans them into the ascending list of kept
+// tokens; CTA 0 of the sample writes keep_idx, the flat source-row list row_map (b N + token: what
+// the next block uses to read the un-pruned x^ in place) and, when it ranked, the finished scores.
+// Then CTA g moves its share of the K kept rows, a warp per row: the dense copy x_out when one is
+// wanted, and, with LT given, LN of the row for the next block (the whole row then sits in one
+// warp's registers: row_vecs <= 32 * MAXV).
+template <int MAXV, typename LT>
+__global__ void __launch_bounds__(512)
+prune_kernel(const PruneArgs a) {
+    __shared__ uint32_t keys[kPruneMaxN];       // keys (when ranking here), then the list of kept tokens
+    __shared__ uint8_t flags[kPruneMaxN];
     __shared__ int wsum[32];
     __shared__ int sh_total;
     grid_dep_launch();
     grid_dep_wait();
-    const int b = blockIdx.y, i = threadIdx.x;
-    const int first = has_cls ? 1 : 0, want = K - first;
-    uint32_t key = 0;
-    if (i < N) {
-        float s;
-        if (nparts > 0) {                  // per-tile partial sums from the GEMM epilogue
-            s = finish_score(scores + ((long long)b * N + i) * partial_stride(nparts), nparts);
-            if (scores_out && blockIdx.x == 0) scores_out[(long long)b * N + i] = s;
-        } else {
-            s = scores[(long long)b * N + i];
-        }
-        key = score_key(s);
-        keys[i] = key;
+    const int b = blockIdx.y, tid = threadIdx.x, nt = blockDim.x, N = a.N, K = a.K;
+    if (a.flags_in) {
+        const uint8_t* fb = a.flags_in + (long long)b * N;
+        for (int i = tid; i < N; i += nt) flags[i] = fb[i];
+    } else {
+        load_keys(a.scores, a.nparts, blockIdx.x == 0 ? a.scores_out : nullptr, b, N, 0, N, keys);
+        __syncthreads();
+        rank_slice(keys, N, K, a.has_cls ? 1 : 0, 0, N, [&](int i, uint8_t f) { flags[i] = f; });
     }
     __syncthreads();
-    int keep = 0;
-    if (i < N) {
-        if (i < first) {
-            keep = 1;
-        } else if (want > 0) {
-            int rank = 0;
-            int j = first;
-            for (; j + 4 <= N; j += 4) {   // keys[j] is a broadcast read: every thread reads the same word
-                const uint32_t k0 = keys[j], k1 = keys[j + 1], k2 = keys[j + 2], k3 = keys[j + 3];
-                rank += (k0 > key) || (k0 == key && j < i);
-                rank += (k1 > key) || (k1 == key && j + 1 < i);
-                rank += (k2 > key) || (k2 == key && j + 2 < i);
-                rank += (k3 > key) || (k3 == key && j + 3 < i);
+    // ---- ascending list of kept tokens ----
+    const int chunk = (N + nt - 1) / nt;
+    const int lo_t = min(tid * chunk, N), hi_t = min(lo_t + chunk, N);
+    int cnt = 0;
+    for (int i = lo_t; i < hi_t; ++i) cnt += flags[i];
+    int pos = block_exclusive_scan(cnt, wsum, &sh_total);
+    int32_t* kept = reinterpret_cast<int32_t*>(keys);
+    for (int i = lo_t; i < hi_t; ++i)
+        if (flags[i]) {
+            if (pos < K) {
+                kept[pos] = i;
+                if (blockIdx.x == 0) {
+                    a.keep_idx[(long long)b * K + pos] = i;
+                    if (a.row_map) a.row_map[(long long)b * K + pos] = (a.b0 + b) * N + i;
+                }
             }
-            for (; j < N; ++j) {
-                const uint32_t k0 = keys[j];
-                rank += (k0 > key) || (k0 == key && j < i);
-            }
-            keep = rank < want;
+            ++pos;
         }
-    }
-    const int pos = block_exclusive_scan(keep, wsum, &sh_total);
-    if (keep && pos < K) {
-        kept[pos] = i;
-        if (blockIdx.x == 0) keep_idx[(long long)b * K + pos] = i;
-    }
     __syncthreads();
-    // rows [lo, hi) of the sample's K kept rows belong to this CTA
+    if (!a.x) return;
+    // ---- rows [lo, hi) of the sample's K kept rows belong to this CTA ----
     const int G = gridDim.x, per = (K + G - 1) / G;
     const int lo = blockIdx.x * per, hi = min(lo + per, K);
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    const int lane = tid & 31, warp = tid >> 5, nwarps = nt >> 5;
     for (int r = lo + warp; r < hi; r += nwarps)
-        copy_row<MAXV, LT>(x + ((long long)b * N + kept[r]) * row_vecs, (long long)b * K + r, row_vecs, lane, x_out, ln);
+        copy_row<MAXV, LT>(a.x + ((long long)b * N + kept[r]) * a.row_vecs, (long long)b * K + r, a.row_vecs, lane, a.x_out, a.ln);
 }
 
 // Nothing dropped (K == N): every token is kept, in order; only the scores remain to be
@@ -475,43 +491,78 @@ cudaError_t select_init() {
 }
 
 cudaError_t launch_select(const float* scores, int nparts, float* scores_out, int B, int N, int K,
-                          int has_cls, int32_t* keep_idx, cudaStream_t st) {
+                          int has_cls, int32_t* keep_idx, int32_t* row_map, uint8_t* flags, size_t flags_bytes,
+                          int sm_count, cudaStream_t st, int* launches) {
+    if (launches) *launches = 1;
     if (B == 0) return cudaSuccess;
     if (K == N) {
         const long long T = (long long)B * N;
         return launch_pdl(keep_all_kernel, dim3((unsigned)((T + 255) / 256)), dim3(256), 0, st, scores, nparts, scores_out, T, N, keep_idx);
     }
-    if (N <= 1024) {
-        return launch_pdl(select_small_kernel, dim3(B), dim3((N + 31) / 32 * 32), 0, st, scores, nparts, scores_out, N, K, has_cls, keep_idx);
-    }
+    if (N <= kPruneMaxN && (N <= kFusedMaxN || flags_bytes >= (size_t)N))
+        return launch_prune(scores, nparts, scores_out, B, N, K, has_cls, keep_idx, row_map, RS_F32, nullptr, 0, nullptr, nullptr,
+                            flags, flags_bytes, sm_count, st, launches);
     return launch_pdl(select_kernel, dim3(B), dim3(kSelThreads), select_smem_bytes(N), st, scores, nparts, scores_out, N, K,
-                      has_cls, keep_idx);
+                      has_cls, keep_idx, row_map);
 }
 
-bool select_gather_fusable(int N, int K) { return N <= 1024 && K < N; }
+bool prune_fusable(int N, int K, size_t flags_bytes) {
+    return N <= kPruneMaxN && K < N && (N <= kFusedMaxN || flags_bytes >= (size_t)N);
+}
 
 bool ln_fusable(rs_dtype dtype, int D) { return (size_t)D * dtype_size(dtype) / 16 <= 32 * 4; }
 
-cudaError_t launch_select_gather(const float* scores, int nparts, float* scores_out, int B, int N, int K, int has_cls,
-                                 int32_t* keep_idx, rs_dtype dtype, const void* x, int D, void* x_out,
-                                 const LnFuse* ln, int sm_count, cudaStream_t st) {
+cudaError_t launch_prune(const float* scores, int nparts, float* scores_out, int B, int N, int K, int has_cls,
+                         int32_t* keep_idx, int32_t* row_map, rs_dtype dtype, const void* x, int D, void* x_out,
+                         const LnFuse* ln, uint8_t* flags, size_t flags_bytes, int sm_count, cudaStream_t st, int* launches) {
+    if (launches) *launches = 0;
     if (B == 0) return cudaSuccess;
-    const int row_vecs = (int)((size_t)D * dtype_size(dtype) / 16);
-    // enough CTAs per sample for about three waves over the SMs (six when a row is also normalised
-    // and the selection every CTA repeats is short: measured), at least a few rows each
-    int G = ((ln && N <= 256 ? 6 : 3) * sm_count + B - 1) / B;
-    G = G < 1 ? 1 : G;
-    if (G > (K + 3) / 4) G = (K + 3) / 4;
-    if (G < 1) G = 1;
-    const dim3 grid(G, B), block((N + 31) / 32 * 32 < 128 ? 128 : (N + 31) / 32 * 32);
-    if (ln && !ln_fusable(dtype, D)) return cudaErrorInvalidValue;
-    const LnFuse none = {nullptr, nullptr, 0.f, nullptr};
-#define RS_SG_CASE(LT)                                                                                                  \
-    launch_pdl(select_gather_small_kernel<4, LT>, grid, block, 0, st, scores, nparts, scores_out, N, K, has_cls, keep_idx, \
-               (const uint4*)x, row_vecs, (uint4*)x_out, ln ? *ln : none)
-    if (!ln) return RS_SG_CASE(void);
-    return dtype == RS_BF16 ? RS_SG_CASE(__nv_bfloat16) : RS_SG_CASE(float);
-#undef RS_SG_CASE
+    const bool two_step = N > kFusedMaxN;
+    if (N > kPruneMaxN || (ln && !ln_fusable(dtype, D)) || (x && !x_out && !ln) || (two_step && flags_bytes < (size_t)N))
+        return cudaErrorInvalidValue;
+    const int row_vecs = x ? (int)((size_t)D * dtype_size(dtype) / 16) : 0;
+    const size_t sz = dtype_size(dtype);
+    // samples per pass: as many as the flag scratch holds (all of them, unless the batch is huge)
+    const int Bc = two_step ? (int)((flags_bytes / (size_t)N) < (size_t)B ? flags_bytes / (size_t)N : (size_t)B) : B;
+    for (int b0 = 0; b0 < B; b0 += Bc) {
+        const int nb = B - b0 < Bc ? B - b0 : Bc;
+        const long long t0 = (long long)b0 * N, k0 = (long long)b0 * K;
+        const float* sc = scores + t0 * (nparts > 0 ? (nparts & 0xffff) * ((nparts >> 16) == RS_DIST_COS ? 3 : 1) : 1);
+        float* so = scores_out ? scores_out + t0 : nullptr;
+        if (two_step) {
+            // tokens per ranking CTA: 64 (4 threads each) up to 1024 tokens, else 128 (8 threads each)
+            const int P = N <= 1024 ? 64 : 128, nt = N <= 1024 ? 256 : 1024;
+            cudaError_t e = launch_pdl(rank_kernel, dim3((N + P - 1) / P, nb), dim3(nt), 0, st, sc, nparts, so, N, K, has_cls, P, flags);
+            if (e != cudaSuccess) return e;
+            if (launches) *launches += 1;
+        }
+        // mover CTAs per sample: about three waves over the SMs (six when a row is also normalised
+        // and the sequence is short: measured), a few rows each; one CTA for the index lists alone
+        int G = 1;
+        if (x) {
+            G = ((ln && N <= 256 ? 6 : 3) * sm_count + nb - 1) / nb;
+            if (G > (K + 3) / 4) G = (K + 3) / 4;
+            if (G < 1) G = 1;
+        }
+        const int nt = N <= 128 ? 128 : 256;
+        PruneArgs a;
+        a.scores = sc; a.nparts = nparts; a.scores_out = so; a.N = N; a.K = K; a.has_cls = has_cls; a.b0 = b0;
+        a.flags_in = two_step ? flags : nullptr;
+        a.keep_idx = keep_idx + k0; a.row_map = row_map ? row_map + k0 : nullptr;
+        a.x = x ? (const uint4*)((const char*)x + (size_t)t0 * D * sz) : nullptr;
+        a.row_vecs = row_vecs;
+        a.x_out = x_out ? (uint4*)((char*)x_out + (size_t)k0 * D * sz) : nullptr;
+        a.ln = ln ? *ln : LnFuse{nullptr, nullptr, 0.f, nullptr};
+        if (ln) a.ln.out = (char*)ln->out + (size_t)k0 * D * sz;
+        cudaError_t e;
+        const dim3 grid(G, nb), block(nt);
+        if (!ln) e = launch_pdl(prune_kernel<4, void>, grid, block, 0, st, a);
+        else if (dtype == RS_BF16) e = launch_pdl(prune_kernel<4, __nv_bfloat16>, grid, block, 0, st, a);
+        else e = launch_pdl(prune_kernel<4, float>, grid, block, 0, st, a);
+        if (e != cudaSuccess) return e;
+        if (launches) *launches += 1;
+    }
+    return cudaSuccess;
 }
 
 cudaError_t launch_gather(rs_dtype dtype, const void* x, const int32_t* keep_idx, int B, int N, int K,
@@ -520,7 +571,7 @@ cudaError_t launch_gather(rs_dtype dtype, const void* x, const int32_t* keep_idx
     if (rows == 0) return cudaSuccess;
     const int row_vecs = (int)((size_t)D * dtype_size(dtype) / 16);
     const unsigned grid = (unsigned)((rows + 7) / 8);
-    if (ln && !ln_fusable(dtype, D)) return cudaErrorInvalidValue;
+    if ((ln && !ln_fusable(dtype, D)) || (!x_out && !ln)) return cudaErrorInvalidValue;
     const LnFuse none = {nullptr, nullptr, 0.f, nullptr};
 #define RS_G_CASE(LT)                                                                                               \
     launch_pdl(gather_kernel<4, LT>, dim3(grid), dim3(256), 0, st, (const uint4*)x, keep_idx, rows, N, K, row_vecs, \

@@ -323,3 +323,30 @@ def test_vit_fwd_equals_the_block_loop(ctx, B, N, D, H, drops, dt):
     with pytest.raises(rs.RsError):
         ctx.vit_fwd(x, model.weights, H, drops[:-1] + [N])       # the last block cannot drop all its tokens
     ctx.async_status()
+
+
+@pytest.mark.parametrize("mode,dist", [("block", "l2"), ("attn", "cos"), ("mlp_delta", "l1")])
+def test_vit_fwd_in_place_pruning_other_scores(ctx, mode, dist):
+    """A pruning block whose compacted tokens nobody asks for writes no dense copy: the next block
+    reads the kept rows of the un-pruned output through the index list (LN1, the projection's
+    residual and, for the whole-block shift, the FC2 epilogue's second residual).  Same bits as
+    chaining rs_block_fwd, for the operation choices and distances of Sec. 3.3 that read the block
+    input in an epilogue."""
+    import paper_2508_00367_b200 as rs
+    B, N, D, H, drops = 3, 333, 256, 4, [40, 33, 0, 50, 7]
+    x = synth.make_tokens(B, N, D, "bf16", seed=81).to(torch.bfloat16).cuda()
+    blocks = [synth.make_block_weights(D, 4 * D, "bf16", seed=90 + l) for l in range(len(drops))]
+    weights = [rs.DeviceBlockWeights(w, torch.bfloat16, ctx.device) for w in blocks]
+    chain, cur = [], x
+    for l, r in enumerate(drops):
+        o = ctx.block_fwd(cur, weights[l], H, r, score_mode=mode, dist=dist)
+        chain.append(o)
+        cur = o["x_out"]
+    got = ctx.vit_fwd(x, weights, H, drops, score_mode=mode, dist=dist)          # only the last block is materialised
+    some = ctx.vit_fwd_taps(x, weights, H, drops, tap_blocks=[2], score_mode=mode, dist=dist)
+    torch.cuda.synchronize()
+    for k in ("x_out", "scores", "keep_idx"):
+        assert torch.equal(got[k], chain[-1][k]), k
+        assert torch.equal(some[2][k], chain[2][k]), k
+        assert torch.equal(some[4][k], chain[4][k]), k
+    ctx.async_status()

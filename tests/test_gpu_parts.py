@@ -133,6 +133,21 @@ def test_topk_compact_full_size_and_guard_bands(ctx):
     assert (ki_buf[:pad] == -77).all() and (ki_buf[-pad:] == -77).all()
 
 
+def test_topk_compact_batch_larger_than_the_flag_scratch(ctx):
+    """Sequences over 256 tokens are ranked by one kernel and moved by another, with a byte per token
+    in between; a batch with more tokens than that scratch holds (1 MiB) runs in several passes."""
+    B, N, D, r = 2100, 520, 8, 100
+    s = _scores(B, N, "ties", 21)
+    x = _tok((B, N, D), torch.float32, 22)
+    xo, keep = ctx.topk_compact(torch.from_numpy(s).cuda(), x.cuda(), r, True)
+    want = orc.topk(s.astype(np.float64), r, True)
+    np.testing.assert_array_equal(keep.cpu().numpy(), want)
+    for b in (0, 1, 2015, 2016, 2017, B - 1):          # both sides of the pass boundary (2016 samples fit)
+        assert torch.equal(xo[b].cpu(), x[b][torch.from_numpy(want[b]).long()])
+    _, keep2 = ctx.topk_compact(torch.from_numpy(s).cuda(), None, r, False)          # indices only
+    np.testing.assert_array_equal(keep2.cpu().numpy(), orc.topk(s.astype(np.float64), r, False))
+
+
 def test_topk_indices_only_and_errors(ctx):
     s = torch.from_numpy(_scores(2, 50, "normal", 1)).cuda()
     _, keep = ctx.topk_compact(s, None, 10, True)
