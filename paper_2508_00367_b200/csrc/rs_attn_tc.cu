@@ -17,6 +17,10 @@
 // next item and the epilogue of the previous one overlap across item boundaries.
 #include <math.h>
 
+#include <map>
+#include <mutex>
+#include <tuple>
+
 #include "rs_internal.h"
 #include "rs_device.cuh"
 #include "rs_once.h"
@@ -48,6 +52,9 @@ struct AttnArgs {
     int dual;                // 1: N <= 128, an item is two heads; 0: an item is two query tiles of one head
     int per;                 // items per (sample, head) [dual = 0] or per sample [dual = 1]
     int n_items;
+    // dual = 0: the first n_pair_items items are pairs of query tiles; the rest are single query tiles,
+    // tile_count of them for each (sample, head) from first_single_bh on (see launch_attn_tc)
+    int n_pair_items, first_single_bh, tile_count;
     float scale_log2;        // scale * log2(e)
     int* status;
 };
@@ -70,11 +77,20 @@ __device__ __forceinline__ Item decode_item(const AttnArgs& a, int w) {
         it.nkv = 1;
         it.slots = it.ng;
     } else {
-        const int qp = w % a.per, bh = w / a.per;
+        int bh;
+        if (w < a.n_pair_items) {
+            const int qp = w % a.per;
+            bh = w / a.per;
+            it.q0[0] = qp * 2 * BQ; it.q0[1] = it.q0[0] + BQ;
+            it.ng = it.q0[1] < a.N ? 2 : 1;
+        } else {
+            const int k = w - a.n_pair_items;
+            bh = a.first_single_bh + k / a.tile_count;
+            it.q0[0] = (k % a.tile_count) * BQ; it.q0[1] = a.N;       // one query tile only
+            it.ng = 1;
+        }
         it.b = bh / a.H;
         it.h[0] = it.h[1] = bh % a.H;
-        it.q0[0] = qp * 2 * BQ; it.q0[1] = it.q0[0] + BQ;
-        it.ng = it.q0[1] < a.N ? 2 : 1;
         it.nkv = (a.N + BKV - 1) / BKV;
         it.slots = it.nkv;
     }
@@ -533,8 +549,52 @@ cudaError_t launch_attn_tc(rs_ctx* ctx, const rs_attn_desc& d, const void* q, co
     args.N = d.N; args.H = d.H;
     args.dual = d.N <= BQ ? 1 : 0;
     args.per = args.dual ? (d.H + 1) / 2 : (d.N + 2 * BQ - 1) / (2 * BQ);
-    const long long items = (long long)args.per * (args.dual ? d.B : (long long)d.B * d.H);
-    if (items >= (1ll << 31)) return cudaErrorInvalidValue;
+    long long items = (long long)args.per * (args.dual ? d.B : (long long)d.B * d.H);
+    if (items >= (1ll << 30)) return cudaErrorInvalidValue;
+    args.n_pair_items = (int)items; args.first_single_bh = d.B * d.H; args.tile_count = (d.N + BQ - 1) / BQ;
+    if (!args.dual) {
+        // Items go to the CTAs round robin, and a pair of query tiles costs twice a single one, so a
+        // last round with few pairs left keeps most SMs idle for a whole pair's time.  The tiles of the
+        // last few (sample, head)s are therefore handed out one by one where that shortens the longest
+        // CTA: the count is the one with the smallest makespan under the cost model pair = 10, single = 7
+        // (a query tile alone runs faster than next to another, but not twice as fast: measured).
+        const long long BH = (long long)d.B * d.H;
+        const int G = ctx->sm_count, nt = args.tile_count, per = args.per;
+        auto makespan = [&](long long hs) {
+            const long long pair_items = (BH - hs) * per, singles = hs * nt, all = pair_items + singles;
+            long long worst = 0;
+            for (int c = 0; c < G && c < all; ++c) {          // CTA c takes items c, c + G, ...
+                long long load = 0;
+                for (long long w = c; w < all; w += G)
+                    load += w < pair_items ? (((w % per) == per - 1 && (nt & 1)) ? 7 : 10) : 7;
+                if (load > worst) worst = load;
+            }
+            return worst;
+        };
+        // (a host loop over the items for every candidate: the answer is remembered per shape)
+        static std::mutex memo_mu;
+        static std::map<std::tuple<long long, int, int>, long long> memo;
+        long long best_hs = 0, best = -1;
+        const auto key = std::make_tuple(BH, d.N, G);
+        std::unique_lock<std::mutex> lock(memo_mu);
+        const auto hit = memo.find(key);
+        if (hit != memo.end()) {
+            best_hs = hit->second;
+        } else {
+            long long hs_max = (2ll * G + nt - 1) / nt + 1;    // enough single tiles for two rounds
+            if (hs_max > BH) hs_max = BH;
+            if (BH * per <= 200000)
+                for (long long hs = 0; hs <= hs_max; ++hs) {
+                    const long long m = makespan(hs);
+                    if (best < 0 || m < best) { best = m; best_hs = hs; }
+                }
+            memo[key] = best_hs;
+        }
+        lock.unlock();
+        args.n_pair_items = (int)((BH - best_hs) * per);
+        args.first_single_bh = (int)(BH - best_hs);
+        items = (BH - best_hs) * per + best_hs * nt;
+    }
     args.n_items = (int)items;
     const float scale = d.scale != 0.f ? d.scale : 0.125f;
     args.scale_log2 = scale * 1.4426950408889634f;
