@@ -63,7 +63,7 @@ bool block_layout(const rs_block_desc& d, BlockWs* ws) {
     ws->x_hat = take(T * D * osz);       // un-pruned block output when the caller gives no x_full
     ws->scores = take(T * 4);            // when the caller gives no scores buffer
     ws->keep = take((size_t)d.B * (size_t)(d.N) * 4);
-    ws->flags = take(T);                 // keep flags between the ranking kernel and the mover
+    ws->flags = take(T + 4 * (T / 64 + 2 * (size_t)d.B) + 16);   // slice counts and keep flags between the ranking kernel and the mover
     ws->total = off;
     return true;
 }
@@ -445,15 +445,16 @@ static rs_status block_fwd_impl(rs_ctx* ctx, const rs_block_desc* d, const rs_bl
     void* dense = dense_out ? x_out : nullptr;
     const int cls = d->has_cls ? 1 : 0;
     uint8_t* flags = (uint8_t*)(base + ws.flags);
+    const size_t flags_bytes = (size_t)T + 4 * ((size_t)T / 64 + 2 * (size_t)d->B) + 16;
     int nl = 1;
-    if (moves && rs::prune_fusable(d->N, K, (size_t)T) && (dense || ln)) {
-        RS_CHECK_LAUNCH(ctx, RS_K_GATHER, st, rs::launch_prune(sel_in, sel_enc, sel_out, d->B, d->N, K, cls, keep, out_map, d->out_dtype, x_hat, D, dense, ln, flags, (size_t)T, ctx->sm_count, st, &nl), "select+gather");
+    if (moves && rs::prune_fusable(d->N, K, flags_bytes) && (dense || ln)) {
+        RS_CHECK_LAUNCH(ctx, RS_K_GATHER, st, rs::launch_prune(sel_in, sel_enc, sel_out, d->B, d->N, K, cls, keep, out_map, d->out_dtype, x_hat, D, dense, ln, flags, flags_bytes, ctx->sm_count, st, &nl), "select+gather");
         ctx->launches += nl - 1;
         return RS_OK;
     }
     // nothing dropped and neither the scores nor the (identity) index list asked for: nothing left to do
     if (!moves && hk && !scores && !keep_idx) return RS_OK;
-    RS_CHECK_LAUNCH(ctx, RS_K_SELECT, st, rs::launch_select(sel_in, sel_enc, sel_out, d->B, d->N, K, cls, keep, out_map, flags, (size_t)T, ctx->sm_count, st, &nl), "select");
+    RS_CHECK_LAUNCH(ctx, RS_K_SELECT, st, rs::launch_select(sel_in, sel_enc, sel_out, d->B, d->N, K, cls, keep, out_map, flags, flags_bytes, ctx->sm_count, st, &nl), "select");
     ctx->launches += nl - 1;
     if (moves && (dense || ln))
         RS_CHECK_LAUNCH(ctx, RS_K_GATHER, st, rs::launch_gather(d->out_dtype, x_hat, keep, d->B, d->N, K, D, dense, ln, st), "gather");

@@ -220,18 +220,11 @@ __device__ __forceinline__ void copy_row(const uint4* __restrict__ src, long lon
 // Selection by counting, and what follows it, for N <= kPruneMaxN tokens.  Token i outranks j iff
 // key_i > key_j, or the keys are equal and i < j (the order the radix path realises too); its rank
 // is the number of tokens that outrank it, and the K - first best-ranked candidates are kept.
-// Integer work only once the keys are formed, hence bit-exact.
+// Integer work only once the keys are formed, hence bit-exact.  Two kernels: rank_kernel spreads the
+// N^2 comparisons of a sample over N / P CTAs and leaves a keep flag per token and a kept count per
+// slice; gather_ranked_kernel gives every kept row a warp, which finds its token from the counts and
+// flags, writes the index lists and moves the row.
 constexpr int kPruneMaxN = 4608;
-constexpr int kFusedMaxN = 256;      // up to here every mover CTA repeats the (short) ranking itself
-
-struct PruneArgs {
-    const float* scores; int nparts; float* scores_out;
-    int N, K, has_cls, b0;            // b0: index of the grid's first sample in the whole batch (row_map is global)
-    const uint8_t* flags_in;         // keep flags from rank_kernel ([B, N]), or null: rank here
-    int32_t* keep_idx; int32_t* row_map;
-    const uint4* x; int row_vecs; uint4* x_out;
-    LnFuse ln;
-};
 
 // Forms the N orderable keys of sample b in shared memory (finishing the scores from the GEMM's
 // partial sums when they arrive that way); the scores of tokens [w0, w1) are also written out.
@@ -250,7 +243,8 @@ __device__ __forceinline__ void load_keys(const float* scores, int nparts, float
 }
 
 // Keep flag of tokens [i0, i0 + P) of a sample whose keys are in shared memory: S threads (a power
-// of two, a group inside a warp) per token, each counting over a strided share of the N keys.
+// of two, a group inside a warp) per token, each counting over a strided share of the N keys.  A
+// token before i outranks it on a tie, a token after it does not: two loops, one comparison each.
 template <typename Put>
 __device__ __forceinline__ void rank_slice(const uint32_t* keys, int N, int K, int first, int i0, int P, Put put) {
     const int nt = blockDim.x, tid = threadIdx.x, want = K - first;
@@ -263,10 +257,10 @@ __device__ __forceinline__ void rank_slice(const uint32_t* keys, int N, int K, i
         int rank = 0;
         if (act && i >= first && want > 0) {
             const uint32_t key = keys[i];
-            for (int j = first + sub; j < N; j += S) {
-                const uint32_t k = keys[j];
-                rank += (k > key) || (k == key && j < i);
-            }
+            for (int j = first + sub; j < i; j += S) rank += keys[j] >= key;
+            // first index of this thread's stride past i
+            int j = i + 1 + ((sub - (i + 1 - first)) & (S - 1));
+            for (; j < N; j += S) rank += keys[j] > key;
         }
         for (int o = S >> 1; o > 0; o >>= 1) rank += __shfl_xor_sync(0xffffffffu, rank, o);
         if (act && sub == 0) put(i, (uint8_t)(i < first ? 1 : (want > 0 && rank < want) ? 1 : 0));
@@ -275,72 +269,77 @@ __device__ __forceinline__ void rank_slice(const uint32_t* keys, int N, int K, i
 
 // Ranking spread over the grid: CTA (g, b) ranks tokens [g P, (g+1) P) of sample b against all N
 // and leaves their keep flags in global memory; N^2 / P comparisons per CTA instead of N^2.
+// It also leaves the number of kept tokens of its slice in counts[b, g]: with those, whoever moves
+// the rows finds the token behind an output position without scanning the sample.
 __global__ void __launch_bounds__(1024)
 rank_kernel(const float* __restrict__ scores, int nparts, float* __restrict__ scores_out, int N, int K, int has_cls,
-            int P, uint8_t* __restrict__ flags) {
+            int P, uint8_t* __restrict__ flags, int32_t* __restrict__ counts) {
     __shared__ uint32_t keys[kPruneMaxN];
+    __shared__ int kept_here;
     grid_dep_launch();
     grid_dep_wait();
     const int b = blockIdx.y, i0 = blockIdx.x * P;
+    if (threadIdx.x == 0) kept_here = 0;
     load_keys(scores, nparts, scores_out, b, N, i0, i0 + P, keys);
     __syncthreads();
     uint8_t* fb = flags + (long long)b * N;
-    rank_slice(keys, N, K, has_cls ? 1 : 0, i0, P, [&](int i, uint8_t f) { fb[i] = f; });
+    rank_slice(keys, N, K, has_cls ? 1 : 0, i0, P, [&](int i, uint8_t f) { fb[i] = f; if (f) atomicAdd(&kept_here, 1); });
+    __syncthreads();
+    if (threadIdx.x == 0) counts[(long long)b * gridDim.x + blockIdx.x] = kept_here;
 }
 
-// The kept tokens' index lists and rows.  Grid (G, B).  Every CTA of sample b gets the sample's N
-// keep flags -- from rank_kernel, or, for short sequences, by ranking all tokens itself (cheaper
-// than a second launch up to kFusedMaxN tokens) -- and scans them into the ascending list of kept
-// tokens; CTA 0 of the sample writes keep_idx, the flat source-row list row_map (b N + token: what
-// the next block uses to read the un-pruned x^ in place) and, when it ranked, the finished scores.
-// Then CTA g moves its share of the K kept rows, a warp per row: the dense copy x_out when one is
-// wanted, and, with LT given, LN of the row for the next block (the whole row then sits in one
-// warp's registers: row_vecs <= 32 * MAXV).
+// The rows of the kept tokens after rank_kernel: one warp per output row (b, r), eight rows per
+// CTA, no block-wide step.  The warp adds up the slice counts of its sample (two slices per lane,
+// at most 64 slices) to find the slice that holds the r-th kept token, then the token inside the
+// slice from its flags; it writes keep_idx and row_map for its row and moves the row: the dense
+// copy when one is wanted and, with LT given, LN of the row for the next block.
 template <int MAXV, typename LT>
-__global__ void __launch_bounds__(512)
-prune_kernel(const PruneArgs a) {
-    __shared__ uint32_t keys[kPruneMaxN];       // keys (when ranking here), then the list of kept tokens
-    __shared__ uint8_t flags[kPruneMaxN];
-    __shared__ int wsum[32];
-    __shared__ int sh_total;
+__global__ void __launch_bounds__(256)
+gather_ranked_kernel(const uint4* __restrict__ x, const uint8_t* __restrict__ flags, const int32_t* __restrict__ counts,
+                     int nsl, int P, long long rows, int N, int K, int b0, int row_vecs, int32_t* __restrict__ keep_idx,
+                     int32_t* __restrict__ row_map, uint4* __restrict__ x_out, const LnFuse ln) {
     grid_dep_launch();
     grid_dep_wait();
-    const int b = blockIdx.y, tid = threadIdx.x, nt = blockDim.x, N = a.N, K = a.K;
-    if (a.flags_in) {
-        const uint8_t* fb = a.flags_in + (long long)b * N;
-        for (int i = tid; i < N; i += nt) flags[i] = fb[i];
-    } else {
-        load_keys(a.scores, a.nparts, blockIdx.x == 0 ? a.scores_out : nullptr, b, N, 0, N, keys);
-        __syncthreads();
-        rank_slice(keys, N, K, a.has_cls ? 1 : 0, 0, N, [&](int i, uint8_t f) { flags[i] = f; });
+    const int lane = threadIdx.x & 31;
+    const long long row = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (row >= rows) return;
+    const int b = (int)(row / K), r = (int)(row - (long long)b * K);
+    const int32_t* cb = counts + (long long)b * nsl;
+    const int c0 = 2 * lane < nsl ? cb[2 * lane] : 0, c1 = 2 * lane + 1 < nsl ? cb[2 * lane + 1] : 0;
+    int inc = c0 + c1;                                  // inclusive prefix over the lanes' slice pairs
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += t;
     }
-    __syncthreads();
-    // ---- ascending list of kept tokens ----
-    const int chunk = (N + nt - 1) / nt;
-    const int lo_t = min(tid * chunk, N), hi_t = min(lo_t + chunk, N);
-    int cnt = 0;
-    for (int i = lo_t; i < hi_t; ++i) cnt += flags[i];
-    int pos = block_exclusive_scan(cnt, wsum, &sh_total);
-    int32_t* kept = reinterpret_cast<int32_t*>(keys);
-    for (int i = lo_t; i < hi_t; ++i)
-        if (flags[i]) {
-            if (pos < K) {
-                kept[pos] = i;
-                if (blockIdx.x == 0) {
-                    a.keep_idx[(long long)b * K + pos] = i;
-                    if (a.row_map) a.row_map[(long long)b * K + pos] = (a.b0 + b) * N + i;
-                }
+    const int before = inc - (c0 + c1);                 // kept tokens in the slices before this lane's pair
+    const unsigned owner = __ballot_sync(0xffffffffu, r >= before && r < inc);
+    const int src_lane = __ffs(owner) - 1;              // exactly one lane holds position r (r < K = total)
+    const int pb = __shfl_sync(0xffffffffu, before, src_lane), pc0 = __shfl_sync(0xffffffffu, c0, src_lane);
+    const int slice = 2 * src_lane + (r - pb >= pc0 ? 1 : 0);
+    int want = r - pb - (r - pb >= pc0 ? pc0 : 0);      // position inside the slice
+    const uint8_t* fb = flags + (long long)b * N + (long long)slice * P;
+    const int lim = min(P, N - slice * P);
+    int token = -1;
+    for (int e = 0; e < lim; e += 32) {
+        const bool f = e + lane < lim && fb[e + lane] != 0;
+        const unsigned m = __ballot_sync(0xffffffffu, f);
+        const int c = __popc(m);
+        if (token < 0) {
+            if (want < c) {                             // the (want+1)-th set bit of m
+                unsigned mm = m;
+                for (int k = 0; k < want; ++k) mm &= mm - 1;
+                token = slice * P + e + (__ffs(mm) - 1);
+            } else {
+                want -= c;
             }
-            ++pos;
         }
-    __syncthreads();
-    if (!a.x) return;
-    // ---- rows [lo, hi) of the sample's K kept rows belong to this CTA ----
-    const int G = gridDim.x, per = (K + G - 1) / G;
-    const int lo = blockIdx.x * per, hi = min(lo + per, K);
-    const int lane = tid & 31, warp = tid >> 5, nwarps = nt >> 5;
-    for (int r = lo + warp; r < hi; r += nwarps)
-        copy_row<MAXV, LT>(a.x + ((long long)b * N + kept[r]) * a.row_vecs, (long long)b * K + r, a.row_vecs, lane, a.x_out, a.ln);
+    }
+    if (lane == 0) {
+        keep_idx[row] = token;
+        if (row_map) row_map[row] = (b0 + b) * N + token;
+    }
+    if (x) copy_row<MAXV, LT>(x + ((long long)b * N + token) * row_vecs, row, row_vecs, lane, x_out, ln);
 }
 
 // Nothing dropped (K == N): every token is kept, in order; only the scores remain to be
@@ -490,6 +489,12 @@ cudaError_t select_init() {
     });
 }
 
+// Scratch bytes per sample of the two-kernel path: the slice counts, then a flag per token.
+static size_t prune_scratch_per_sample(int N) {
+    const int P = N <= 1024 ? 64 : 128, nsl = (N + P - 1) / P;
+    return (size_t)nsl * 4 + (size_t)((N + 3) / 4 * 4);
+}
+
 cudaError_t launch_select(const float* scores, int nparts, float* scores_out, int B, int N, int K,
                           int has_cls, int32_t* keep_idx, int32_t* row_map, uint8_t* flags, size_t flags_bytes,
                           int sm_count, cudaStream_t st, int* launches) {
@@ -499,7 +504,7 @@ cudaError_t launch_select(const float* scores, int nparts, float* scores_out, in
         const long long T = (long long)B * N;
         return launch_pdl(keep_all_kernel, dim3((unsigned)((T + 255) / 256)), dim3(256), 0, st, scores, nparts, scores_out, T, N, keep_idx);
     }
-    if (N <= kPruneMaxN && (N <= kFusedMaxN || flags_bytes >= (size_t)N))
+    if (prune_fusable(N, K, flags_bytes))
         return launch_prune(scores, nparts, scores_out, B, N, K, has_cls, keep_idx, row_map, RS_F32, nullptr, 0, nullptr, nullptr,
                             flags, flags_bytes, sm_count, st, launches);
     return launch_pdl(select_kernel, dim3(B), dim3(kSelThreads), select_smem_bytes(N), st, scores, nparts, scores_out, N, K,
@@ -507,7 +512,7 @@ cudaError_t launch_select(const float* scores, int nparts, float* scores_out, in
 }
 
 bool prune_fusable(int N, int K, size_t flags_bytes) {
-    return N <= kPruneMaxN && K < N && (N <= kFusedMaxN || flags_bytes >= (size_t)N);
+    return N <= kPruneMaxN && K < N && flags_bytes >= prune_scratch_per_sample(N);
 }
 
 bool ln_fusable(rs_dtype dtype, int D) { return (size_t)D * dtype_size(dtype) / 16 <= 32 * 4; }
@@ -517,50 +522,46 @@ cudaError_t launch_prune(const float* scores, int nparts, float* scores_out, int
                          const LnFuse* ln, uint8_t* flags, size_t flags_bytes, int sm_count, cudaStream_t st, int* launches) {
     if (launches) *launches = 0;
     if (B == 0) return cudaSuccess;
-    const bool two_step = N > kFusedMaxN;
-    if (N > kPruneMaxN || (ln && !ln_fusable(dtype, D)) || (x && !x_out && !ln) || (two_step && flags_bytes < (size_t)N))
+    const size_t per_sample = prune_scratch_per_sample(N);
+    if (N > kPruneMaxN || (ln && !ln_fusable(dtype, D)) || (x && !x_out && !ln) || flags_bytes < per_sample ||
+        (reinterpret_cast<uintptr_t>(flags) & 3u))
         return cudaErrorInvalidValue;
     const int row_vecs = x ? (int)((size_t)D * dtype_size(dtype) / 16) : 0;
     const size_t sz = dtype_size(dtype);
-    // samples per pass: as many as the flag scratch holds (all of them, unless the batch is huge)
-    const int Bc = two_step ? (int)((flags_bytes / (size_t)N) < (size_t)B ? flags_bytes / (size_t)N : (size_t)B) : B;
+    const LnFuse none = {nullptr, nullptr, 0.f, nullptr};
+    // samples per pass: as many as the scratch holds (all of them, unless the batch is huge)
+    const int Bc = (int)((flags_bytes / per_sample) < (size_t)B ? flags_bytes / per_sample : (size_t)B);
     for (int b0 = 0; b0 < B; b0 += Bc) {
         const int nb = B - b0 < Bc ? B - b0 : Bc;
         const long long t0 = (long long)b0 * N, k0 = (long long)b0 * K;
         const float* sc = scores + t0 * (nparts > 0 ? (nparts & 0xffff) * ((nparts >> 16) == RS_DIST_COS ? 3 : 1) : 1);
         float* so = scores_out ? scores_out + t0 : nullptr;
-        if (two_step) {
-            // tokens per ranking CTA: 64 (4 threads each) up to 1024 tokens, else 128 (8 threads each)
-            const int P = N <= 1024 ? 64 : 128, nt = N <= 1024 ? 256 : 1024;
-            cudaError_t e = launch_pdl(rank_kernel, dim3((N + P - 1) / P, nb), dim3(nt), 0, st, sc, nparts, so, N, K, has_cls, P, flags);
-            if (e != cudaSuccess) return e;
-            if (launches) *launches += 1;
-        }
-        // mover CTAs per sample: about three waves over the SMs (six when a row is also normalised
-        // and the sequence is short: measured), a few rows each; one CTA for the index lists alone
-        int G = 1;
-        if (x) {
-            G = ((ln && N <= 256 ? 6 : 3) * sm_count + nb - 1) / nb;
-            if (G > (K + 3) / 4) G = (K + 3) / 4;
-            if (G < 1) G = 1;
-        }
-        const int nt = N <= 128 ? 128 : 256;
-        PruneArgs a;
-        a.scores = sc; a.nparts = nparts; a.scores_out = so; a.N = N; a.K = K; a.has_cls = has_cls; a.b0 = b0;
-        a.flags_in = two_step ? flags : nullptr;
-        a.keep_idx = keep_idx + k0; a.row_map = row_map ? row_map + k0 : nullptr;
-        a.x = x ? (const uint4*)((const char*)x + (size_t)t0 * D * sz) : nullptr;
-        a.row_vecs = row_vecs;
-        a.x_out = x_out ? (uint4*)((char*)x_out + (size_t)k0 * D * sz) : nullptr;
-        a.ln = ln ? *ln : LnFuse{nullptr, nullptr, 0.f, nullptr};
-        if (ln) a.ln.out = (char*)ln->out + (size_t)k0 * D * sz;
+        const uint4* xs = x ? (const uint4*)((const char*)x + (size_t)t0 * D * sz) : nullptr;
+        uint4* xo = x_out ? (uint4*)((char*)x_out + (size_t)k0 * D * sz) : nullptr;
+        LnFuse lnc = ln ? *ln : none;
+        if (ln) lnc.out = (char*)ln->out + (size_t)k0 * D * sz;
         cudaError_t e;
-        const dim3 grid(G, nb), block(nt);
-        if (!ln) e = launch_pdl(prune_kernel<4, void>, grid, block, 0, st, a);
-        else if (dtype == RS_BF16) e = launch_pdl(prune_kernel<4, __nv_bfloat16>, grid, block, 0, st, a);
-        else e = launch_pdl(prune_kernel<4, float>, grid, block, 0, st, a);
-        if (e != cudaSuccess) return e;
-        if (launches) *launches += 1;
+        {
+            // ranking: 64 tokens per CTA (4 threads each) up to 1024 tokens, else 128 (8 threads each);
+            // then a warp per kept row
+            const int P = N <= 1024 ? 64 : 128, nt = N <= 1024 ? 256 : 1024, nsl = (N + P - 1) / P;
+            int32_t* counts = reinterpret_cast<int32_t*>(flags);
+            uint8_t* fl = flags + (size_t)nb * nsl * 4;
+            e = launch_pdl(rank_kernel, dim3(nsl, nb), dim3(nt), 0, st, sc, nparts, so, N, K, has_cls, P, fl, counts);
+            if (e != cudaSuccess) return e;
+            const long long rows = (long long)nb * K;
+            const dim3 grid((unsigned)((rows + 7) / 8)), block(256);
+            int32_t* rm = row_map ? row_map + k0 : nullptr;
+#define RS_GR_CASE(LT)                                                                                                  \
+    launch_pdl(gather_ranked_kernel<4, LT>, grid, block, 0, st, xs, (const uint8_t*)fl, (const int32_t*)counts, nsl, P, \
+               rows, N, K, b0, row_vecs, keep_idx + k0, rm, xo, lnc)
+            if (!ln) e = RS_GR_CASE(void);
+            else if (dtype == RS_BF16) e = RS_GR_CASE(__nv_bfloat16);
+            else e = RS_GR_CASE(float);
+#undef RS_GR_CASE
+            if (e != cudaSuccess) return e;
+            if (launches) *launches += 2;
+        }
     }
     return cudaSuccess;
 }

@@ -274,9 +274,10 @@ def test_graph_replay_equals_eager(ctx):
             assert torch.equal(a["keep_idx"], b["keep_idx"])
             assert torch.equal(a["x_out"].view(torch.int16), b["x_out"].view(torch.int16))
             assert torch.equal(a["scores"], b["scores"])
-    # eight kernels per block (selection and gather are one here); the block after a pruning block
-    # gets its LN1 from that block's compaction kernel and launches none: blocks 0 and 2 -> 8, block 1 -> 7
-    assert model.launches_per_forward(B, N, D) == 8 * L - 1
+    # seven kernels up to the FC2 epilogue, then two for a block that drops tokens (ranking, rows) or one
+    # (scores and identity indices) for a tapped block that drops none; the block after a pruning block
+    # gets its LN1 from that block's row kernel and launches none: blocks 0 and 2 -> 9, block 1 -> 7
+    assert model.launches_per_forward(B, N, D) == 9 + 7 + 9
     ctx.async_status()
 
 

@@ -134,15 +134,19 @@ def test_topk_compact_full_size_and_guard_bands(ctx):
 
 
 def test_topk_compact_batch_larger_than_the_flag_scratch(ctx):
-    """Sequences over 256 tokens are ranked by one kernel and moved by another, with a byte per token
-    in between; a batch with more tokens than that scratch holds (1 MiB) runs in several passes."""
+    """Tokens are ranked by one kernel and moved by another, with a byte per token (and a count per 64
+    tokens) in between; a batch with more tokens than that scratch holds (1 MiB)
+    runs in several passes."""
     B, N, D, r = 2100, 520, 8, 100
     s = _scores(B, N, "ties", 21)
     x = _tok((B, N, D), torch.float32, 22)
     xo, keep = ctx.topk_compact(torch.from_numpy(s).cuda(), x.cuda(), r, True)
     want = orc.topk(s.astype(np.float64), r, True)
     np.testing.assert_array_equal(keep.cpu().numpy(), want)
-    for b in (0, 1, 2015, 2016, 2017, B - 1):          # both sides of the pass boundary (2016 samples fit)
+    per_sample = 4 * ((N + 63) // 64) + (N + 3) // 4 * 4
+    cut = (1 << 20) // per_sample                        # samples that fit one pass
+    assert 1 < cut < B
+    for b in (0, 1, cut - 1, cut, cut + 1, B - 1):       # both sides of the pass boundary
         assert torch.equal(xo[b].cpu(), x[b][torch.from_numpy(want[b]).long()])
     _, keep2 = ctx.topk_compact(torch.from_numpy(s).cuda(), None, r, False)          # indices only
     np.testing.assert_array_equal(keep2.cpu().numpy(), orc.topk(s.astype(np.float64), r, False))
