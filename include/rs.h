@@ -57,8 +57,8 @@ typedef enum { RS_DIST_L2 = 0, RS_DIST_L1 = 1, RS_DIST_COS = 2 } rs_dist;
 /* Which pair of representations the block scores (Sec. 3.3 "Operation choice"). */
 typedef enum {
     RS_SCORE_MLP = 0,       /* (ii)  s = D(MLP(LN(x')), x')      -- the paper's default     */
-    RS_SCORE_MLP_DELTA = 1, /*       s = D(x^, x') = |MLP(LN(x'))| -- "before and after the
-                                     MLP layer" read with the residual included             */
+    RS_SCORE_MLP_DELTA = 1, /*       s = D(x^, x') = |MLP(LN(x'))| -- the main figure's caption
+                                     read as the shift of the residual stream across the MLP */
     RS_SCORE_ATTN = 2,      /* (i)   s = D(SA(LN(x)), x)         -- shift through attention  */
     RS_SCORE_BLOCK = 3      /* (iii) s = D(x^, x)                -- shift through the block  */
 } rs_score_mode;

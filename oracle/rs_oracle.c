@@ -179,7 +179,7 @@ static int orc_int_cmp(const void* pa, const void* pb) {
     return (a > b) - (a < b);
 }
 
-/* "Dropped the tokens having the lowest k scores": keep the K = N - r
+/* Sec. 3.2: the r lowest-score tokens are removed, i.e. keep the K = N - r
  * top-ranked tokens of every sample, listed in ascending index.  Returns 0, or
  * -1 for r outside [0, N-1]. */
 int orc_topk(const double* scores, int B, int N, int r, int has_cls, int32_t* keep_idx) {
@@ -258,7 +258,7 @@ void orc_grid_gather(const double* x, const int32_t* keep_rows, const int32_t* k
  *   m  = MLP(LN(x'))              (Eq. MLP without the residual)
  *   x^ = m + x'
  *   score_mode 0: s = ||m - x'||  (operation choice (ii), literal formula)
- *   score_mode 1: s = ||x^ - x'|| = ||m||  (the "before and after the MLP layer" reading)
+ *   score_mode 1: s = ||x^ - x'|| = ||m||  (the figure caption's reading of the MLP shift, residual included)
  *   score_mode 2: s = D(SA(LN(x)), x)      (operation choice (i))
  *   score_mode 3: s = D(x^, x)             (operation choice (iii))
  * Outputs (any may be NULL except x_hat): x_prime, m, x_hat [B,N,D]; scores
