@@ -235,6 +235,38 @@ RS_API rs_status rs_vit_fwd(rs_ctx* ctx, const rs_vit_desc* desc /*host*/,
                             const void* x, void* x_out, float* scores_last, int32_t* keep_last,
                             void* workspace, size_t workspace_bytes, void* stream);
 
+/* ---- per-sample token counts (Sec. 3.1: the reduced token set, here with a count of its own per ----
+ * sample, as a score threshold or a per-sample ratio gives; Sec. 4.1 "Settings" prunes by ratio).
+ * Layout: padded.  Every sample owns N rows of its tensors; sample b's seq_lens[b] tokens sit at the
+ * front of its rows, the rows behind them are padding.  Padding rows of an INPUT must hold finite
+ * values (zeros will do): they are multiplied by zero weights, never selected.  Padding rows of the
+ * token OUTPUT x_out are written as zeros, of keep_idx as -1; other outputs (attention rows, scores,
+ * x_full) are unspecified but finite there.  seq_lens, drops, lens_out (dev): [B] int32.  Values are
+ * read on the device and clamped there: seq_lens to [1, N], drops to [0, seq_lens[b] - 1], and the
+ * kept count seq_lens[b] - drops[b] to at most the row stride of the outputs.  Tensor-core path only
+ * (RS_BF16, head_dim 64; for the block D and D_mlp multiples of 128) and N <= 4608:
+ * RS_ERR_UNSUPPORTED otherwise, before any launch.
+ *
+ * rs_attn_fwd_ragged: rs_attn_fwd where sample b attends over its first seq_lens[b] tokens (Eq. sa
+ * on that many rows).
+ * rs_topk_compact_ragged: rs_topk_compact where sample b drops the drops[b] lowest-score tokens of
+ * its first seq_lens[b]; x_out [B, K_pad, D] and keep_idx [B, K_pad] have row stride K_pad >= every
+ * kept count; lens_out (optional) receives the kept counts.
+ * rs_block_fwd_ragged: rs_block_fwd on such a batch; desc->N is the padded length, desc->r fixes the
+ * row stride K_pad = N - r of x_out and keep_idx (so r must not exceed any drops[b]); keep_idx is
+ * required.  Workspace as for rs_block_fwd with the same descriptor. */
+RS_API rs_status rs_attn_fwd_ragged(rs_ctx* ctx, const rs_attn_desc* desc /*host*/, const void* q, const void* k,
+                                    const void* v, void* out, const int32_t* seq_lens, void* stream);
+RS_API rs_status rs_topk_compact_ragged(rs_ctx* ctx, rs_dtype dtype, int B, int N, int D, int K_pad, int has_cls,
+                                        const float* scores, const void* x, void* x_out, int32_t* keep_idx,
+                                        const int32_t* seq_lens, const int32_t* drops, int32_t* lens_out,
+                                        void* stream);
+RS_API rs_status rs_block_fwd_ragged(rs_ctx* ctx, const rs_block_desc* desc /*host*/,
+                                     const rs_block_weights* weights /*host struct of dev pointers*/, const void* x,
+                                     void* x_out, float* scores, int32_t* keep_idx, void* x_full,
+                                     const int32_t* seq_lens, const int32_t* drops, int32_t* lens_out,
+                                     void* workspace, size_t workspace_bytes, void* stream);
+
 /* ---- rs_block_fwd_static: rs_block_fwd for callers that cannot allocate ----------------
  * (The paper has no counterpart; this is a packaging variant of rs_block_fwd.)
  * Some callers have no way to obtain device memory when they reach the block:

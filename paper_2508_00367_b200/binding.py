@@ -28,7 +28,7 @@ EXPORTS = ("rs_create", "rs_destroy", "rs_last_error", "rs_async_status", "rs_us
            "rs_block_workspace_bytes", "rs_block_fwd", "rs_timing_enable", "rs_timing_read",
            "rs_static_scratch_bytes", "rs_block_fwd_static", "rs_linear_fwd", "rs_vit_workspace_bytes", "rs_vit_fwd",
            "rs_vit_fwd_taps", "rs_linewise_compact", "rs_static_async_status", "rs_linear_uses_tensor_cores",
-           "rs_block_uses_tensor_cores")
+           "rs_block_uses_tensor_cores", "rs_attn_fwd_ragged", "rs_topk_compact_ragged", "rs_block_fwd_ragged", "rs_tmap_cache_stats")
 LIN_EPILOGUE = {"bias": 0, "gelu": 1, "residual": 2}
 KERNEL_CLASSES = ("layernorm", "gemm", "attn", "score", "select", "gather")
 
@@ -131,6 +131,15 @@ def load_library() -> ctypes.CDLL:
     lib.rs_linear_uses_tensor_cores.restype = ci
     lib.rs_block_uses_tensor_cores.argtypes = [vp, ctypes.POINTER(BlockDesc)]
     lib.rs_block_uses_tensor_cores.restype = ci
+    lib.rs_tmap_cache_stats.argtypes = [vp, ctypes.POINTER(ctypes.c_longlong), ctypes.POINTER(ctypes.c_longlong)]
+    lib.rs_tmap_cache_stats.restype = ci
+    lib.rs_attn_fwd_ragged.argtypes = [vp, ctypes.POINTER(AttnDesc), vp, vp, vp, vp, vp, vp]
+    lib.rs_attn_fwd_ragged.restype = ci
+    lib.rs_topk_compact_ragged.argtypes = [vp, ci, ci, ci, ci, ci, ci, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.rs_topk_compact_ragged.restype = ci
+    lib.rs_block_fwd_ragged.argtypes = [vp, ctypes.POINTER(BlockDesc), ctypes.POINTER(BlockWeights), vp, vp, vp, vp, vp,
+                                        vp, vp, vp, vp, ctypes.c_size_t, vp]
+    lib.rs_block_fwd_ragged.restype = ci
     lib.rs_vit_workspace_bytes.argtypes = [ctypes.POINTER(VitDesc), ctypes.POINTER(ci)]
     lib.rs_vit_workspace_bytes.restype = ctypes.c_size_t
     lib.rs_vit_fwd.argtypes = [vp, ctypes.POINTER(VitDesc), ctypes.POINTER(BlockWeights), ctypes.POINTER(ci), vp, vp, vp,
@@ -211,6 +220,12 @@ class Context:
     def linear_uses_tensor_cores(self, dtype, M: int, N: int, K: int) -> bool:
         return bool(self.lib.rs_linear_uses_tensor_cores(self.handle, RS_BF16 if dtype == torch.bfloat16 else RS_F32, M, N, K))
 
+    def tmap_cache_stats(self):
+        """(hits, misses) of the context's tensor-map cache."""
+        h, m = ctypes.c_longlong(), ctypes.c_longlong()
+        self._check(self.lib.rs_tmap_cache_stats(self.handle, ctypes.byref(h), ctypes.byref(m)))
+        return int(h.value), int(m.value)
+
     def launch_count(self) -> int:
         return int(self.lib.rs_launch_count(self.handle))
 
@@ -239,6 +254,60 @@ class Context:
         self._check(self.lib.rs_attn_fwd(self.handle, ctypes.byref(d), _ptr(q), _ptr(k), _ptr(v), _ptr(out),
                                          _stream(q.device)))
         return out
+
+    # ---- per-sample token counts (padded layout) ----
+    def attn_fwd_ragged(self, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, seq_lens: torch.Tensor,
+                        scale: float = 0.0, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """rs_attn_fwd_ragged: sample b attends over its first seq_lens[b] tokens; rows behind them are unspecified."""
+        B, N, H, dh = q.shape
+        assert seq_lens.dtype == torch.int32 and seq_lens.is_cuda and seq_lens.numel() == B
+        if out is None:
+            out = torch.zeros(B, N, H * dh, dtype=q.dtype, device=q.device)
+        d = AttnDesc(_dt(q), B, N, H, dh, float(scale),
+                     q.stride(0), q.stride(1), q.stride(2), k.stride(0), k.stride(1), k.stride(2),
+                     v.stride(0), v.stride(1), v.stride(2))
+        self._check(self.lib.rs_attn_fwd_ragged(self.handle, ctypes.byref(d), _ptr(q), _ptr(k), _ptr(v), _ptr(out),
+                                                _ptr(seq_lens), _stream(q.device)))
+        return out
+
+    def topk_compact_ragged(self, scores: torch.Tensor, x: Optional[torch.Tensor], seq_lens: torch.Tensor,
+                            drops: torch.Tensor, K_pad: int, has_cls: bool = True):
+        """rs_topk_compact_ragged -> (x_out [B, K_pad, D] or None, keep_idx [B, K_pad], lens_out [B])."""
+        B, N = scores.shape
+        dev = scores.device
+        keep_idx = torch.empty(B, K_pad, dtype=torch.int32, device=dev)
+        lens_out = torch.empty(B, dtype=torch.int32, device=dev)
+        D, dt, x_out = 8, RS_F32, None
+        if x is not None:
+            D, dt = x.shape[2], _dt(x)
+            x_out = torch.empty(B, K_pad, D, dtype=x.dtype, device=dev)
+        self._check(self.lib.rs_topk_compact_ragged(self.handle, dt, B, N, D, K_pad, int(has_cls), _ptr(scores), _ptr(x),
+                                                    _ptr(x_out), _ptr(keep_idx), _ptr(seq_lens), _ptr(drops),
+                                                    _ptr(lens_out), _stream(dev)))
+        return x_out, keep_idx, lens_out
+
+    def block_fwd_ragged(self, x: torch.Tensor, weights: "DeviceBlockWeights", H: int, seq_lens: torch.Tensor,
+                         drops: torch.Tensor, K_pad: int, has_cls: bool = True, out_dtype=None,
+                         want_full: bool = False) -> Dict[str, torch.Tensor]:
+        """rs_block_fwd_ragged on a padded batch.  Returns dict(x_out [B, K_pad, D], scores [B, N], keep_idx
+        [B, K_pad], lens_out [B][, x_full])."""
+        assert x.is_cuda and x.is_contiguous()
+        B, N, D = x.shape
+        desc = self.block_desc(B, N, D, H, weights.D_mlp, N - K_pad, x.dtype, out_dtype, has_cls)
+        odt = _torch_dt(desc.out_dtype)
+        ws = torch.empty(max(self.block_workspace_bytes(desc), 256), dtype=torch.uint8, device=x.device)
+        res = dict(x_out=torch.empty(B, K_pad, D, dtype=odt, device=x.device),
+                   scores=torch.empty(B, N, dtype=torch.float32, device=x.device),
+                   keep_idx=torch.empty(B, K_pad, dtype=torch.int32, device=x.device),
+                   lens_out=torch.empty(B, dtype=torch.int32, device=x.device))
+        x_full = torch.empty(B, N, D, dtype=odt, device=x.device) if want_full else None
+        self._check(self.lib.rs_block_fwd_ragged(self.handle, ctypes.byref(desc), ctypes.byref(weights.struct), _ptr(x),
+                                                 _ptr(res["x_out"]), _ptr(res["scores"]), _ptr(res["keep_idx"]), _ptr(x_full),
+                                                 _ptr(seq_lens), _ptr(drops), _ptr(res["lens_out"]), _ptr(ws), ws.numel(),
+                                                 _stream(x.device)))
+        if want_full:
+            res["x_full"] = x_full
+        return res
 
     # ---- rs_linear_fwd ----
     def linear_fwd(self, a: torch.Tensor, w: torch.Tensor, bias: Optional[torch.Tensor] = None,

@@ -77,8 +77,9 @@ rs_status rs_create(rs_ctx** out, int device) {
     *out = nullptr;
     int count = 0;
     if (cudaGetDeviceCount(&count) != cudaSuccess || device < 0 || device >= count) return RS_ERR_CUDA;
-    rs_ctx* ctx = (rs_ctx*)calloc(1, sizeof(rs_ctx));
+    rs_ctx* ctx = (rs_ctx*)aligned_alloc(64, (sizeof(rs_ctx) + 63) / 64 * 64);
     if (!ctx) return RS_ERR_CUDA;
+    memset(ctx, 0, sizeof(rs_ctx));
     ctx->device = device;
     strcpy(ctx->err, "ok");
     cudaDeviceProp prop;
@@ -176,6 +177,13 @@ int rs_uses_tensor_cores(const rs_ctx* ctx, rs_dtype dtype) {
 
 long long rs_launch_count(const rs_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
+rs_status rs_tmap_cache_stats(const rs_ctx* ctx, long long* hits, long long* misses) {
+    if (!ctx || !hits || !misses) return RS_ERR_INVALID_ARG;
+    *hits = ctx->tmap_hits;
+    *misses = ctx->tmap_misses;
+    return RS_OK;
+}
+
 int rs_linear_uses_tensor_cores(const rs_ctx* ctx, rs_dtype dtype, long long M, int N, int K) {
     return ctx && ctx->use_tc && dtype == RS_BF16 && rs::gemm_tc_supported(M, N, K);
 }
@@ -203,7 +211,7 @@ rs_status rs_attn_fwd(rs_ctx* ctx, const rs_attn_desc* d, const void* q, const v
         if (st[i] < 0 || (st[i] % 8) != 0) return fail(ctx, RS_ERR_INVALID_ARG, "rs_attn_fwd: strides must be non-negative multiples of 8");
     if (!(d->scale >= 0.f)) return fail(ctx, RS_ERR_INVALID_ARG, "rs_attn_fwd: scale must be >= 0");
     if (ctx->use_tc && rs::attn_tc_supported(*d))
-        RS_CHECK_LAUNCH(ctx, RS_K_ATTN, (cudaStream_t)stream, rs::launch_attn_tc(ctx, *d, q, k, v, out, (cudaStream_t)stream), "tensor-core attention launch");
+        RS_CHECK_LAUNCH(ctx, RS_K_ATTN, (cudaStream_t)stream, rs::launch_attn_tc(ctx, *d, q, k, v, out, nullptr, (cudaStream_t)stream), "tensor-core attention launch");
     else
         RS_CHECK_LAUNCH(ctx, RS_K_ATTN, (cudaStream_t)stream, rs::launch_attn_simt(*d, q, k, v, out, (cudaStream_t)stream), "attention launch");
     return RS_OK;
@@ -273,7 +281,7 @@ rs_status rs_topk_compact(rs_ctx* ctx, rs_dtype dtype, int B, int N, int D, int 
     }
     int nl = 1;
     if (x && rs::prune_fusable(N, K, kFlagScratch)) {
-        RS_CHECK_LAUNCH(ctx, RS_K_GATHER, st, rs::launch_prune(scores, 0, nullptr, B, N, K, has_cls ? 1 : 0, keep_idx, nullptr, dtype, x, D, x_out, nullptr, ctx->d_flags, kFlagScratch, ctx->sm_count, st, &nl), "select+gather launch");
+        RS_CHECK_LAUNCH(ctx, RS_K_GATHER, st, rs::launch_prune(scores, 0, nullptr, B, N, K, has_cls ? 1 : 0, keep_idx, nullptr, dtype, x, D, x_out, nullptr, ctx->d_flags, kFlagScratch, ctx->sm_count, st, &nl, nullptr, nullptr, nullptr), "select+gather launch");
         ctx->launches += nl - 1;
         return RS_OK;
     }
@@ -328,6 +336,7 @@ rs_status rs_linewise_compact(rs_ctx* ctx, rs_dtype dtype, int B, int H, int W, 
 //   out_map: where to leave this block's row map (b * N + kept token) for the next block; with it and
 //            dense_out == false the dense copy x_out is not written at all: the next block reads x^
 //            through the map (Sec. 3.1: the reduced token set as an index list).
+//   seq_lens, drops, lens_out: per-sample token counts (rs_block_fwd_ragged); null otherwise.
 struct LoopHooks {
     const int32_t* in_map;
     const void* x_ln;
@@ -335,6 +344,9 @@ struct LoopHooks {
     int32_t* out_map;
     bool dense_out;
     bool* ln_done;
+    const int32_t* seq_lens;
+    const int32_t* drops;
+    int32_t* lens_out;
 };
 
 static rs_status block_fwd_impl(rs_ctx* ctx, const rs_block_desc* d, const rs_block_weights* w, const void* x,
@@ -384,13 +396,15 @@ static rs_status block_fwd_impl(rs_ctx* ctx, const rs_block_desc* d, const rs_bl
     int32_t* keep = keep_idx ? keep_idx : (int32_t*)(base + ws.keep);
     // The un-pruned output goes to x_full if given, straight to x_out when nothing is
     // dropped, else to scratch.
-    void* x_hat = x_full ? x_full : (d->r == 0 ? x_out : (void*)(base + ws.x_hat));
+    const bool ragged = hk && hk->seq_lens;
+    void* x_hat = x_full ? x_full : ((d->r == 0 && !ragged) ? x_out : (void*)(base + ws.x_hat));
 
     const bool tc = rs_block_uses_tensor_cores(ctx, d) != 0;
     if (ctx->require_tc && d->dtype == RS_BF16 && !tc)
         return fail(ctx, RS_ERR_UNSUPPORTED, "rs_block_fwd: shape outside the tensor-core kernels (D, D_mlp multiples of 128) and RS_REQUIRE_TC is set");
     const int32_t* in_map = hk ? hk->in_map : nullptr;
     if (in_map && !tc) return fail(ctx, RS_ERR_UNSUPPORTED, "rs_block_fwd: a row-mapped input needs the tensor-core kernels");
+    if (ragged && (!tc || d->N > 4608)) return fail(ctx, RS_ERR_UNSUPPORTED, "rs_block_fwd_ragged: needs the tensor-core kernels (bf16, D and D_mlp multiples of 128) and N <= 4608");
     const size_t sz = rs::dtype_size(d->dtype);
     rs_attn_desc ad;
     ad.dtype = d->dtype; ad.B = d->B; ad.N = d->N; ad.H = d->H; ad.head_dim = 64; ad.scale = d->scale;
@@ -409,7 +423,7 @@ static rs_status block_fwd_impl(rs_ctx* ctx, const rs_block_desc* d, const rs_bl
     }
     if (tc) {
         RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_tc(ctx, rs::RS_EPI_BIAS, x_ln, w->w_qkv, w->b_qkv, nullptr, nullptr, nullptr, qkv, RS_BF16, nullptr, 0, 0, T, 3 * D, D, st), "QKV");
-        RS_CHECK_LAUNCH(ctx, RS_K_ATTN, st, rs::launch_attn_tc(ctx, ad, qkv, kp, vp, o, st), "attention");
+        RS_CHECK_LAUNCH(ctx, RS_K_ATTN, st, rs::launch_attn_tc(ctx, ad, qkv, kp, vp, o, hk ? hk->seq_lens : nullptr, st), "attention");
         // shift through attention (operation choice (i)): partial sums of (SA(LN(x)) - x)^2 from this epilogue
         nparts = rs::gemm_tc_score_parts(ctx, T, D);
         float* attn_parts = d->score_mode == RS_SCORE_ATTN ? m : nullptr;
@@ -445,10 +459,18 @@ static rs_status block_fwd_impl(rs_ctx* ctx, const rs_block_desc* d, const rs_bl
     void* dense = dense_out ? x_out : nullptr;
     const int cls = d->has_cls ? 1 : 0;
     uint8_t* flags = (uint8_t*)(base + ws.flags);
+    if (ragged) {
+        // per-sample counts: sample b keeps lens[b] - drops[b] of its first lens[b] tokens; K is the row stride
+        int nlr = 0;
+        const size_t fb = (size_t)T + 4 * ((size_t)T / 64 + 2 * (size_t)d->B) + 16;
+        RS_CHECK_LAUNCH(ctx, RS_K_GATHER, st, rs::launch_prune(sel_in, sel_enc, sel_out, d->B, d->N, K, cls, keep, nullptr, d->out_dtype, x_hat, D, x_out, nullptr, flags, fb, ctx->sm_count, st, &nlr, hk->seq_lens, hk->drops, hk->lens_out), "select+gather (per-sample counts)");
+        ctx->launches += nlr - 1;
+        return RS_OK;
+    }
     const size_t flags_bytes = (size_t)T + 4 * ((size_t)T / 64 + 2 * (size_t)d->B) + 16;
     int nl = 1;
     if (moves && rs::prune_fusable(d->N, K, flags_bytes) && (dense || ln)) {
-        RS_CHECK_LAUNCH(ctx, RS_K_GATHER, st, rs::launch_prune(sel_in, sel_enc, sel_out, d->B, d->N, K, cls, keep, out_map, d->out_dtype, x_hat, D, dense, ln, flags, flags_bytes, ctx->sm_count, st, &nl), "select+gather");
+        RS_CHECK_LAUNCH(ctx, RS_K_GATHER, st, rs::launch_prune(sel_in, sel_enc, sel_out, d->B, d->N, K, cls, keep, out_map, d->out_dtype, x_hat, D, dense, ln, flags, flags_bytes, ctx->sm_count, st, &nl, nullptr, nullptr, nullptr), "select+gather");
         ctx->launches += nl - 1;
         return RS_OK;
     }
@@ -465,6 +487,57 @@ rs_status rs_block_fwd(rs_ctx* ctx, const rs_block_desc* d, const rs_block_weigh
                        void* x_out, float* scores, int32_t* keep_idx, void* x_full, void* workspace,
                        size_t workspace_bytes, void* stream) {
     return block_fwd_impl(ctx, d, w, x, x_out, scores, keep_idx, x_full, workspace, workspace_bytes, stream, nullptr);
+}
+
+rs_status rs_block_fwd_ragged(rs_ctx* ctx, const rs_block_desc* d, const rs_block_weights* w, const void* x,
+                              void* x_out, float* scores, int32_t* keep_idx, void* x_full, const int32_t* seq_lens,
+                              const int32_t* drops, int32_t* lens_out, void* workspace, size_t workspace_bytes,
+                              void* stream) {
+    if (!ctx) return RS_ERR_INVALID_ARG;
+    if (!seq_lens || !drops || !keep_idx) return fail(ctx, RS_ERR_INVALID_ARG, "rs_block_fwd_ragged: seq_lens, drops and keep_idx are required");
+    const LoopHooks hk = {nullptr, nullptr, nullptr, nullptr, true, nullptr, seq_lens, drops, lens_out};
+    return block_fwd_impl(ctx, d, w, x, x_out, scores, keep_idx, x_full, workspace, workspace_bytes, stream, &hk);
+}
+
+rs_status rs_attn_fwd_ragged(rs_ctx* ctx, const rs_attn_desc* d, const void* q, const void* k, const void* v,
+                             void* out, const int32_t* seq_lens, void* stream) {
+    if (!ctx) return RS_ERR_INVALID_ARG;
+    if (!seq_lens) return fail(ctx, RS_ERR_INVALID_ARG, "rs_attn_fwd_ragged: null seq_lens");
+    if (!d || !q || !k || !v || !out) return fail(ctx, RS_ERR_INVALID_ARG, "rs_attn_fwd_ragged: null argument");
+    if (!valid_dtype(d->dtype) || d->B < 1 || d->N < 1 || d->H < 1) return fail(ctx, RS_ERR_INVALID_ARG, "rs_attn_fwd_ragged: bad descriptor");
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || (reinterpret_cast<uintptr_t>(seq_lens) & 3u))
+        return fail(ctx, RS_ERR_INVALID_ARG, "rs_attn_fwd_ragged: misaligned pointer");
+    if (!(d->scale >= 0.f)) return fail(ctx, RS_ERR_INVALID_ARG, "rs_attn_fwd_ragged: scale must be >= 0");
+    if (!ctx->use_tc || !rs::attn_tc_supported(*d))
+        return fail(ctx, RS_ERR_UNSUPPORTED, "rs_attn_fwd_ragged: needs the tensor-core kernel (bf16, head_dim 64, strides multiples of 8)");
+    RS_CHECK_LAUNCH(ctx, RS_K_ATTN, (cudaStream_t)stream, rs::launch_attn_tc(ctx, *d, q, k, v, out, seq_lens, (cudaStream_t)stream), "tensor-core attention launch");
+    return RS_OK;
+}
+
+rs_status rs_topk_compact_ragged(rs_ctx* ctx, rs_dtype dtype, int B, int N, int D, int K_pad, int has_cls,
+                                 const float* scores, const void* x, void* x_out, int32_t* keep_idx,
+                                 const int32_t* seq_lens, const int32_t* drops, int32_t* lens_out, void* stream) {
+    if (!ctx) return RS_ERR_INVALID_ARG;
+    if (!valid_dtype(dtype)) return fail(ctx, RS_ERR_INVALID_ARG, "rs_topk_compact_ragged: bad dtype");
+    if (B < 0 || N < 1 || K_pad < 1 || K_pad > N) return fail(ctx, RS_ERR_INVALID_ARG, "rs_topk_compact_ragged: need B >= 0, 1 <= K_pad <= N");
+    if (N > 4608) return fail(ctx, RS_ERR_UNSUPPORTED, "rs_topk_compact_ragged: N > 4608");
+    if (B == 0) return RS_OK;
+    if (!scores || !keep_idx || !seq_lens || !drops) return fail(ctx, RS_ERR_INVALID_ARG, "rs_topk_compact_ragged: null scores, keep_idx, seq_lens or drops");
+    if ((x == nullptr) != (x_out == nullptr)) return fail(ctx, RS_ERR_INVALID_ARG, "rs_topk_compact_ragged: x and x_out must both be given or both be NULL");
+    if (x) {
+        if (D < 8 || (D % 8) != 0) return fail(ctx, RS_ERR_INVALID_ARG, "rs_topk_compact_ragged: D must be a positive multiple of 8");
+        if (!aligned16(x) || !aligned16(x_out)) return fail(ctx, RS_ERR_INVALID_ARG, "rs_topk_compact_ragged: misaligned pointer");
+        const size_t sz = rs::dtype_size(dtype);
+        const char* xa = (const char*)x;
+        const char* xo = (const char*)x_out;
+        const size_t xbytes = (size_t)B * N * D * sz, obytes = (size_t)B * K_pad * D * sz;
+        if (xa < xo + obytes && xo < xa + xbytes) return fail(ctx, RS_ERR_INVALID_ARG, "rs_topk_compact_ragged: x_out overlaps x");
+    }
+    int nl = 1;
+    cudaStream_t st = (cudaStream_t)stream;
+    RS_CHECK_LAUNCH(ctx, RS_K_GATHER, st, rs::launch_prune(scores, 0, nullptr, B, N, K_pad, has_cls ? 1 : 0, keep_idx, nullptr, dtype, x, D, x_out, nullptr, ctx->d_flags, kFlagScratch, ctx->sm_count, st, &nl, seq_lens, drops, lens_out), "select+gather launch (per-sample counts)");
+    ctx->launches += nl - 1;
+    return RS_OK;
 }
 
 }  // extern "C"
@@ -541,7 +614,7 @@ rs_status rs_vit_fwd_taps(rs_ctx* ctx, const rs_vit_desc* d, const rs_block_weig
         const rs::LnFuse next = {last ? nullptr : weights[l + 1].ln1_g, last ? nullptr : weights[l + 1].ln1_b, eps, ln_buf};
         bool ln_done = false;
         const LoopHooks hk = {cur_map, cur_ln, (last || !next.gamma || !next.beta) ? nullptr : &next,
-                              in_place ? maps[l & 1] : nullptr, !in_place, &ln_done};
+                              in_place ? maps[l & 1] : nullptr, !in_place, &ln_done, nullptr, nullptr, nullptr};
         rs_status st = block_fwd_impl(ctx, &bd, &weights[l], cur, out, taps->scores ? taps->scores[l] : nullptr,
                                       taps->keep_idx ? taps->keep_idx[l] : nullptr, in_place ? act[l & 1] : nullptr, base,
                                       p.block_ws, stream, &hk);

@@ -56,13 +56,15 @@ struct AttnArgs {
     // tile_count of them for each (sample, head) from first_single_bh on (see launch_attn_tc)
     int n_pair_items, first_single_bh, tile_count;
     float scale_log2;        // scale * log2(e)
+    const int* lens;         // optional [B]: sample b attends over its first lens[b] tokens only (clamped to 1 .. N)
     int* status;
 };
 
 // One work item, decoded the same way by every role.
 struct Item {
     int b, h[2], q0[2];      // sample; head and first query row of tile A / B
-    int ng;                  // 1 or 2 query tiles present
+    int n;                   // tokens of the sample (N, or its own length)
+    int ng;                  // query tiles present: 1 or 2 (0: the item lies past the sample's own length and is skipped)
     int nkv;                 // key tiles per query tile
     int slots;               // K/V ring stages the item consumes
 };
@@ -73,6 +75,7 @@ __device__ __forceinline__ Item decode_item(const AttnArgs& a, int w) {
         it.b = w / a.per;
         it.h[0] = 2 * hp; it.h[1] = 2 * hp + 1;
         it.q0[0] = it.q0[1] = 0;
+        it.n = a.lens ? min(max(__ldg(a.lens + it.b), 1), a.N) : a.N;
         it.ng = it.h[1] < a.H ? 2 : 1;
         it.nkv = 1;
         it.slots = it.ng;
@@ -82,19 +85,25 @@ __device__ __forceinline__ Item decode_item(const AttnArgs& a, int w) {
             const int qp = w % a.per;
             bh = w / a.per;
             it.q0[0] = qp * 2 * BQ; it.q0[1] = it.q0[0] + BQ;
-            it.ng = it.q0[1] < a.N ? 2 : 1;
         } else {
             const int k = w - a.n_pair_items;
             bh = a.first_single_bh + k / a.tile_count;
             it.q0[0] = (k % a.tile_count) * BQ; it.q0[1] = a.N;       // one query tile only
-            it.ng = 1;
         }
         it.b = bh / a.H;
         it.h[0] = it.h[1] = bh % a.H;
-        it.nkv = (a.N + BKV - 1) / BKV;
+        it.n = a.lens ? min(max(__ldg(a.lens + it.b), 1), a.N) : a.N;
+        it.ng = (it.q0[0] < it.n ? 1 : 0) + (it.q0[1] < it.n ? 1 : 0);
+        it.nkv = (it.n + BKV - 1) / BKV;
         it.slots = it.nkv;
     }
     return it;
+}
+// First item at or after w (in this CTA's stride) that has work; n_items if none.
+__device__ __forceinline__ int next_item(const AttnArgs& a, int w, int stride) {
+    if (!a.lens) return w;
+    while (w < a.n_items && decode_item(a, w).ng == 0) w += stride;
+    return w;
 }
 
 __device__ __forceinline__ float ex2(float x) {
@@ -209,7 +218,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int N = args.N;
 
     if (threadIdx.x == 0) {
         prefetch_tmap(&tmQ); prefetch_tmap(&tmK); prefetch_tmap(&tmV); prefetch_tmap(&tmO);
@@ -239,7 +247,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         if (elect_one()) {
             uint32_t kv_it = 0, item_n = 0;
             bool ok = true;
-            for (int w = blockIdx.x; w < args.n_items && ok; w += gridDim.x, ++item_n) {
+            for (int w = next_item(args, blockIdx.x, gridDim.x); w < args.n_items && ok; w = next_item(args, w + gridDim.x, gridDim.x), ++item_n) {
                 const Item it = decode_item(args, w);
                 const uint32_t qb = item_n & 1u;
                 if (!mbar_wait(&q_empty[qb], ((item_n >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
@@ -265,7 +273,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         }
     } else if (warp == 9) {
         // ---------------- MMA issuer ----------------
-        if (elect_one() && blockIdx.x < args.n_items) {
+        if (elect_one() && next_item(args, blockIdx.x, gridDim.x) < args.n_items) {
             constexpr uint32_t idesc_o = idesc_bf16(BQ, DH, 0, 1), idesc_s_full = idesc_bf16(BQ, BKV, 0, 0);
             // descriptors as halves: per product only the low half moves (address >> 4)
             constexpr uint32_t kTile16 = TILE_BYTES >> 4;
@@ -312,11 +320,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             auto issue_s_one = [&](const Item& it, uint32_t qb, uint32_t kv0, int j, int g) {
                 const uint32_t t = kv0 + (args.dual ? g : j);
                 if (!mbar_wait(&k_full[t % NS], (t / NS) & 1u, abort_flag)) { ok = false; return; }
-                issue_s(g, qb, t % NS, min(BKV, N - j * BKV));
+                issue_s(g, qb, t % NS, min(BKV, it.n - j * BKV));
             };
 
             uint32_t item_n = 0, kv0 = 0;
-            int w = blockIdx.x;
+            int w = next_item(args, blockIdx.x, gridDim.x);
             Item cur = decode_item(args, w);
             ok = mbar_wait(&q_full[0], 0, abort_flag);
 #pragma unroll
@@ -324,7 +332,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 if (ok && g < cur.ng) issue_s_one(cur, 0, kv0, 0, g);
             while (ok) {
                 const uint32_t qb = item_n & 1u;
-                const int wn = w + gridDim.x;
+                const int wn = next_item(args, w + gridDim.x, gridDim.x);
                 Item nxt = cur;
                 for (int j = 0; j < cur.nkv && ok; ++j) {
                     // Look ahead, per query tile: the tile's next Q K^T (of this item, or the first of the
@@ -341,7 +349,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     const Item& sit = last ? nxt : cur;
                     const uint32_t skv0 = last ? kv0 + cur.slots : kv0;
                     const int sj = last ? 0 : j + 1;
-                    const int valid = min(BKV, N - j * BKV);
+                    const int valid = min(BKV, cur.n - j * BKV);
 #pragma unroll
                     for (int g = 0; g < 2; ++g) {
                         if (!ok) break;
@@ -380,7 +388,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             if (g >= it.ng) continue;
             float m_l2 = 0.f, l_run = 0.f;               // running maximum (times scale*log2 e) and sum
             for (int j = 0; j < it.nkv && ok; ++j, ++cnt) {
-                const int valid = min(BKV, N - j * BKV);
+                const int valid = min(BKV, it.n - j * BKV);
                 // the warp moves as one through the collective tensor-memory accesses below
                 if (!__all_sync(0xffffffffu, mbar_wait(&s_full[g], cnt & 1u, abort_flag))) { ok = false; break; }
                 tc_fence_after();
@@ -469,7 +477,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             fence_async_smem();
             __syncwarp();
             const int row0 = (g ? it.q0[1] : it.q0[0]) + q * 32;
-            if (lane == 0 && row0 < N) {
+            if (lane == 0 && row0 < it.n) {
                 tma_store_4d(&tmO, smem + OFF_OST + (g * 4 + q) * 4096, 0, g ? it.h[1] : it.h[0], row0, it.b);
                 tma_store_commit();
             }
@@ -488,24 +496,15 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     }
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-// [B, N, H, 64] view with element strides; box = 128 rows of one head of one sample.
-bool make_tmap_qkv(void* encode_fn, CUtensorMap* out, const void* base, int B, int N, int H, long long bs,
+// [B, N, H, 64] view with element strides; box = box_rows rows of one head of one sample.
+bool make_tmap_qkv(rs_ctx* ctx, CUtensorMap* out, const void* base, int B, int N, int H, long long bs,
                    long long rs_, long long hs, int box_rows = 128) {
-    EncodeTiledFn fn = reinterpret_cast<EncodeTiledFn>(encode_fn);
-    const cuuint64_t dims[4] = {64, (cuuint64_t)H, (cuuint64_t)N, (cuuint64_t)B};
+    const unsigned long long dims[4] = {64, (unsigned long long)H, (unsigned long long)N, (unsigned long long)B};
     // a dimension of extent 1 never uses its stride; give it a harmless valid one
-    const cuuint64_t hs_b = (H > 1 ? (cuuint64_t)hs : 64) * 2, rs_b = (N > 1 ? (cuuint64_t)rs_ : 64) * 2,
-                     bs_b = (B > 1 ? (cuuint64_t)bs : 64) * 2;
-    const cuuint64_t strides[3] = {hs_b, rs_b, bs_b};
-    const cuuint32_t box[4] = {64, 1, (cuuint32_t)box_rows, 1};
-    const cuuint32_t estr[4] = {1, 1, 1, 1};
-    return fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    const unsigned long long strides[3] = {(H > 1 ? (unsigned long long)hs : 64) * 2, (N > 1 ? (unsigned long long)rs_ : 64) * 2,
+                                           (B > 1 ? (unsigned long long)bs : 64) * 2};
+    const unsigned int box[4] = {64, 1, (unsigned int)box_rows, 1};
+    return tc_encode_cached(ctx, out, base, 4, 0, dims, strides, box, 128);
 }
 
 }  // namespace
@@ -525,7 +524,7 @@ bool attn_tc_supported(const rs_attn_desc& d) {
 }
 
 cudaError_t launch_attn_tc(rs_ctx* ctx, const rs_attn_desc& d, const void* q, const void* k, const void* v,
-                           void* out, cudaStream_t st) {
+                           void* out, const int32_t* seq_lens, cudaStream_t st) {
     if (!ctx->encode_tiled) return cudaErrorNotSupported;
     static PerDeviceOnce attr_once;   // the attribute belongs to the device current at the call
     int dev = -1;
@@ -539,10 +538,10 @@ cudaError_t launch_attn_tc(rs_ctx* ctx, const rs_attn_desc& d, const void* q, co
     if (e != cudaSuccess) return e;
     CUtensorMap tmQ, tmK, tmV, tmO;
     // out is [B, N, H, 64] contiguous; a softmax warp stores its 32 rows of one head at a time
-    if (!make_tmap_qkv(ctx->encode_tiled, &tmO, out, d.B, d.N, d.H, (long long)d.N * d.H * 64, (long long)d.H * 64, 64, 32) ||
-        !make_tmap_qkv(ctx->encode_tiled, &tmQ, q, d.B, d.N, d.H, d.q_batch_stride, d.q_row_stride, d.q_head_stride) ||
-        !make_tmap_qkv(ctx->encode_tiled, &tmK, k, d.B, d.N, d.H, d.k_batch_stride, d.k_row_stride, d.k_head_stride) ||
-        !make_tmap_qkv(ctx->encode_tiled, &tmV, v, d.B, d.N, d.H, d.v_batch_stride, d.v_row_stride, d.v_head_stride))
+    if (!make_tmap_qkv(ctx, &tmO, out, d.B, d.N, d.H, (long long)d.N * d.H * 64, (long long)d.H * 64, 64, 32) ||
+        !make_tmap_qkv(ctx, &tmQ, q, d.B, d.N, d.H, d.q_batch_stride, d.q_row_stride, d.q_head_stride) ||
+        !make_tmap_qkv(ctx, &tmK, k, d.B, d.N, d.H, d.k_batch_stride, d.k_row_stride, d.k_head_stride) ||
+        !make_tmap_qkv(ctx, &tmV, v, d.B, d.N, d.H, d.v_batch_stride, d.v_row_stride, d.v_head_stride))
         return cudaErrorInvalidValue;
     AttnArgs args;
     args.out = (__nv_bfloat16*)out;
@@ -598,6 +597,7 @@ cudaError_t launch_attn_tc(rs_ctx* ctx, const rs_attn_desc& d, const void* q, co
     args.n_items = (int)items;
     const float scale = d.scale != 0.f ? d.scale : 0.125f;
     args.scale_log2 = scale * 1.4426950408889634f;
+    args.lens = seq_lens;
     args.status = ctx->d_status;
     // One resident CTA per SM walks the item list, so set-up, loads and epilogues overlap across
     // items (also for long items: measured 2-5 % over one CTA per item at N = 2305 ... 4097).

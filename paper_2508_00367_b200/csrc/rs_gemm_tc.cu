@@ -18,6 +18,8 @@
 //                  optionally partial sums of (a - x)^2 per row    (shift through attention, choice (i))
 //   EPI_SCORE      m = acc + b;  out = m + x';  partial sums of (m - x')^2, m^2 or (out - x)^2 per row
 //                                                          -> bf16/fp32 (FC2 + residual + shift score)
+#include <string.h>
+
 #include "rs_internal.h"
 #include "rs_device.cuh"
 #include "rs_once.h"
@@ -446,36 +448,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
 // Tensor map over a row-major matrix [rows, cols] (cols contiguous) of 2- or 4-byte elements,
 // box [box_rows, 128 bytes of columns], 128-byte swizzle.
-bool make_tmap_2d(void* encode_fn, CUtensorMap* out, const void* base, int elem_bytes, uint64_t rows, uint64_t cols,
+bool make_tmap_2d(rs_ctx* ctx, CUtensorMap* out, const void* base, int elem_bytes, uint64_t rows, uint64_t cols,
                   uint32_t box_rows) {
-    EncodeTiledFn fn = reinterpret_cast<EncodeTiledFn>(encode_fn);
-    const cuuint64_t dims[2] = {cols, rows};
-    const cuuint64_t strides[1] = {cols * (uint64_t)elem_bytes};
-    const cuuint32_t box[2] = {(cuuint32_t)(128 / elem_bytes), box_rows};
-    const cuuint32_t estr[2] = {1, 1};
-    return fn(out, elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
-              const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    const unsigned long long dims[2] = {cols, rows}, strides[1] = {cols * (uint64_t)elem_bytes};
+    const unsigned int box[2] = {(unsigned int)(128 / elem_bytes), box_rows};
+    return tc_encode_cached(ctx, out, base, 2, elem_bytes == 2 ? 0 : 1, dims, strides, box, 128);
 }
 
 // Tensor map over the bf16 residual [rows, cols] of the projection: box [32 rows, 32 columns = 64 bytes],
 // 64-byte swizzle, zeros for rows past the matrix.
-bool make_tmap_res(void* encode_fn, CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols) {
-    EncodeTiledFn fn = reinterpret_cast<EncodeTiledFn>(encode_fn);
-    const cuuint64_t dims[2] = {cols, rows};
-    const cuuint64_t strides[1] = {cols * 2};
-    const cuuint32_t box[2] = {32, 32};
-    const cuuint32_t estr[2] = {1, 1};
-    return fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+bool make_tmap_res(rs_ctx* ctx, CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols) {
+    const unsigned long long dims[2] = {cols, rows}, strides[1] = {cols * 2};
+    const unsigned int box[2] = {32, 32};
+    return tc_encode_cached(ctx, out, base, 2, 0, dims, strides, box, 64);
 }
 
 template <int BN, int EPI, typename OutT>
@@ -529,6 +516,45 @@ int pick_bn(long long M, int N, int sm_count) {
 
 }  // namespace
 
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+bool tc_encode_cached(rs_ctx* ctx, CUtensorMap* out, const void* base, int rank, int dtype, const unsigned long long* dims,
+                      const unsigned long long* strides, const unsigned int* box, int swizzle_bytes) {
+    if (!ctx->encode_tiled || rank < 2 || rank > 4) return false;
+    rs_tmap_key key;
+    memset(&key, 0, sizeof(key));
+    key.base = base; key.rank = (unsigned)rank; key.dtype = (unsigned)dtype; key.swizzle = (unsigned)swizzle_bytes;
+    for (int i = 0; i < rank; ++i) { key.dims[i] = dims[i]; key.box[i] = box[i]; }
+    for (int i = 0; i + 1 < rank; ++i) key.strides[i] = strides[i];
+    unsigned long long h = (unsigned long long)(uintptr_t)base * 0x9E3779B97F4A7C15ull;
+    for (int i = 0; i < rank; ++i) h = (h ^ key.dims[i] ^ ((unsigned long long)key.box[i] << 40)) * 0x9E3779B97F4A7C15ull;
+    h ^= (unsigned long long)swizzle_bytes << 8 | (unsigned long long)dtype;
+    rs_tmap_slot& slot = ctx->tmaps[(h >> 32) % kTmapSlots];
+    if (slot.valid && memcmp(&slot.key, &key, sizeof(key)) == 0) {
+        *out = slot.map;
+        ctx->tmap_hits += 1;
+        return true;
+    }
+    EncodeTiledFn fn = reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled);
+    cuuint64_t d[4], st[3];
+    cuuint32_t bx[4], estr[4] = {1, 1, 1, 1};
+    for (int i = 0; i < rank; ++i) { d[i] = dims[i]; bx[i] = box[i]; }
+    for (int i = 0; i + 1 < rank; ++i) st[i] = strides[i];
+    const CUtensorMapSwizzle sw = swizzle_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : swizzle_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B
+                                                                                                         : CU_TENSOR_MAP_SWIZZLE_NONE;
+    CUtensorMap m;
+    if (fn(&m, dtype == 0 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, (cuuint32_t)rank,
+           const_cast<void*>(base), d, st, bx, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return false;
+    slot.map = m; slot.key = key; slot.valid = 1;
+    ctx->tmap_misses += 1;
+    *out = m;
+    return true;
+}
+
 void* tc_get_encode_fn() {
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult qres;
@@ -553,10 +579,10 @@ cudaError_t launch_gemm_tc(rs_ctx* ctx, int epi, const void* A, const void* W, c
     const int bn = pick_bn(M, N, ctx->sm_count);
     const int out_bytes = (epi == EPI_RESID || (epi == EPI_SCORE && out_dtype == RS_F32)) ? 4 : 2;
     CUtensorMap tmA, tmB, tmOut, tmRes;
-    if (epi == EPI_RESID && !row_map && !make_tmap_res(ctx->encode_tiled, &tmRes, residual, (uint64_t)M, (uint64_t)N)) return cudaErrorInvalidValue;
-    if (!make_tmap_2d(ctx->encode_tiled, &tmA, A, 2, (uint64_t)M, (uint64_t)K, BM) ||
-        !make_tmap_2d(ctx->encode_tiled, &tmB, W, 2, (uint64_t)N, (uint64_t)K, (uint32_t)(bn / 2)) ||
-        !make_tmap_2d(ctx->encode_tiled, &tmOut, out, out_bytes, (uint64_t)M, (uint64_t)N, 32))
+    if (epi == EPI_RESID && !row_map && !make_tmap_res(ctx, &tmRes, residual, (uint64_t)M, (uint64_t)N)) return cudaErrorInvalidValue;
+    if (!make_tmap_2d(ctx, &tmA, A, 2, (uint64_t)M, (uint64_t)K, BM) ||
+        !make_tmap_2d(ctx, &tmB, W, 2, (uint64_t)N, (uint64_t)K, (uint32_t)(bn / 2)) ||
+        !make_tmap_2d(ctx, &tmOut, out, out_bytes, (uint64_t)M, (uint64_t)N, 32))
         return cudaErrorInvalidValue;
     if (epi != EPI_RESID || row_map) tmRes = tmOut;  // unused by the other epilogues and by the mapped residual
     GemmArgs args;

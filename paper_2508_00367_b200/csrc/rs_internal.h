@@ -1,6 +1,7 @@
 // Internal declarations shared by the translation units of the library: the
 // context object and the host-side launchers of every kernel.
 #pragma once
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
 #include <stdint.h>
@@ -8,6 +9,22 @@
 
 #include "rs.h"
 #include "rs_profile.h"
+
+// Tensor maps are encoded once per (pointer, shape, box) and kept in the context: a block's launches
+// name the same few buffers over and over, and every cuTensorMapEncodeTiled call costs about a
+// microsecond of host time.  Direct-mapped, 64 slots; a slot is simply overwritten on a clash.
+struct rs_tmap_key {
+    const void* base;
+    unsigned long long dims[4], strides[3];
+    unsigned int box[4];
+    unsigned int rank, dtype, swizzle, pad;
+};
+struct rs_tmap_slot {
+    CUtensorMap map;
+    rs_tmap_key key;
+    int valid;
+};
+enum { kTmapSlots = 64 };
 
 struct rs_ctx {
     int device;
@@ -23,6 +40,8 @@ struct rs_ctx {
     cudaEvent_t* ev;       // 2 * kMaxTimed events, created on first enable
     unsigned char* ev_class;
     char err[512];
+    long long tmap_hits, tmap_misses;
+    rs_tmap_slot tmaps[kTmapSlots];   // (CUtensorMap wants 64-byte alignment: the context is allocated accordingly)
 };
 
 enum { kMaxTimed = 8192 };
@@ -98,7 +117,8 @@ bool prune_fusable(int N, int K, size_t flags_bytes);
 cudaError_t launch_prune(const float* scores, int nparts, float* scores_out, int B, int N, int K, int has_cls,
                          int32_t* keep_idx, int32_t* row_map, rs_dtype dtype, const void* x, int D, void* x_out,
                          const LnFuse* ln /*null: none*/, uint8_t* flags, size_t flags_bytes, int sm_count,
-                         cudaStream_t st, int* launches);
+                         cudaStream_t st, int* launches, const int32_t* seq_lens /*dev [B] or null*/,
+                         const int32_t* drops /*dev [B], with seq_lens*/, int32_t* lens_out /*dev [B] or null*/);
 // Line-wise pruning of a 2-D token grid: keep_rows [B, Hk], keep_cols [B, Wk] and, when x is given,
 // x_out[b, i, j, :] = x[b, keep_rows[b, i], keep_cols[b, j], :].  H, W <= linewise_max_lines().
 int linewise_max_lines();
@@ -119,6 +139,10 @@ cudaError_t launch_attn_simt(const rs_attn_desc& d, const void* q, const void* k
 // ---- tcgen05 GEMM (rs_gemm_tc.cu): bf16 operands, fp32 accumulation in tensor memory ----
 enum { RS_EPI_BIAS = 0, RS_EPI_BIAS_GELU = 1, RS_EPI_RESID = 2, RS_EPI_SCORE = 3 };
 void* tc_get_encode_fn();                       // cuTensorMapEncodeTiled via the runtime, or null
+// Tiled tensor map of `rank` dimensions over bf16 (dtype 0) or fp32 (dtype 1) elements, through the
+// context's cache; strides in bytes for dimensions 1 .. rank-1.  False when the driver refuses it.
+bool tc_encode_cached(rs_ctx* ctx, CUtensorMap* out, const void* base, int rank, int dtype, const unsigned long long* dims,
+                      const unsigned long long* strides, const unsigned int* box, int swizzle_bytes);
 bool gemm_tc_supported(long long M, int N, int K);
 int gemm_tc_score_parts(const rs_ctx* ctx, long long M, int N);   // partial sums per row written by RS_EPI_SCORE
 // out[M, N] = epilogue(A[M, K] . W[N, K]^T); see rs_gemm_tc.cu for the epilogues.
@@ -131,7 +155,8 @@ cudaError_t launch_gemm_tc(rs_ctx* ctx, int epi, const void* A, const void* W, c
 
 // ---- tcgen05 attention (rs_attn_tc.cu): bf16, head dimension 64 ----
 bool attn_tc_supported(const rs_attn_desc& d);
+// seq_lens (optional, dev [B]): sample b attends over its first seq_lens[b] tokens only.
 cudaError_t launch_attn_tc(rs_ctx* ctx, const rs_attn_desc& d, const void* q, const void* k, const void* v,
-                           void* out, cudaStream_t st);
+                           void* out, const int32_t* seq_lens, cudaStream_t st);
 
 }  // namespace rs

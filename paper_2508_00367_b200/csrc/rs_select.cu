@@ -271,19 +271,34 @@ __device__ __forceinline__ void rank_slice(const uint32_t* keys, int N, int K, i
 // and leaves their keep flags in global memory; N^2 / P comparisons per CTA instead of N^2.
 // It also leaves the number of kept tokens of its slice in counts[b, g]: with those, whoever moves
 // the rows finds the token behind an output position without scanning the sample.
+// Per-sample lengths (lens, drops non-null): sample b has n_b = lens[b] tokens (clamped to 1 .. N) at
+// the front of its N rows and drops r_b = drops[b] of them (clamped to 0 .. n_b - 1); the rows past
+// n_b are never kept.
+struct Ragged { const int32_t* lens; const int32_t* drops; int32_t* lens_out; };
+__device__ __forceinline__ void sample_counts(const Ragged& rg, int b, int N, int K, int* n_b, int* k_b) {
+    if (!rg.lens) { *n_b = N; *k_b = K; return; }
+    const int n = min(max(__ldg(rg.lens + b), 1), N);
+    const int r = min(max(__ldg(rg.drops + b), 0), n - 1);
+    *n_b = n; *k_b = min(n - r, K);          // K: the row stride of the outputs, an upper bound of every count
+}
+
 __global__ void __launch_bounds__(1024)
 rank_kernel(const float* __restrict__ scores, int nparts, float* __restrict__ scores_out, int N, int K, int has_cls,
-            int P, uint8_t* __restrict__ flags, int32_t* __restrict__ counts) {
+            int P, uint8_t* __restrict__ flags, int32_t* __restrict__ counts, const Ragged rg, int b0) {
     __shared__ uint32_t keys[kPruneMaxN];
     __shared__ int kept_here;
     grid_dep_launch();
     grid_dep_wait();
     const int b = blockIdx.y, i0 = blockIdx.x * P;
+    int n_b, k_b;
+    sample_counts(rg, b0 + b, N, K, &n_b, &k_b);
     if (threadIdx.x == 0) kept_here = 0;
     load_keys(scores, nparts, scores_out, b, N, i0, i0 + P, keys);
     __syncthreads();
     uint8_t* fb = flags + (long long)b * N;
-    rank_slice(keys, N, K, has_cls ? 1 : 0, i0, P, [&](int i, uint8_t f) { fb[i] = f; if (f) atomicAdd(&kept_here, 1); });
+    // (the stride between samples stays N; only the first n_b keys take part)
+    rank_slice(keys, n_b, k_b, has_cls ? 1 : 0, i0, P, [&](int i, uint8_t f) { fb[i] = f; if (f) atomicAdd(&kept_here, 1); });
+    for (int i = max(i0, n_b) + (int)threadIdx.x; i < min(i0 + P, N); i += blockDim.x) fb[i] = 0;
     __syncthreads();
     if (threadIdx.x == 0) counts[(long long)b * gridDim.x + blockIdx.x] = kept_here;
 }
@@ -297,13 +312,26 @@ template <int MAXV, typename LT>
 __global__ void __launch_bounds__(256)
 gather_ranked_kernel(const uint4* __restrict__ x, const uint8_t* __restrict__ flags, const int32_t* __restrict__ counts,
                      int nsl, int P, long long rows, int N, int K, int b0, int row_vecs, int32_t* __restrict__ keep_idx,
-                     int32_t* __restrict__ row_map, uint4* __restrict__ x_out, const LnFuse ln) {
+                     int32_t* __restrict__ row_map, uint4* __restrict__ x_out, const LnFuse ln, const Ragged rg) {
     grid_dep_launch();
     grid_dep_wait();
     const int lane = threadIdx.x & 31;
     const long long row = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
     if (row >= rows) return;
     const int b = (int)(row / K), r = (int)(row - (long long)b * K);
+    if (rg.lens) {
+        // K is the row stride of the outputs here; sample b keeps k_b <= K rows: the rest of its
+        // block is zero-filled (index -1) so that whatever reads the padded buffer next sees finite rows
+        int n_b, k_b;
+        sample_counts(rg, b0 + b, N, K, &n_b, &k_b);
+        if (r == 0 && lane == 0 && rg.lens_out) rg.lens_out[b0 + b] = k_b;
+        if (r >= k_b) {
+            if (lane == 0) { keep_idx[row] = -1; if (row_map) row_map[row] = -1; }
+            if (x && x_out)
+                for (int iv = lane; iv < row_vecs; iv += 32) x_out[row * row_vecs + iv] = make_uint4(0u, 0u, 0u, 0u);
+            return;
+        }
+    }
     const int32_t* cb = counts + (long long)b * nsl;
     const int c0 = 2 * lane < nsl ? cb[2 * lane] : 0, c1 = 2 * lane + 1 < nsl ? cb[2 * lane + 1] : 0;
     int inc = c0 + c1;                                  // inclusive prefix over the lanes' slice pairs
@@ -506,7 +534,7 @@ cudaError_t launch_select(const float* scores, int nparts, float* scores_out, in
     }
     if (prune_fusable(N, K, flags_bytes))
         return launch_prune(scores, nparts, scores_out, B, N, K, has_cls, keep_idx, row_map, RS_F32, nullptr, 0, nullptr, nullptr,
-                            flags, flags_bytes, sm_count, st, launches);
+                            flags, flags_bytes, sm_count, st, launches, nullptr, nullptr, nullptr);
     return launch_pdl(select_kernel, dim3(B), dim3(kSelThreads), select_smem_bytes(N), st, scores, nparts, scores_out, N, K,
                       has_cls, keep_idx, row_map);
 }
@@ -519,7 +547,9 @@ bool ln_fusable(rs_dtype dtype, int D) { return (size_t)D * dtype_size(dtype) / 
 
 cudaError_t launch_prune(const float* scores, int nparts, float* scores_out, int B, int N, int K, int has_cls,
                          int32_t* keep_idx, int32_t* row_map, rs_dtype dtype, const void* x, int D, void* x_out,
-                         const LnFuse* ln, uint8_t* flags, size_t flags_bytes, int sm_count, cudaStream_t st, int* launches) {
+                         const LnFuse* ln, uint8_t* flags, size_t flags_bytes, int sm_count, cudaStream_t st, int* launches,
+                         const int32_t* seq_lens, const int32_t* drops, int32_t* lens_out) {
+    const Ragged rg = {seq_lens, drops, lens_out};
     if (launches) *launches = 0;
     if (B == 0) return cudaSuccess;
     const size_t per_sample = prune_scratch_per_sample(N);
@@ -547,14 +577,14 @@ cudaError_t launch_prune(const float* scores, int nparts, float* scores_out, int
             const int P = N <= 1024 ? 64 : 128, nt = N <= 1024 ? 256 : 1024, nsl = (N + P - 1) / P;
             int32_t* counts = reinterpret_cast<int32_t*>(flags);
             uint8_t* fl = flags + (size_t)nb * nsl * 4;
-            e = launch_pdl(rank_kernel, dim3(nsl, nb), dim3(nt), 0, st, sc, nparts, so, N, K, has_cls, P, fl, counts);
+            e = launch_pdl(rank_kernel, dim3(nsl, nb), dim3(nt), 0, st, sc, nparts, so, N, K, has_cls, P, fl, counts, rg, b0);
             if (e != cudaSuccess) return e;
             const long long rows = (long long)nb * K;
             const dim3 grid((unsigned)((rows + 7) / 8)), block(256);
             int32_t* rm = row_map ? row_map + k0 : nullptr;
 #define RS_GR_CASE(LT)                                                                                                  \
     launch_pdl(gather_ranked_kernel<4, LT>, grid, block, 0, st, xs, (const uint8_t*)fl, (const int32_t*)counts, nsl, P, \
-               rows, N, K, b0, row_vecs, keep_idx + k0, rm, xo, lnc)
+               rows, N, K, b0, row_vecs, keep_idx + k0, rm, xo, lnc, rg)
             if (!ln) e = RS_GR_CASE(void);
             else if (dtype == RS_BF16) e = RS_GR_CASE(__nv_bfloat16);
             else e = RS_GR_CASE(float);

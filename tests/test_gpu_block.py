@@ -351,3 +351,27 @@ def test_vit_fwd_in_place_pruning_other_scores(ctx, mode, dist):
         assert torch.equal(some[2][k], chain[2][k]), k
         assert torch.equal(some[4][k], chain[4][k]), k
     ctx.async_status()
+
+
+def test_tensor_maps_are_encoded_once_per_buffer(ctx):
+    """A repeated block call on the same buffers encodes no tensor map again (the context keeps them per
+    pointer, shape and box), and gives the same bits."""
+    import paper_2508_00367_b200 as rs
+    B, N, D, H, r = 2, 150, 256, 4, 10
+    x = synth.make_tokens(B, N, D, "bf16", seed=3).to(torch.bfloat16).cuda()
+    w = synth.make_block_weights(D, 4 * D, "bf16", seed=4)
+    dw = rs.DeviceBlockWeights(w, torch.bfloat16, ctx.device)
+    desc = ctx.block_desc(B, N, D, H, dw.D_mlp, r, torch.bfloat16)
+    ws = torch.empty(ctx.block_workspace_bytes(desc), dtype=torch.uint8, device="cuda")
+    bufs = dict(x_out=torch.empty(B, N - r, D, dtype=torch.bfloat16, device="cuda"),
+                scores=torch.empty(B, N, dtype=torch.float32, device="cuda"),
+                keep_idx=torch.empty(B, N - r, dtype=torch.int32, device="cuda"))
+    first = {k: v.clone() for k, v in ctx.block_fwd(x, dw, H, r, workspace=ws, **bufs).items()}
+    h0, m0 = ctx.tmap_cache_stats()
+    again = ctx.block_fwd(x, dw, H, r, workspace=ws, **bufs)
+    h1, m1 = ctx.tmap_cache_stats()
+    torch.cuda.synchronize()
+    assert m1 == m0 and h1 > h0, (h0, m0, h1, m1)
+    for k in first:
+        assert torch.equal(first[k], again[k]), k
+    ctx.async_status()
