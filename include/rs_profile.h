@@ -29,7 +29,7 @@ RS_API rs_status rs_timing_read(rs_ctx* ctx, void* stream, double* ms /*host[RS_
                                 long long* launches /*host[RS_K_COUNT]*/);
 
 /* Tensor maps (the TMA descriptors of the tensor-core kernels) are encoded once per (pointer,
- * shape, box) and kept in a 64-slot cache of the context.  Hits and misses so far (host counters). */
+ * shape, box) and kept in a 128-slot cache of the context.  Hits and misses so far (host counters). */
 RS_API rs_status rs_tmap_cache_stats(const rs_ctx* ctx, long long* hits /*host*/, long long* misses /*host*/);
 
 #ifdef __cplusplus

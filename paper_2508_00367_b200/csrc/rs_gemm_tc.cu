@@ -531,12 +531,19 @@ bool tc_encode_cached(rs_ctx* ctx, CUtensorMap* out, const void* base, int rank,
     unsigned long long h = (unsigned long long)(uintptr_t)base * 0x9E3779B97F4A7C15ull;
     for (int i = 0; i < rank; ++i) h = (h ^ key.dims[i] ^ ((unsigned long long)key.box[i] << 40)) * 0x9E3779B97F4A7C15ull;
     h ^= (unsigned long long)swizzle_bytes << 8 | (unsigned long long)dtype;
-    rs_tmap_slot& slot = ctx->tmaps[(h >> 32) % kTmapSlots];
-    if (slot.valid && memcmp(&slot.key, &key, sizeof(key)) == 0) {
-        *out = slot.map;
-        ctx->tmap_hits += 1;
-        return true;
+    // eight neighbouring slots are probed; a new map takes the first free one of them, else the home slot
+    const unsigned home = (unsigned)((h >> 32) % kTmapSlots);
+    rs_tmap_slot* free_slot = nullptr;
+    for (unsigned pr = 0; pr < 8; ++pr) {
+        rs_tmap_slot& c = ctx->tmaps[(home + pr) % kTmapSlots];
+        if (c.valid && memcmp(&c.key, &key, sizeof(key)) == 0) {
+            *out = c.map;
+            ctx->tmap_hits += 1;
+            return true;
+        }
+        if (!c.valid && !free_slot) free_slot = &c;
     }
+    rs_tmap_slot& slot = free_slot ? *free_slot : ctx->tmaps[home];
     EncodeTiledFn fn = reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled);
     cuuint64_t d[4], st[3];
     cuuint32_t bx[4], estr[4] = {1, 1, 1, 1};

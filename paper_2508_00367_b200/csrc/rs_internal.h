@@ -12,7 +12,7 @@
 
 // Tensor maps are encoded once per (pointer, shape, box) and kept in the context: a block's launches
 // name the same few buffers over and over, and every cuTensorMapEncodeTiled call costs about a
-// microsecond of host time.  Direct-mapped, 64 slots; a slot is simply overwritten on a clash.
+// microsecond of host time.  128 slots, eight probed per lookup; a full neighbourhood evicts its home slot.
 struct rs_tmap_key {
     const void* base;
     unsigned long long dims[4], strides[3];
@@ -24,7 +24,7 @@ struct rs_tmap_slot {
     rs_tmap_key key;
     int valid;
 };
-enum { kTmapSlots = 64 };
+enum { kTmapSlots = 128 };
 
 struct rs_ctx {
     int device;
