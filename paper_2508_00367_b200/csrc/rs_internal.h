@@ -96,7 +96,7 @@ cudaError_t launch_residual_score(const float* m, const float* x_prime, const vo
 // from which the score is finished here (and written to scores_out when non-null).
 // row_map (optional, [B, K] int32): flat source row b * N + keep_idx[b, j] of every kept token, with
 // which the next block reads the un-pruned rows in place.
-// flags / flags_bytes: 4-byte aligned scratch between the ranking kernel and the row kernel (a byte
+// flags / flags_bytes: 4-byte aligned scratch between the flag kernel and the row kernel (a byte
 // per token and a count per 64 or 128 tokens; with less than the whole batch needs, the batch is
 // processed in several passes, with less than one sample needs the radix kernel runs instead).
 // *launches (optional) receives the number of kernels launched.
@@ -110,8 +110,8 @@ bool ln_fusable(rs_dtype dtype, int D);   // the row fits the registers of one w
 // x_out may be null when ln is given: only the normalised rows are written (no dense copy).
 cudaError_t launch_gather(rs_dtype dtype, const void* x, const int32_t* keep_idx, int B, int N, int K,
                           int D, void* x_out, const LnFuse* ln /*null: none*/, cudaStream_t st);
-// Selection, index lists and the rows' move (N <= 4608 and something is dropped): a ranking kernel
-// spread over the grid (a CTA per 64 or 128 tokens of a sample), then a warp per kept row.
+// Selection, index lists and the rows' move (N <= 4608 and something is dropped): a kernel that finds
+// the cut of every sample and flags its kept tokens (a CTA per sample), then a warp per kept row.
 // x null: indices only.  x given: x_out (dense copy) and / or ln (normalised rows) must be given.
 bool prune_fusable(int N, int K, size_t flags_bytes);
 cudaError_t launch_prune(const float* scores, int nparts, float* scores_out, int B, int N, int K, int has_cls,

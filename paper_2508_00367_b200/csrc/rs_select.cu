@@ -225,6 +225,7 @@ __device__ __forceinline__ void copy_row(const uint4* __restrict__ src, long lon
 // slice; gather_ranked_kernel gives every kept row a warp, which finds its token from the counts and
 // flags, writes the index lists and moves the row.
 constexpr int kPruneMaxN = 4608;
+constexpr int kRankMaxN = 2048;      // up to here the N^2 ranking spread over the grid beats the per-sample search
 
 // Forms the N orderable keys of sample b in shared memory (finishing the scores from the GEMM's
 // partial sums when they arrive that way); the scores of tokens [w0, w1) are also written out.
@@ -297,13 +298,97 @@ rank_kernel(const float* __restrict__ scores, int nparts, float* __restrict__ sc
     __syncthreads();
     uint8_t* fb = flags + (long long)b * N;
     // (the stride between samples stays N; only the first n_b keys take part)
-    rank_slice(keys, n_b, k_b, has_cls ? 1 : 0, i0, P, [&](int i, uint8_t f) { fb[i] = f; if (f) atomicAdd(&kept_here, 1); });
+    int mine = 0;                                        // this thread's kept tokens (at most one per pass)
+    rank_slice(keys, n_b, k_b, has_cls ? 1 : 0, i0, P, [&](int i, uint8_t f) { fb[i] = f; mine += f; });
     for (int i = max(i0, n_b) + (int)threadIdx.x; i < min(i0 + P, N); i += blockDim.x) fb[i] = 0;
+    mine = __reduce_add_sync(0xffffffffu, mine);
+    if ((threadIdx.x & 31) == 0 && mine) atomicAdd(&kept_here, mine);
     __syncthreads();
     if (threadIdx.x == 0) counts[(long long)b * gridDim.x + blockIdx.x] = kept_here;
 }
 
-// The rows of the kept tokens after rank_kernel: one warp per output row (b, r), eight rows per
+// Keep flags of one sample, one CTA per sample, O(N) work per step (sequences over kRankMaxN
+// tokens): the key t of the last token that makes the cut is found by binary search over the 32 bits
+// of the key space (the largest t with at least `want` keys >= t; a block-wide count per bit, one
+// counting barrier per candidate slot of a thread), tokens with a larger key are kept and the ties at
+// t go to the lowest indices (a prefix count).  The same kept set as ranking every token against
+// every other, without the N^2 comparisons.  Same outputs as rank_kernel: a flag per token and the
+// number of kept tokens of every P-token slice in counts[b, 0 .. nsl).
+__global__ void __launch_bounds__(1024)
+flag_kernel(const float* __restrict__ scores, int nparts, float* __restrict__ scores_out, int N, int K, int has_cls,
+            int P, int nsl, uint8_t* __restrict__ flags, int32_t* __restrict__ counts, const Ragged rg, int b0) {
+    __shared__ uint32_t keys[kPruneMaxN];
+    __shared__ __align__(16) uint8_t sflags[kPruneMaxN];
+    __shared__ int wsum[32];
+    __shared__ int sh_total;
+    grid_dep_launch();
+    grid_dep_wait();
+    const int b = blockIdx.x, tid = threadIdx.x, nt = blockDim.x;
+    int n_b, k_b;
+    sample_counts(rg, b0 + b, N, K, &n_b, &k_b);
+    const int first = has_cls ? 1 : 0, want = k_b - first;
+    load_keys(scores, nparts, scores_out, b, N, 0, N, keys);
+    __syncthreads();
+    // this thread's candidates, strided over the sample (at most kKeysPerThread each), in registers
+    constexpr int kKeysPerThread = (kPruneMaxN + 1023) / 1024;
+    uint32_t kreg[kKeysPerThread];
+    bool kval[kKeysPerThread];
+#pragma unroll
+    for (int e = 0; e < kKeysPerThread; ++e) {
+        const int i = first + tid + e * nt;
+        kval[e] = i < n_b;
+        kreg[e] = kval[e] ? keys[i] : 0u;
+    }
+    const int kpt = (n_b - first + nt - 1) / nt;         // candidate slots in use (the same for every thread)
+    uint32_t t = 0;
+    int need_eq = 0;
+    if (want > 0) {
+        for (int bit = 31; bit >= 0; --bit) {
+            const uint32_t cand = t | (1u << bit);
+            int total = 0;
+#pragma unroll
+            for (int e = 0; e < kKeysPerThread; ++e)
+                if (e < kpt) total += __syncthreads_count(kval[e] && kreg[e] >= cand);
+            if (total >= want) t = cand;
+        }
+        int gt = 0;
+#pragma unroll
+        for (int e = 0; e < kKeysPerThread; ++e)
+            if (e < kpt) gt += __syncthreads_count(kval[e] && kreg[e] > t);
+        need_eq = want - gt;                             // ties at t that are kept, lowest indices first
+    }
+    // flags over contiguous per-thread chunks, so that the ties' prefix count runs in index order
+    const int chunk = (N + nt - 1) / nt;
+    const int lo = min(tid * chunk, N), hi = min(lo + chunk, N);
+    int eq_cnt = 0;
+    if (want > 0)
+        for (int i = max(lo, first); i < min(hi, n_b); ++i) eq_cnt += keys[i] == t;
+    int eq_rank = block_exclusive_scan(eq_cnt, wsum, &sh_total);
+    uint8_t* fb = flags + (long long)b * N;
+    for (int i = lo; i < hi; ++i) {
+        bool keep = false;
+        if (i < first) keep = true;
+        else if (i < n_b && want > 0) {
+            const uint32_t k = keys[i];
+            keep = k > t;
+            if (k == t) { keep = eq_rank < need_eq; ++eq_rank; }
+        }
+        fb[i] = keep ? 1 : 0;
+        sflags[i] = keep ? 1 : 0;
+    }
+    __syncthreads();
+    // kept tokens per slice: a thread per slice adds up its P flag bytes (four at a time)
+    for (int sl = tid; sl < nsl; sl += nt) {
+        const int i0 = sl * P, i1 = min(i0 + P, N);
+        int c = 0;
+        int i = i0;
+        for (; i + 4 <= i1; i += 4) c += (int)((*reinterpret_cast<const uint32_t*>(sflags + i) * 0x01010101u) >> 24);
+        for (; i < i1; ++i) c += sflags[i];
+        counts[(long long)b * nsl + sl] = c;
+    }
+}
+
+// The rows of the kept tokens after rank_kernel or flag_kernel: one warp per output row (b, r), eight rows per
 // CTA, no block-wide step.  The warp adds up the slice counts of its sample (two slices per lane,
 // at most 64 slices) to find the slice that holds the r-th kept token, then the token inside the
 // slice from its flags; it writes keep_idx and row_map for its row and moves the row: the dense
@@ -577,7 +662,12 @@ cudaError_t launch_prune(const float* scores, int nparts, float* scores_out, int
             const int P = N <= 1024 ? 64 : 128, nt = N <= 1024 ? 256 : 1024, nsl = (N + P - 1) / P;
             int32_t* counts = reinterpret_cast<int32_t*>(flags);
             uint8_t* fl = flags + (size_t)nb * nsl * 4;
-            e = launch_pdl(rank_kernel, dim3(nsl, nb), dim3(nt), 0, st, sc, nparts, so, N, K, has_cls, P, fl, counts, rg, b0);
+            // (the ranking spread over the grid is the faster of the two up to kRankMaxN tokens -- 10 against
+            // 14 us at 577 tokens, 17 against 20 at 1729 -- the per-sample search beyond: 31 against 57 us at 4097)
+            if (N <= kRankMaxN)
+                e = launch_pdl(rank_kernel, dim3(nsl, nb), dim3(nt), 0, st, sc, nparts, so, N, K, has_cls, P, fl, counts, rg, b0);
+            else
+                e = launch_pdl(flag_kernel, dim3(nb), dim3(1024), 0, st, sc, nparts, so, N, K, has_cls, P, nsl, fl, counts, rg, b0);
             if (e != cudaSuccess) return e;
             const long long rows = (long long)nb * K;
             const dim3 grid((unsigned)((rows + 7) / 8)), block(256);
