@@ -106,9 +106,17 @@ select_kernel(const float* __restrict__ scores, int nparts, float* __restrict__ 
         for (int shift = 24; shift >= 0; shift -= 8) {
             if (tid < 256) hist[tid] = 0;
             __syncthreads();
-            for (int i = first + tid; i < N; i += kSelThreads) {
-                const uint32_t k = keys[i];
-                if ((k & mask) == prefix) atomicAdd(&hist[(k >> shift) & 255u], 1);
+            // Scores of one sample lie close together, so most keys share their upper bytes and one bin
+            // takes almost every increment of a pass: lanes with the same bin add once, through one of them.
+            for (int i0 = first; i0 < N; i0 += kSelThreads) {
+                const int i = i0 + tid;
+                uint32_t bin = 256u;                           // not a candidate of this pass
+                if (i < N) {
+                    const uint32_t k = keys[i];
+                    if ((k & mask) == prefix) bin = (k >> shift) & 255u;
+                }
+                const unsigned peers = __match_any_sync(0xffffffffu, bin);
+                if (bin < 256u && (tid & 31) == __ffs(peers) - 1) atomicAdd(&hist[bin], __popc(peers));
             }
             __syncthreads();
             if (tid < 32) {                // warp 0: walk the bins from the top
@@ -307,8 +315,9 @@ rank_kernel(const float* __restrict__ scores, int nparts, float* __restrict__ sc
     if (threadIdx.x == 0) counts[(long long)b * gridDim.x + blockIdx.x] = kept_here;
 }
 
-// Keep flags of one sample, one CTA per sample, O(N) work per step (sequences over kRankMaxN
-// tokens): the key t of the last token that makes the cut is found by binary search over the 32 bits
+// Keep flags of one sample, one CTA per sample, O(N) work per step (per-sample token counts over
+// kRankMaxN tokens; with a common count the radix kernel below and the plain row kernel are faster
+// there): the key t of the last token that makes the cut is found by binary search over the 32 bits
 // of the key space (the largest t with at least `want` keys >= t; a block-wide count per bit, one
 // counting barrier per candidate slot of a thread), tokens with a larger key are kept and the ties at
 // t go to the lowest indices (a prefix count).  The same kept set as ranking every token against
@@ -625,7 +634,9 @@ cudaError_t launch_select(const float* scores, int nparts, float* scores_out, in
 }
 
 bool prune_fusable(int N, int K, size_t flags_bytes) {
-    return N <= kPruneMaxN && K < N && flags_bytes >= prune_scratch_per_sample(N);
+    // (beyond kRankMaxN tokens the radix selection and the plain row kernel are the faster pair: 24
+    // against 31 us at 4097 tokens, B = 4)
+    return N <= kRankMaxN && K < N && flags_bytes >= prune_scratch_per_sample(N);
 }
 
 bool ln_fusable(rs_dtype dtype, int D) { return (size_t)D * dtype_size(dtype) / 16 <= 32 * 4; }
@@ -663,7 +674,8 @@ cudaError_t launch_prune(const float* scores, int nparts, float* scores_out, int
             int32_t* counts = reinterpret_cast<int32_t*>(flags);
             uint8_t* fl = flags + (size_t)nb * nsl * 4;
             // (the ranking spread over the grid is the faster of the two up to kRankMaxN tokens -- 10 against
-            // 14 us at 577 tokens, 17 against 20 at 1729 -- the per-sample search beyond: 31 against 57 us at 4097)
+            // 14 us at 577 tokens, 17 against 20 at 1729 -- the per-sample search beyond: 31 against 57 us at 4097;
+            // only batches with per-sample counts come here with more than kRankMaxN tokens)
             if (N <= kRankMaxN)
                 e = launch_pdl(rank_kernel, dim3(nsl, nb), dim3(nt), 0, st, sc, nparts, so, N, K, has_cls, P, fl, counts, rg, b0);
             else
