@@ -103,6 +103,9 @@ rs_status rs_create(rs_ctx** out, int device) {
     const char* no_tc = getenv("RS_DISABLE_TC");
     ctx->encode_tiled = rs::tc_get_encode_fn();
     ctx->use_tc = (ctx->encode_tiled != nullptr) && !(no_tc && no_tc[0] == '1');
+    // RS_ATTN_KERNEL=2 / 3 pins the attention kernel (cross-check of the two against each other)
+    const char* ak = getenv("RS_ATTN_KERNEL");
+    ctx->attn_kernel = ak && (ak[0] == '2' || ak[0] == '3') ? ak[0] - '0' : 0;
     const char* req = getenv("RS_REQUIRE_TC");
     ctx->require_tc = req && req[0] == '1';
     *out = ctx;

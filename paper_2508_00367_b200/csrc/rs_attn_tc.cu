@@ -22,6 +22,7 @@
 #include <tuple>
 
 #include "rs_internal.h"
+#include "rs_attn.cuh"
 #include "rs_device.cuh"
 #include "rs_once.h"
 #include "rs_tc.cuh"
@@ -31,6 +32,7 @@ namespace rs {
 namespace {
 
 using namespace tc;
+using namespace attn;
 
 constexpr int BQ = 128, BKV = 128, DH = 64;
 constexpr int TILE_BYTES = 128 * DH * 2;        // 16 KB: a [128, 64] bf16 tile
@@ -104,43 +106,6 @@ __device__ __forceinline__ int next_item(const AttnArgs& a, int w, int stride) {
     if (!a.lens) return w;
     while (w < a.n_items && decode_item(a, w).ng == 0) w += stride;
     return w;
-}
-
-__device__ __forceinline__ float ex2(float x) {
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-
-__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
-    __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
-    return *reinterpret_cast<uint32_t*>(&h);
-}
-
-__device__ __forceinline__ float max3(float a, float b, float c) {
-    float r;
-    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
-    return r;
-}
-
-// Packed fp32 pairs (two lanes of arithmetic per instruction on sm_100).
-__device__ __forceinline__ uint64_t pack2(float a, float b) {
-    uint64_t r;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
-    return r;
-}
-__device__ __forceinline__ void unpack2(uint64_t v, float& a, float& b) {
-    asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v));
-}
-__device__ __forceinline__ uint64_t ffma2(uint64_t a, uint64_t b, uint64_t c) {
-    uint64_t r;
-    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
-    return r;
-}
-__device__ __forceinline__ uint64_t fadd2(uint64_t a, uint64_t b) {
-    uint64_t r;
-    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-    return r;
 }
 
 // Maximum of the first NC values of a row of S held in registers.  MASK 0: all NC are keys.
@@ -572,24 +537,47 @@ cudaError_t launch_attn_tc(rs_ctx* ctx, const rs_attn_desc& d, const void* q, co
         };
         // (a host loop over the items for every candidate: the answer is remembered per shape)
         static std::mutex memo_mu;
-        static std::map<std::tuple<long long, int, int>, long long> memo;
-        long long best_hs = 0, best = -1;
+        struct Plan { long long best_hs; int three, wrap3; };
+        static std::map<std::tuple<long long, int, int>, Plan> memo;
+        Plan plan = {0, 0, 0};
         const auto key = std::make_tuple(BH, d.N, G);
         std::unique_lock<std::mutex> lock(memo_mu);
         const auto hit = memo.find(key);
         if (hit != memo.end()) {
-            best_hs = hit->second;
+            plan = hit->second;
         } else {
             long long hs_max = (2ll * G + nt - 1) / nt + 1;    // enough single tiles for two rounds
             if (hs_max > BH) hs_max = BH;
-            if (BH * per <= 200000)
+            long long best = -1;
+            if (BH * per <= 200000) {
                 for (long long hs = 0; hs <= hs_max; ++hs) {
                     const long long m = makespan(hs);
-                    if (best < 0 || m < best) { best = m; best_hs = hs; }
+                    if (best < 0 || m < best) { best = m; plan.best_hs = hs; }
                 }
-            memo[key] = best_hs;
+                // This kernel or the one with three query tiles per CTA (rs_attn_tc3.cu)?  Both are
+                // paced by the longest CTA: its items (in tenths) times the key tiles of an item,
+                // plus a cost per item; microseconds fitted to CUDA-event times of thirteen shapes
+                // from N = 197 to 4097 (worst error 6 % and 9 %).  Sequences with lengths of their
+                // own stay here.
+                int wrap3 = 0;
+                const long long u3 = attn_tc3_plan(BH, d.N, G, &wrap3);
+                const double t2 = best / 10.0 * (((d.N + BKV - 1) / BKV) * 1.505 + 2.51) + 2.32;
+                const double t3 = u3 / 10.0 * (((d.N + 63) / 64) * 1.136 + 1.00) + 6.71;
+                plan.three = t3 < t2;
+                plan.wrap3 = wrap3;
+            }
+            memo[key] = plan;
         }
         lock.unlock();
+        const int force = ctx->attn_kernel;                    // RS_ATTN_KERNEL=2 / 3: one kernel for every shape it takes
+        if (!seq_lens && (force == 3 || (force != 2 && plan.three))) {
+            CUtensorMap tmK3, tmV3;
+            if (!make_tmap_qkv(ctx, &tmK3, k, d.B, d.N, d.H, d.k_batch_stride, d.k_row_stride, d.k_head_stride, 64) ||
+                !make_tmap_qkv(ctx, &tmV3, v, d.B, d.N, d.H, d.v_batch_stride, d.v_row_stride, d.v_head_stride, 64))
+                return cudaErrorInvalidValue;
+            return launch_attn_tc3(ctx, d, tmQ, tmK3, tmV3, tmO, plan.wrap3, st);
+        }
+        const long long best_hs = plan.best_hs;
         args.n_pair_items = (int)((BH - best_hs) * per);
         args.first_single_bh = (int)(BH - best_hs);
         items = (BH - best_hs) * per + best_hs * nt;

@@ -33,6 +33,7 @@ struct rs_ctx {
     int require_tc;        // RS_REQUIRE_TC=1: a bf16 shape the tensor-core kernels cannot take is an error
     int* d_status;         // device status word (0 = ok), first bytes of a small allocation made by rs_create
     unsigned char* d_flags; // keep-flag scratch of rs_topk_compact (kFlagScratch bytes, same allocation)
+    int attn_kernel;        // RS_ATTN_KERNEL: 0 the faster attention kernel per shape (cost model), 2 / 3 always that one
     long long launches;    // kernels launched through this context
     void* encode_tiled;    // cuTensorMapEncodeTiled entry point (driver API), or null
     int timing;            // bracket launches with events
@@ -155,6 +156,10 @@ cudaError_t launch_gemm_tc(rs_ctx* ctx, int epi, const void* A, const void* W, c
 
 // ---- tcgen05 attention (rs_attn_tc.cu): bf16, head dimension 64 ----
 bool attn_tc_supported(const rs_attn_desc& d);
+// Three query tiles per CTA (rs_attn_tc3.cu), N > 128: the longest CTA's load under its item list, and the launch.
+long long attn_tc3_plan(long long BH, int N, int G, int* wrap);
+cudaError_t launch_attn_tc3(rs_ctx* ctx, const rs_attn_desc& d, const CUtensorMap& tmQ, const CUtensorMap& tmK,
+                            const CUtensorMap& tmV, const CUtensorMap& tmO, int wrap, cudaStream_t st);
 // seq_lens (optional, dev [B]): sample b attends over its first seq_lens[b] tokens only.
 cudaError_t launch_attn_tc(rs_ctx* ctx, const rs_attn_desc& d, const void* q, const void* k, const void* v,
                            void* out, const int32_t* seq_lens, cudaStream_t st);

@@ -114,6 +114,8 @@ rs_status rs_block_fwd_static(const rs_block_desc* desc, const rs_block_weights*
     ctx.d_status = status;          // same kernels as rs_block_fwd, tensor cores included
     ctx.encode_tiled = encode;
     const char* no_tc = getenv("RS_DISABLE_TC");
+    const char* ak = getenv("RS_ATTN_KERNEL");
+    ctx.attn_kernel = ak && (ak[0] == '2' || ak[0] == '3') ? ak[0] - '0' : 0;
     ctx.use_tc = (encode != nullptr) && !(no_tc && no_tc[0] == '1');
     st = rs_block_fwd(&ctx, desc, weights, x, x_out, scores, keep_idx, x_full, scratch, RS_STATIC_SCRATCH_BYTES,
                       stream);

@@ -250,6 +250,53 @@ def test_attn_full_size_video_shape_sampled(ctx):
     parity.check_float(got[:, rows], orc.round_to(want, "bf16"), "bf16", rounded_output=True)
 
 
+@pytest.fixture(scope="module")
+def pinned():
+    """A context per attention kernel: RS_ATTN_KERNEL is read when the context is made."""
+    import os
+    import paper_2508_00367_b200 as rs
+    made = {}
+    for kernel in (2, 3):
+        os.environ["RS_ATTN_KERNEL"] = str(kernel)
+        try:
+            made[kernel] = rs.Context(0)
+        finally:
+            del os.environ["RS_ATTN_KERNEL"]
+    yield made
+    for c in made.values():
+        c.async_status()
+        c.close()
+
+
+# Both attention kernels on every shape either takes: two query tiles per CTA (kernel 2) and three with
+# 64-key tiles (kernel 3).  Token counts around the tile edges (128 rows, 64 keys, groups of three tiles);
+# the last two batches are large enough that the leftover tiles of the heads go to the CTAs which the
+# last round of groups left out, two to some of them (170 heads), or take turns over all CTAs (200).
+@pytest.mark.parametrize("kernel", [2, 3])
+@pytest.mark.parametrize("B,N,H", [(1, 129, 2), (1, 192, 1), (1, 193, 1), (1, 257, 2), (2, 384, 3), (1, 385, 2),
+                                   (1, 513, 4), (1, 577, 4), (1, 1099, 1), (10, 513, 17), (8, 513, 25)])
+def test_attn_each_kernel_pinned(pinned, kernel, B, N, H):
+    qkv = _tok((B, N, 3, H, 64), torch.bfloat16, N * 11 + H)
+    dq = qkv.cuda()
+    got = pinned[kernel].attn_fwd(dq[:, :, 0], dq[:, :, 1], dq[:, :, 2]).cpu().double().numpy()
+    f = qkv.double().numpy()
+    want = orc.attn(f[:, :, 0], f[:, :, 1], f[:, :, 2]).reshape(B, N, H * 64)
+    parity.check_float(got, orc.round_to(want, "bf16"), "bf16", rounded_output=True)
+
+
+@pytest.mark.parametrize("kernel", [2, 3])
+def test_attn_each_kernel_full_size_video_shape_sampled(pinned, kernel):
+    B, N, H = 1, 4097, 2
+    qkv = _tok((B, N, 3, H, 64), torch.bfloat16, 99)
+    dq = qkv.cuda()
+    got = pinned[kernel].attn_fwd(dq[:, :, 0], dq[:, :, 1], dq[:, :, 2]).cpu().double().numpy()
+    f = qkv.double().numpy()
+    rows = np.unique(np.concatenate([np.arange(0, 3), np.arange(126, 131), np.arange(382, 387), np.arange(N - 3, N),
+                                     np.random.default_rng(2).integers(0, N, 48)]))
+    want = orc.attn(f[:, :, 0], f[:, :, 1], f[:, :, 2]).reshape(B, N, H * 64)[:, rows]
+    parity.check_float(got[:, rows], orc.round_to(want, "bf16"), "bf16", rounded_output=True)
+
+
 def test_attn_rejects_bad_arguments(ctx):
     import paper_2508_00367_b200 as rs
     q = torch.zeros(1, 4, 2, 32, device="cuda")

@@ -38,9 +38,19 @@ def test_attn_ragged_per_sample_lengths(ctx, N, H, lens):
     for b, n in enumerate(lens):
         want = orc.attn(f[b:b + 1, :n, 0], f[b:b + 1, :n, 1], f[b:b + 1, :n, 2]).reshape(n, H * 64)
         parity.check_float(out[b, :n].double().numpy(), orc.round_to(want, "bf16"), "bf16", rounded_output=True)
-    # the same call with every length = N is the dense entry point, bit for bit
-    full = ctx.attn_fwd_ragged(dq[:, :, 0], dq[:, :, 1], dq[:, :, 2], _i32([N] * B))
-    assert torch.equal(full, ctx.attn_fwd(dq[:, :, 0], dq[:, :, 1], dq[:, :, 2]))
+    # the same call with every length = N is the dense entry point, bit for bit, when the dense call runs the
+    # kernel that takes per-sample lengths (the dense entry point may pick the other kernel for a shape)
+    import os
+    import paper_2508_00367_b200 as rs
+    os.environ["RS_ATTN_KERNEL"] = "2"
+    try:
+        two = rs.Context(0)
+    finally:
+        del os.environ["RS_ATTN_KERNEL"]
+    full = two.attn_fwd_ragged(dq[:, :, 0], dq[:, :, 1], dq[:, :, 2], _i32([N] * B))
+    assert torch.equal(full, two.attn_fwd(dq[:, :, 0], dq[:, :, 1], dq[:, :, 2]))
+    two.async_status()
+    two.close()
 
 
 @pytest.mark.parametrize("N,D,dtype", [(197, 64, torch.bfloat16), (600, 32, torch.float32), (1500, 8, torch.float32)])

@@ -63,13 +63,21 @@ def test_static_scratch_block_matches_workspace_block(dtype, B, N, D, H, r):
     keep = torch.empty(B, K, dtype=torch.int32, device="cuda")
     err = ctypes.create_string_buffer(256)
     stream = ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+    # (Python's collector is kept out of the measured stretch: tensors that earlier tests left in
+    # reference cycles would otherwise be returned to torch's allocator in the middle of it.)
+    import gc
+    gc.collect()
     torch.cuda.synchronize()
-    free0, alloc0, reserved0 = torch.cuda.mem_get_info()[0], torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
-    st = lib.rs_block_fwd_static(ctypes.byref(desc), ctypes.byref(dw.struct), x.data_ptr(), x_out.data_ptr(),
-                                 scores.data_ptr(), keep.data_ptr(), None, stream, err, 256)
-    assert st == 0, err.value
-    assert lib.rs_static_async_status(stream, err, 256) == 0, err.value
-    assert torch.cuda.mem_get_info()[0] == free0
-    assert torch.cuda.memory_allocated() == alloc0 and torch.cuda.memory_reserved() == reserved0
+    gc.disable()
+    try:
+        free0, alloc0, reserved0 = torch.cuda.mem_get_info()[0], torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
+        st = lib.rs_block_fwd_static(ctypes.byref(desc), ctypes.byref(dw.struct), x.data_ptr(), x_out.data_ptr(),
+                                     scores.data_ptr(), keep.data_ptr(), None, stream, err, 256)
+        assert st == 0, err.value
+        assert lib.rs_static_async_status(stream, err, 256) == 0, err.value
+        assert torch.cuda.mem_get_info()[0] == free0
+        assert torch.cuda.memory_allocated() == alloc0 and torch.cuda.memory_reserved() == reserved0
+    finally:
+        gc.enable()
     assert torch.equal(x_out, want[1]["x_out"]) and torch.equal(keep, want[1]["keep_idx"]) and torch.equal(scores, want[1]["scores"])
     ctx.close()
