@@ -89,7 +89,11 @@ RS_API int rs_linear_uses_tensor_cores(const rs_ctx* ctx, rs_dtype dtype, long l
  * h*head_stride + c  (strides in elements), so the three may alias one packed
  * [B, N, 3, H, 64] buffer.  Strides must be multiples of 8 elements.
  * out (dev): [B, N, H*head_dim] contiguous, same dtype.  No [N, N] buffer is
- * ever written to global memory.  scale == 0 selects 1/sqrt(head_dim). */
+ * ever written to global memory.  scale == 0 selects 1/sqrt(head_dim).
+ * Two tensor-core kernels serve bf16 (two or three 128-row query tiles per thread block); the
+ * library picks the one its cost model expects to be faster for B, N and H, so the result for
+ * one shape is reproducible bit for bit but the rounding order may differ between shapes.
+ * RS_ATTN_KERNEL=2 or =3 in the environment at rs_create pins one of them where it applies. */
 typedef struct {
     rs_dtype dtype;
     int B, N, H, head_dim;
