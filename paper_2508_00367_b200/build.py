@@ -33,7 +33,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     flags = [f for f in NVCC_FLAGS if f != "--use_fast_math=false"]
-    cmd = [nvcc, *flags, "-shared", "-I", INCLUDE, "-I", CSRC, "-o", LIB, *sources(), "-lcudart"]
+    cmd = [nvcc, *flags, "-shared", "-I", INCLUDE, "-I", CSRC, "-o", LIB, *sources(), "-lcudart", "-ldl"]
     if verbose:
         cmd.insert(1, "-Xptxas=-v")
         print(" ".join(cmd))

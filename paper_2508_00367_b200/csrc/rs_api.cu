@@ -6,6 +6,8 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "rs_internal.h"
 #include <vector>
 
@@ -28,12 +30,19 @@ rs_status cuda_fail(rs_ctx* ctx, cudaError_t e, const char* what) {
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 bool valid_dtype(int t) { return t == RS_F32 || t == RS_BF16; }
 
-// Launch wrapper: counts the launch and, when timing is on, brackets it with events.
+// Launch wrapper: counts the launch and, when timing is on, brackets it with events.  RS_LOG=1
+// prints a line per launch on stderr, RS_NVTX=1 wraps the host side of each launch in an NVTX range
+// named after the step (both read at rs_create; host-side only, nothing changes in the kernels).
 #define RS_CHECK_LAUNCH(ctx, cls, st, expr, what)                                  \
     do {                                                                           \
         const bool timed__ = (ctx)->timing && (ctx)->n_events < kMaxTimed;         \
         if (timed__) cudaEventRecord((ctx)->ev[2 * (ctx)->n_events], (st));        \
+        if ((ctx)->nvtx) nvtxRangePushA(what);                                     \
         cudaError_t e__ = (expr);                                                  \
+        if ((ctx)->nvtx) nvtxRangePop();                                           \
+        if ((ctx)->log)                                                            \
+            fprintf(stderr, "rs: launch %lld class %d: %s -> %s\n", (ctx)->launches, (int)(cls), what, \
+                    e__ == cudaSuccess ? "ok" : cudaGetErrorString(e__));          \
         if (e__ != cudaSuccess) return cuda_fail(ctx, e__, what);                  \
         if (timed__) {                                                             \
             cudaEventRecord((ctx)->ev[2 * (ctx)->n_events + 1], (st));             \
@@ -106,6 +115,10 @@ rs_status rs_create(rs_ctx** out, int device) {
     // RS_ATTN_KERNEL=2 / 3 pins the attention kernel (cross-check of the two against each other)
     const char* ak = getenv("RS_ATTN_KERNEL");
     ctx->attn_kernel = ak && (ak[0] == '2' || ak[0] == '3') ? ak[0] - '0' : 0;
+    const char* lg = getenv("RS_LOG");
+    ctx->log = lg && lg[0] == '1';
+    const char* nv = getenv("RS_NVTX");
+    ctx->nvtx = nv && nv[0] == '1';
     const char* req = getenv("RS_REQUIRE_TC");
     ctx->require_tc = req && req[0] == '1';
     *out = ctx;

@@ -33,6 +33,7 @@ struct rs_ctx {
     int require_tc;        // RS_REQUIRE_TC=1: a bf16 shape the tensor-core kernels cannot take is an error
     int* d_status;         // device status word (0 = ok), first bytes of a small allocation made by rs_create
     unsigned char* d_flags; // keep-flag scratch of rs_topk_compact (kFlagScratch bytes, same allocation)
+    int log, nvtx;          // RS_LOG=1: a line per launch on stderr; RS_NVTX=1: an NVTX range around each launch call
     int attn_kernel;        // RS_ATTN_KERNEL: 0 the faster attention kernel per shape (cost model), 2 / 3 always that one
     long long launches;    // kernels launched through this context
     void* encode_tiled;    // cuTensorMapEncodeTiled entry point (driver API), or null

@@ -297,6 +297,31 @@ def test_attn_each_kernel_full_size_video_shape_sampled(pinned, kernel):
     parity.check_float(got[:, rows], orc.round_to(want, "bf16"), "bf16", rounded_output=True)
 
 
+def test_launch_log_and_nvtx_ranges_change_nothing(ctx, capfd):
+    """RS_LOG=1 prints one line per kernel launch on stderr and RS_NVTX=1 wraps each launch call in a
+    range (both are host-side and read when the context is made); the results are the same bits."""
+    import os
+    import paper_2508_00367_b200 as rs
+    os.environ["RS_LOG"] = "1"
+    os.environ["RS_NVTX"] = "1"
+    try:
+        noisy = rs.Context(0)
+    finally:
+        del os.environ["RS_LOG"], os.environ["RS_NVTX"]
+    qkv = _tok((2, 300, 3, 2, 64), torch.bfloat16, 5).cuda()
+    a, b = _tok((3, 50, 64), torch.bfloat16, 6).cuda(), _tok((3, 50, 64), torch.bfloat16, 7).cuda()
+    capfd.readouterr()
+    n0 = noisy.launch_count()
+    got = noisy.attn_fwd(qkv[:, :, 0], qkv[:, :, 1], qkv[:, :, 2])
+    sc = noisy.shift_score(a, b)
+    noisy.async_status()
+    lines = [ln for ln in capfd.readouterr().err.splitlines() if ln.startswith("rs: launch ")]
+    assert len(lines) == noisy.launch_count() - n0 == 2 and all(ln.endswith("-> ok") for ln in lines), lines
+    assert torch.equal(got, ctx.attn_fwd(qkv[:, :, 0], qkv[:, :, 1], qkv[:, :, 2]))
+    assert torch.equal(sc, ctx.shift_score(a, b))
+    noisy.close()
+
+
 def test_attn_rejects_bad_arguments(ctx):
     import paper_2508_00367_b200 as rs
     q = torch.zeros(1, 4, 2, 32, device="cuda")
