@@ -271,6 +271,20 @@ RS_API rs_status rs_block_fwd_ragged(rs_ctx* ctx, const rs_block_desc* desc /*ho
                                      const int32_t* seq_lens, const int32_t* drops, int32_t* lens_out,
                                      void* workspace, size_t workspace_bytes, void* stream);
 
+/* rs_vit_fwd_ragged: the layer loop on a batch with per-sample token counts -- rs_block_fwd_ragged
+ * chained L times inside the library, the same bits as chaining the calls.  pad_drops (host[L]): the
+ * padded length shrinks from N_l to N_{l+1} = N_l - pad_drops[l] after block l (so pad_drops[l] must
+ * not exceed any sample's own drop count there, or kept tokens are cut off at the row stride).
+ * seq_lens (dev [B]): token counts entering block 0.  sample_drops (dev [L, B]): row l holds the
+ * tokens each sample drops after block l (clamped on the device like drops above).  x (dev):
+ * [B, N, D]; x_out (dev): [B, N_L, D]; keep_last (dev, optional): [B, N_L]; lens_out (dev, optional):
+ * [B] counts after the last block.  workspace: at least rs_vit_workspace_bytes(desc, pad_drops). */
+RS_API rs_status rs_vit_fwd_ragged(rs_ctx* ctx, const rs_vit_desc* desc /*host*/,
+                                   const rs_block_weights* weights /*host[L]*/, const int* pad_drops /*host[L]*/,
+                                   const void* x, void* x_out, int32_t* keep_last, const int32_t* seq_lens,
+                                   const int32_t* sample_drops, int32_t* lens_out, void* workspace,
+                                   size_t workspace_bytes, void* stream);
+
 /* ---- rs_block_fwd_static: rs_block_fwd for callers that cannot allocate ----------------
  * (The paper has no counterpart; this is a packaging variant of rs_block_fwd.)
  * Some callers have no way to obtain device memory when they reach the block:

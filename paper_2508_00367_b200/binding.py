@@ -28,7 +28,7 @@ EXPORTS = ("rs_create", "rs_destroy", "rs_last_error", "rs_async_status", "rs_us
            "rs_block_workspace_bytes", "rs_block_fwd", "rs_timing_enable", "rs_timing_read",
            "rs_static_scratch_bytes", "rs_block_fwd_static", "rs_linear_fwd", "rs_vit_workspace_bytes", "rs_vit_fwd",
            "rs_vit_fwd_taps", "rs_linewise_compact", "rs_static_async_status", "rs_linear_uses_tensor_cores",
-           "rs_block_uses_tensor_cores", "rs_attn_fwd_ragged", "rs_topk_compact_ragged", "rs_block_fwd_ragged", "rs_tmap_cache_stats")
+           "rs_block_uses_tensor_cores", "rs_attn_fwd_ragged", "rs_topk_compact_ragged", "rs_block_fwd_ragged", "rs_vit_fwd_ragged", "rs_tmap_cache_stats")
 LIN_EPILOGUE = {"bias": 0, "gelu": 1, "residual": 2}
 KERNEL_CLASSES = ("layernorm", "gemm", "attn", "score", "select", "gather")
 
@@ -148,6 +148,9 @@ def load_library() -> ctypes.CDLL:
     lib.rs_vit_fwd_taps.argtypes = [vp, ctypes.POINTER(VitDesc), ctypes.POINTER(BlockWeights), ctypes.POINTER(ci), vp,
                                     ctypes.POINTER(VitTaps), vp, ctypes.c_size_t, vp]
     lib.rs_vit_fwd_taps.restype = ci
+    lib.rs_vit_fwd_ragged.argtypes = [vp, ctypes.POINTER(VitDesc), ctypes.POINTER(BlockWeights), ctypes.POINTER(ci), vp, vp, vp,
+                                      vp, vp, vp, vp, ctypes.c_size_t, vp]
+    lib.rs_vit_fwd_ragged.restype = ci
     _lib = lib
     return lib
 
@@ -307,6 +310,31 @@ class Context:
                                                  _stream(x.device)))
         if want_full:
             res["x_full"] = x_full
+        return res
+
+    def vit_fwd_ragged(self, x: torch.Tensor, weights: Sequence["DeviceBlockWeights"], H: int, pad_drops: Sequence[int],
+                       seq_lens: torch.Tensor, sample_drops: torch.Tensor, has_cls: bool = True) -> Dict[str, torch.Tensor]:
+        """rs_vit_fwd_ragged: the layer loop on a padded batch with per-sample token counts.  sample_drops is
+        [L, B] int32 on the device.  Returns dict(x_out [B, N_L, D], keep_idx [B, N_L], lens_out [B])."""
+        assert x.is_cuda and x.is_contiguous() and len(weights) == len(pad_drops)
+        B, N, D = x.shape
+        L = len(weights)
+        assert sample_drops.dtype == torch.int32 and sample_drops.is_contiguous() and tuple(sample_drops.shape) == (L, B)
+        assert seq_lens.dtype == torch.int32 and seq_lens.numel() == B
+        desc = VitDesc(_dt(x), B, N, D, H, weights[0].D_mlp, L, int(has_cls), 0.0, 0.0, SCORE_MODE["mlp"], DIST["l2"])
+        cdrops = (ctypes.c_int * L)(*[int(r) for r in pad_drops])
+        warr = (BlockWeights * L)(*[w.struct for w in weights])
+        need = int(self.lib.rs_vit_workspace_bytes(ctypes.byref(desc), cdrops))
+        if need == 0:
+            raise RsError(1, "rs_vit_fwd_ragged: bad descriptor or schedule")
+        ws = torch.empty(need, dtype=torch.uint8, device=x.device)
+        n_out = N - sum(int(r) for r in pad_drops)
+        res = dict(x_out=torch.empty(B, n_out, D, dtype=x.dtype, device=x.device),
+                   keep_idx=torch.empty(B, n_out, dtype=torch.int32, device=x.device),
+                   lens_out=torch.empty(B, dtype=torch.int32, device=x.device))
+        self._check(self.lib.rs_vit_fwd_ragged(self.handle, ctypes.byref(desc), warr, cdrops, _ptr(x), _ptr(res["x_out"]),
+                                               _ptr(res["keep_idx"]), _ptr(seq_lens), _ptr(sample_drops), _ptr(res["lens_out"]),
+                                               _ptr(ws), ws.numel(), _stream(x.device)))
         return res
 
     # ---- rs_linear_fwd ----

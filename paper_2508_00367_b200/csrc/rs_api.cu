@@ -643,6 +643,46 @@ rs_status rs_vit_fwd_taps(rs_ctx* ctx, const rs_vit_desc* d, const rs_block_weig
     return RS_OK;
 }
 
+rs_status rs_vit_fwd_ragged(rs_ctx* ctx, const rs_vit_desc* d, const rs_block_weights* weights, const int* pad_drops,
+                            const void* x, void* x_out, int32_t* keep_last, const int32_t* seq_lens,
+                            const int32_t* sample_drops, int32_t* lens_out, void* workspace, size_t workspace_bytes,
+                            void* stream) {
+    if (!ctx) return RS_ERR_INVALID_ARG;
+    if (!d || !weights || !pad_drops || !x || !x_out || !seq_lens || !sample_drops || d->L < 1)
+        return fail(ctx, RS_ERR_INVALID_ARG, "rs_vit_fwd_ragged: null argument");
+    VitPlan p;
+    if (!valid_dtype(d->dtype) || !vit_plan(*d, pad_drops, &p))
+        return fail(ctx, RS_ERR_INVALID_ARG, "rs_vit_fwd_ragged: bad descriptor or schedule (need 0 <= pad_drops[l] <= N_l - 1)");
+    if (!workspace || workspace_bytes < p.total)
+        return fail(ctx, RS_ERR_WORKSPACE, "rs_vit_fwd_ragged: workspace of %zu bytes needed, %zu given", p.total, workspace_bytes);
+    if (reinterpret_cast<uintptr_t>(workspace) & 255u)
+        return fail(ctx, RS_ERR_INVALID_ARG, "rs_vit_fwd_ragged: workspace must be 256-byte aligned");
+    if ((reinterpret_cast<uintptr_t>(seq_lens) & 3u) || (reinterpret_cast<uintptr_t>(sample_drops) & 3u))
+        return fail(ctx, RS_ERR_INVALID_ARG, "rs_vit_fwd_ragged: misaligned count arrays");
+    char* base = (char*)workspace;
+    void* act[2] = {base + p.block_ws, base + p.block_ws + p.act_bytes};
+    // the per-sample counts between the blocks live where rs_vit_fwd keeps its row-index lists
+    int32_t* lens[2] = {(int32_t*)(base + p.block_ws + 3 * p.act_bytes), (int32_t*)(base + p.block_ws + 3 * p.act_bytes + p.map_bytes)};
+    const void* cur = x;
+    const int32_t* cur_lens = seq_lens;
+    int n = d->N;
+    for (int l = 0; l < d->L; ++l) {
+        const bool last = l == d->L - 1;
+        rs_block_desc bd = {d->dtype, d->dtype, d->B, n, d->D, d->H, d->D_mlp, pad_drops[l], d->has_cls, d->ln_eps, d->scale,
+                            d->score_mode, d->dist};
+        void* out = last ? x_out : act[l & 1];
+        int32_t* next_lens = last ? lens_out : lens[l & 1];
+        const LoopHooks hk = {nullptr, nullptr, nullptr, nullptr, true, nullptr, cur_lens, sample_drops + (size_t)l * d->B, next_lens};
+        rs_status st = block_fwd_impl(ctx, &bd, &weights[l], cur, out, nullptr, last ? keep_last : nullptr, nullptr, base,
+                                      p.block_ws, stream, &hk);
+        if (st != RS_OK) return st;
+        cur = out;
+        cur_lens = next_lens;
+        n -= pad_drops[l];
+    }
+    return RS_OK;
+}
+
 rs_status rs_vit_fwd(rs_ctx* ctx, const rs_vit_desc* d, const rs_block_weights* weights, const int* drops,
                      const void* x, void* x_out, float* scores_last, int32_t* keep_last, void* workspace,
                      size_t workspace_bytes, void* stream) {

@@ -113,6 +113,38 @@ def test_block_ragged_matches_the_oracle_per_sample(ctx):
     ctx.async_status()
 
 
+def test_vit_fwd_ragged_equals_the_chain_of_ragged_blocks(ctx):
+    """rs_vit_fwd_ragged is rs_block_fwd_ragged chained inside the library: the same bits as chaining the
+    calls (each of which is compared with the oracle above), and the counts add up."""
+    import paper_2508_00367_b200 as rs
+    N, D, H, L = 300, 256, 4, 3
+    lens = [300, 41, 129, 257, 180]
+    B = len(lens)
+    drops = [[30, 5, 10, 64, 20], [20, 0, 40, 33, 100], [0, 35, 9, 60, 7]]      # [L][B]
+    pad = [min(d) for d in drops]                                               # 5, 0, 0: the padded length 300 -> 295
+    x = synth.make_tokens(B, N, D, "bf16", seed=91)
+    for b, n in enumerate(lens):
+        x[b, n:] = 0
+    dws = [rs.DeviceBlockWeights(synth.make_block_weights(D, 4 * D, "bf16", seed=92 + l), torch.bfloat16, ctx.device)
+           for l in range(L)]
+    dx = x.to(torch.bfloat16).cuda()
+    got = ctx.vit_fwd_ragged(dx, dws, H, pad, _i32(lens), _i32(drops))
+    cur, cur_lens, n = dx, _i32(lens), N
+    for l in range(L):
+        step = ctx.block_fwd_ragged(cur, dws[l], H, cur_lens, _i32(drops[l]), n - pad[l])
+        cur, cur_lens, n = step["x_out"], step["lens_out"], n - pad[l]
+    assert torch.equal(got["x_out"], cur) and torch.equal(got["keep_idx"], step["keep_idx"])
+    assert torch.equal(got["lens_out"], cur_lens)
+    want = [max(ln - drops[0][b], 1) for b, ln in enumerate(lens)]
+    for l in (1, 2):
+        want = [max(w - min(drops[l][b], w - 1), 1) for b, w in enumerate(want)]
+    assert got["lens_out"].cpu().tolist() == want
+    for b, k in enumerate(want):
+        assert (got["x_out"][b, k:] == 0).all() and (got["keep_idx"][b, k:] == -1).all()
+        assert torch.isfinite(got["x_out"][b, :k].float()).all() and got["x_out"][b, :k].float().abs().sum() > 0
+    ctx.async_status()
+
+
 def test_ragged_rejects_what_it_cannot_run(ctx):
     import paper_2508_00367_b200 as rs
     q = torch.zeros(1, 8, 1, 64, device="cuda")                  # fp32: no tensor-core kernel
