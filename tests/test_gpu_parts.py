@@ -99,6 +99,29 @@ def test_topk_compact_bit_exact(ctx, kind, N):
             assert torch.equal(xo.cpu().view(torch.int16), ref.view(torch.int16))
 
 
+@pytest.mark.parametrize("kind", ["normal", "ties", "special"])
+def test_topk_compact_longest_sequence(ctx, kind):
+    # the largest token count the selection takes (the radix kernel's keys fill its shared memory)
+    B, N, D = 2, 32768, 8
+    s = _scores(B, N, kind, 5)
+    x = _tok((B, N, D), torch.float32, 6)
+    for r in (1, N // 3, N - 1):
+        xo, keep = ctx.topk_compact(torch.from_numpy(s).cuda(), x.cuda(), r, True)
+        want = orc.topk(s.astype(np.float64), r, True)
+        np.testing.assert_array_equal(keep.cpu().numpy(), want, err_msg=f"r={r}")
+        ref = torch.stack([x[b][torch.from_numpy(want[b]).long()] for b in range(B)])
+        assert torch.equal(xo.cpu(), ref)
+
+
+def test_attn_is_reproducible_bit_for_bit(pinned):
+    # the same call twice, each kernel: no result depends on the order in which CTAs or warps finish
+    qkv = _tok((3, 700, 3, 5, 64), torch.bfloat16, 17).cuda()
+    for c in pinned.values():
+        a = c.attn_fwd(qkv[:, :, 0], qkv[:, :, 1], qkv[:, :, 2])
+        b = c.attn_fwd(qkv[:, :, 0], qkv[:, :, 1], qkv[:, :, 2])
+        assert torch.equal(a, b)
+
+
 @pytest.mark.parametrize("dtype,D", [("f32", 384), ("bf16", 768), ("bf16", 1024), ("f32", 8)])
 def test_topk_compact_rows(ctx, dtype, D):
     B, N, r = 5, 197, 16
