@@ -330,12 +330,14 @@ def measure_workload(ctx, wl, args, dev, rank, world, headline: bool, sampler=No
             dist.barrier()
         torch.cuda.synchronize()
 
-    def timed(fn, steps):
+    def timed(fn, steps, tail=None):
         barrier()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
         for i in range(steps):
             fn(i)
+        if tail is not None:
+            tail()                        # whatever the steps left running on other streams ends inside the region
         e1.record()
         torch.cuda.synchronize()
         ms = e0.elapsed_time(e1) / steps
@@ -368,11 +370,17 @@ def measure_workload(ctx, wl, args, dev, rank, world, headline: bool, sampler=No
 
     if headline:
         # End to end: host buffers in, host buffer out, through the same public call.  The upload of
-        # step i+1 runs on a copy stream while step i computes (two device input buffers).
+        # a step's input and the download of the previous step's result run on a copy stream while
+        # a forward computes (two device input buffers; the result leaves through two device staging
+        # buffers, because the model's own output buffer is overwritten by the next forward).
         dxs = [torch.empty_like(dev_x[0]) for _ in range(2)]
-        copy_stream = torch.cuda.Stream(device=dev)
+        copy_stream = torch.cuda.Stream(device=dev)          # uploads
+        down_stream = torch.cuda.Stream(device=dev)          # downloads (a stream of their own: they wait for a forward)
         ev_in = [torch.cuda.Event() for _ in range(2)]      # upload into dxs[k] finished
         ev_free = [torch.cuda.Event() for _ in range(2)]    # forward reading dxs[k] finished
+        stage = [torch.empty_like(host_out, device=dev) for _ in range(2)]
+        ev_out = [torch.cuda.Event() for _ in range(2)]     # result copied into stage[k]
+        ev_down = [torch.cuda.Event() for _ in range(2)]    # stage[k] read out to the host
 
         def step_e2e(i):
             k = i % 2
@@ -384,13 +392,20 @@ def measure_workload(ctx, wl, args, dev, rank, world, headline: bool, sampler=No
             main.wait_event(ev_in[k])
             outs = model.forward(dxs[k], graph=use_graph)
             ev_free[k].record(main)
-            host_out.copy_(outs[-1]["x_out"], non_blocking=True)
+            main.wait_event(ev_down[k])
+            stage[k].copy_(outs[-1]["x_out"], non_blocking=True)
+            ev_out[k].record(main)
+            with torch.cuda.stream(down_stream):
+                down_stream.wait_event(ev_out[k])
+                host_out.copy_(stage[k], non_blocking=True)
+                ev_down[k].record(down_stream)
 
         for k in range(2):
             ev_free[k].record(torch.cuda.current_stream(dev))
+            ev_down[k].record(torch.cuda.current_stream(dev))
         for i in range(4):
             step_e2e(i)
-        res["ms_e2e"] = timed(step_e2e, args.steps)
+        res["ms_e2e"] = timed(step_e2e, args.steps, tail=lambda: torch.cuda.current_stream(dev).wait_stream(down_stream))
         res["h2d"] = host_x[0].numel() * host_x[0].element_size()
         res["d2h"] = host_out.numel() * host_out.element_size()
 
