@@ -316,7 +316,9 @@ def measure_workload(ctx, wl, args, dev, rank, world, headline: bool, sampler=No
 
     tdt = torch.bfloat16 if wl.dtype == "bf16" else torch.float32
     x0, blocks = synth.make_workload(wl, seed=0)
-    model = rs.PrunedViT(ctx, blocks, wl.H, list(wl.drops), tdt, tap_blocks=[])   # only the final tokens are materialised
+    # only the final tokens are materialised; LN1 of the blocks that follow a non-pruning block is applied inside
+    # their QKV product (rs_prepare_ln1_fold) unless --no-ln-fold
+    model = rs.PrunedViT(ctx, blocks, wl.H, list(wl.drops), tdt, tap_blocks=[], fold_ln1=not args.no_ln_fold)
     del blocks
     gen = torch.Generator().manual_seed(100 + rank)
     host_x = [x0.to(tdt).pin_memory()] + [
@@ -588,6 +590,7 @@ def main(argv=None):
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-other-workloads", action="store_true", help="skip the `workloads` object (the other bf16 configurations)")
     ap.add_argument("--no-isolated", action="store_true", help="skip the stand-alone attention / score / compaction timings")
+    ap.add_argument("--no-ln-fold", action="store_true", help="keep LN1 a kernel of its own in every block")
     ap.add_argument("--no-graph", action="store_true", help="launch every kernel from the host instead of replaying a CUDA graph")
     args = ap.parse_args(argv)
     from paper_2508_00367_b200 import synth

@@ -172,7 +172,28 @@ typedef struct {           /* all dev pointers */
     const void *w_qkv /*[3D,D]*/, *w_o /*[D,D]*/, *w_fc1 /*[D_mlp,D]*/, *w_fc2 /*[D,D_mlp]*/; /* dtype */
     const float *b_qkv, *b_o, *b_fc1, *b_fc2;        /* fp32; may be NULL */
     const float *ln1_g, *ln1_b, *ln2_g, *ln2_b;      /* fp32 */
+    /* Optional, all three or none (NULL): the block's first LayerNorm folded into its QKV projection, as
+     * rs_prepare_ln1_fold writes them.  Only rs_vit_fwd / rs_vit_fwd_taps use them. */
+    const void* w_qkv_ln;    /* [3D, D] dtype: w_qkv with column k scaled by ln1_g[k] */
+    const float* c_qkv_ln;   /* [3D] fp32: row sums of w_qkv_ln */
+    const float* b_qkv_ln;   /* [3D] fp32: b_qkv + w_qkv . ln1_b */
 } rs_block_weights;
+
+/* ---- rs_prepare_ln1_fold: LayerNorm folded into the projection that follows it (Eq. att: the ----
+ * block computes SA(LN(x)); the paper fixes the arithmetic, not where the normalisation is applied).
+ * For a row x with mean mu and reciprocal standard deviation rstd over its D features,
+ *   LN(x) W^T + b  =  rstd * (x W'^T - mu * c) + b',   W'[n,k] = W[n,k] g[k],  c[n] = sum_k W'[n,k],
+ *   b'[n] = b[n] + sum_k W[n,k] beta[k],
+ * so the projection can read the un-normalised tokens and the LayerNorm kernel (a full read and write of
+ * the [T, D] activations) disappears; mu and rstd come from sums that the previous block's last
+ * product leaves behind.  This call writes W' (rounded to `dtype`), c (sums of the rounded W') and b'
+ * into caller buffers; put them in rs_block_weights and the layer loop uses the folded form for every
+ * block whose predecessor drops no token (after a pruning block the normalisation already rides in
+ * the kernel that moves the kept rows).  RS_BF16 only; D a multiple of 128.  Results differ from
+ * the unfolded loop by rounding (W g is rounded once more, LN(x) is not rounded to bf16). */
+RS_API rs_status rs_prepare_ln1_fold(rs_ctx* ctx, rs_dtype dtype, int D, const void* w_qkv, const float* b_qkv,
+                                     const float* ln1_g, const float* ln1_b, void* w_out, float* c_out,
+                                     float* b_out, void* stream);
 
 /* 1 if rs_block_fwd runs this descriptor on the tcgen05 kernels, 0 if on the fp32-FMA kernels
  * (see rs_linear_uses_tensor_cores). */

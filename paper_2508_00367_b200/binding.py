@@ -28,7 +28,7 @@ EXPORTS = ("rs_create", "rs_destroy", "rs_last_error", "rs_async_status", "rs_us
            "rs_block_workspace_bytes", "rs_block_fwd", "rs_timing_enable", "rs_timing_read",
            "rs_static_scratch_bytes", "rs_block_fwd_static", "rs_linear_fwd", "rs_vit_workspace_bytes", "rs_vit_fwd",
            "rs_vit_fwd_taps", "rs_linewise_compact", "rs_static_async_status", "rs_linear_uses_tensor_cores",
-           "rs_block_uses_tensor_cores", "rs_attn_fwd_ragged", "rs_topk_compact_ragged", "rs_block_fwd_ragged", "rs_vit_fwd_ragged", "rs_tmap_cache_stats")
+           "rs_block_uses_tensor_cores", "rs_attn_fwd_ragged", "rs_topk_compact_ragged", "rs_block_fwd_ragged", "rs_vit_fwd_ragged", "rs_prepare_ln1_fold", "rs_tmap_cache_stats")
 LIN_EPILOGUE = {"bias": 0, "gelu": 1, "residual": 2}
 KERNEL_CLASSES = ("layernorm", "gemm", "attn", "score", "select", "gather")
 
@@ -73,7 +73,7 @@ class VitTaps(ctypes.Structure):
 class BlockWeights(ctypes.Structure):
     _fields_ = [(n, ctypes.c_void_p) for n in
                 ("w_qkv", "w_o", "w_fc1", "w_fc2", "b_qkv", "b_o", "b_fc1", "b_fc2",
-                 "ln1_g", "ln1_b", "ln2_g", "ln2_b")]
+                 "ln1_g", "ln1_b", "ln2_g", "ln2_b", "w_qkv_ln", "c_qkv_ln", "b_qkv_ln")]
 
 
 _lib = None
@@ -151,6 +151,8 @@ def load_library() -> ctypes.CDLL:
     lib.rs_vit_fwd_ragged.argtypes = [vp, ctypes.POINTER(VitDesc), ctypes.POINTER(BlockWeights), ctypes.POINTER(ci), vp, vp, vp,
                                       vp, vp, vp, vp, ctypes.c_size_t, vp]
     lib.rs_vit_fwd_ragged.restype = ci
+    lib.rs_prepare_ln1_fold.argtypes = [vp, ci, ci, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.rs_prepare_ln1_fold.restype = ci
     _lib = lib
     return lib
 
@@ -559,6 +561,20 @@ class DeviceBlockWeights:
         self.struct = BlockWeights(*[None if self.t[n] is None else self.t[n].data_ptr()
                                      for n in self.MATS + self.VECS])
 
+    def fold_ln1(self, ctx: "Context"):
+        """rs_prepare_ln1_fold: LN1 folded into the QKV weights (bf16 only), for the layer loop."""
+        w = self.t["w_qkv"]
+        assert w.dtype == torch.bfloat16
+        D = w.shape[1]
+        self.t["w_qkv_ln"] = torch.empty_like(w)
+        self.t["c_qkv_ln"] = torch.empty(3 * D, dtype=torch.float32, device=w.device)
+        self.t["b_qkv_ln"] = torch.empty(3 * D, dtype=torch.float32, device=w.device)
+        ctx._check(ctx.lib.rs_prepare_ln1_fold(ctx.handle, RS_BF16, D, _ptr(w), _ptr(self.t["b_qkv"]), _ptr(self.t["ln1_g"]),
+                                               _ptr(self.t["ln1_b"]), _ptr(self.t["w_qkv_ln"]), _ptr(self.t["c_qkv_ln"]),
+                                               _ptr(self.t["b_qkv_ln"]), _stream(w.device)))
+        for n in ("w_qkv_ln", "c_qkv_ln", "b_qkv_ln"):
+            setattr(self.struct, n, self.t[n].data_ptr())
+
 
 class PrunedViT:
     """Layer loop of the pruned forward pass: block l+1 consumes block l's
@@ -566,7 +582,7 @@ class PrunedViT:
 
     def __init__(self, ctx: Context, blocks: Sequence[Dict[str, torch.Tensor]], H: int, drops: Sequence[int],
                  dtype: torch.dtype, has_cls: bool = True, score_mode: str = "mlp", dist: str = "l2",
-                 tap_blocks: Optional[Sequence[int]] = None):
+                 tap_blocks: Optional[Sequence[int]] = None, fold_ln1: bool = False):
         """tap_blocks: the blocks whose compacted tokens x_out the caller wants (the last block always);
         None = every block.  A pruning block that is not tapped writes no dense copy of its kept
         tokens: the next block reads them in place through the index list.  Scores and kept indices
@@ -577,6 +593,11 @@ class PrunedViT:
         self.tapped = set(range(L)) if tap_blocks is None else (set(int(b) for b in tap_blocks) | {L - 1})
         self.has_cls, self.score_mode, self.dist = has_cls, score_mode, dist
         self.weights: List[DeviceBlockWeights] = [DeviceBlockWeights(w, dtype, ctx.device) for w in blocks]
+        if fold_ln1 and dtype == torch.bfloat16:
+            # LN1 of a block whose predecessor drops no token is applied inside its QKV product
+            for l in range(1, L):
+                if self.drops[l - 1] == 0:
+                    self.weights[l].fold_ln1(ctx)
         self._plan = None
 
     def plan(self, B: int, N: int, D: int):

@@ -363,6 +363,13 @@ struct LoopHooks {
     const int32_t* seq_lens;
     const int32_t* drops;
     int32_t* lens_out;
+    // LN1 folded into QKV (the layer loop, blocks whose predecessor drops nothing and whose weights carry
+    // the folded form): stats_in / parts_in = the row sums the previous block's FC2 left of this block's
+    // input; stats_out / parts_out = where this block's FC2 leaves them for the next block.
+    const float* stats_in;
+    int parts_in;
+    float* stats_out;
+    int* parts_out;
 };
 
 static rs_status block_fwd_impl(rs_ctx* ctx, const rs_block_desc* d, const rs_block_weights* w, const void* x,
@@ -433,12 +440,19 @@ static rs_status block_fwd_impl(rs_ctx* ctx, const rs_block_desc* d, const rs_bl
 
     // x' = SA(LN(x)) + x                                                  (Eq. att)
     const void* x_ln = hk ? hk->x_ln : nullptr;
-    if (!x_ln) {
+    const bool fold_ln1 = tc && hk && hk->stats_in && !x_ln && !in_map && w->w_qkv_ln && w->c_qkv_ln && w->b_qkv_ln;
+    if (!x_ln && !fold_ln1) {
         RS_CHECK_LAUNCH(ctx, RS_K_LAYERNORM, st, rs::launch_layernorm(d->dtype, d->dtype, x, w->ln1_g, w->ln1_b, eps, T, D, u, in_map, st), "LN1");
         x_ln = u;
     }
     if (tc) {
-        RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_tc(ctx, rs::RS_EPI_BIAS, x_ln, w->w_qkv, w->b_qkv, nullptr, nullptr, nullptr, qkv, RS_BF16, nullptr, 0, 0, T, 3 * D, D, st), "QKV");
+        if (fold_ln1) {
+            // LN1 applied in the epilogue: the product reads the block input itself
+            const rs::GemmLn ln = {nullptr, nullptr, hk->stats_in, hk->parts_in, w->c_qkv_ln, eps};
+            RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_tc(ctx, rs::RS_EPI_BIAS, x, w->w_qkv_ln, w->b_qkv_ln, nullptr, nullptr, nullptr, qkv, RS_BF16, nullptr, 0, 0, T, 3 * D, D, st, &ln), "LN1+QKV");
+        } else {
+            RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_tc(ctx, rs::RS_EPI_BIAS, x_ln, w->w_qkv, w->b_qkv, nullptr, nullptr, nullptr, qkv, RS_BF16, nullptr, 0, 0, T, 3 * D, D, st), "QKV");
+        }
         RS_CHECK_LAUNCH(ctx, RS_K_ATTN, st, rs::launch_attn_tc(ctx, ad, qkv, kp, vp, o, hk ? hk->seq_lens : nullptr, st), "attention");
         // shift through attention (operation choice (i)): partial sums of (SA(LN(x)) - x)^2 from this epilogue
         nparts = rs::gemm_tc_score_parts(ctx, T, D);
@@ -458,7 +472,8 @@ static rs_status block_fwd_impl(rs_ctx* ctx, const rs_block_desc* d, const rs_bl
         float* fc2_parts = d->score_mode == RS_SCORE_ATTN ? m + (size_t)T * nparts * 3 : m;
         const int kind = d->score_mode == RS_SCORE_MLP_DELTA ? 1 : d->score_mode == RS_SCORE_BLOCK ? 2 : 0;
         RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_tc(ctx, rs::RS_EPI_BIAS_GELU, u, w->w_fc1, w->b_fc1, nullptr, nullptr, nullptr, h, RS_BF16, nullptr, 0, 0, T, Dm, D, st), "FC1");
-        RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_tc(ctx, rs::RS_EPI_SCORE, h, w->w_fc2, w->b_fc2, x_prime, x, in_map, x_hat, d->out_dtype, fc2_parts, kind, (int)d->dist, T, D, Dm, st), "FC2+residual+score");
+        const rs::GemmLn lnout = {hk ? hk->stats_out : nullptr, hk ? hk->parts_out : nullptr, nullptr, 0, nullptr, 0.f};
+        RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_tc(ctx, rs::RS_EPI_SCORE, h, w->w_fc2, w->b_fc2, x_prime, x, in_map, x_hat, d->out_dtype, fc2_parts, kind, (int)d->dist, T, D, Dm, st, (hk && hk->stats_out) ? &lnout : nullptr), "FC2+residual+score");
     } else {
         RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_simt(d->dtype, u, w->w_fc1, w->b_fc1, 1, nullptr, RS_F32, h, d->dtype, T, Dm, D, st), "FC1");
         RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_simt(d->dtype, h, w->w_fc2, w->b_fc2, 0, nullptr, RS_F32, m, RS_F32, T, D, Dm, st), "FC2");
@@ -511,7 +526,7 @@ rs_status rs_block_fwd_ragged(rs_ctx* ctx, const rs_block_desc* d, const rs_bloc
                               void* stream) {
     if (!ctx) return RS_ERR_INVALID_ARG;
     if (!seq_lens || !drops || !keep_idx) return fail(ctx, RS_ERR_INVALID_ARG, "rs_block_fwd_ragged: seq_lens, drops and keep_idx are required");
-    const LoopHooks hk = {nullptr, nullptr, nullptr, nullptr, true, nullptr, seq_lens, drops, lens_out};
+    const LoopHooks hk = {nullptr, nullptr, nullptr, nullptr, true, nullptr, seq_lens, drops, lens_out, nullptr, 0, nullptr, nullptr};
     return block_fwd_impl(ctx, d, w, x, x_out, scores, keep_idx, x_full, workspace, workspace_bytes, stream, &hk);
 }
 
@@ -562,7 +577,7 @@ namespace {
 
 // Plan of the layer loop: per-block descriptors, the largest block scratch and the size of one
 // of the two token buffers the blocks alternate between.  False on a bad descriptor / schedule.
-struct VitPlan { size_t block_ws, act_bytes, map_bytes, total; int n_final; };
+struct VitPlan { size_t block_ws, act_bytes, map_bytes, stats_bytes, total; int n_final; };
 
 bool vit_plan(const rs_vit_desc& d, const int* drops, VitPlan* p) {
     if (!drops || d.L < 1 || d.B < 1 || d.N < 1) return false;
@@ -579,8 +594,10 @@ bool vit_plan(const rs_vit_desc& d, const int* drops, VitPlan* p) {
     p->block_ws = rs::align_up(block_ws, 256);
     p->act_bytes = rs::align_up((size_t)d.B * d.N * d.D * rs::dtype_size(d.dtype), 256);
     p->map_bytes = rs::align_up((size_t)d.B * d.N * sizeof(int32_t), 256);
-    // block scratch, two token buffers, one LN buffer, two row maps
-    p->total = p->block_ws + 3 * p->act_bytes + 2 * p->map_bytes;
+    // row sums for a LayerNorm folded into the next block's QKV: up to 2 * D / 128 pairs of floats per row
+    p->stats_bytes = rs::align_up((size_t)d.B * d.N * (2 * (size_t)d.D / 128 + 2) * 8, 256);
+    // block scratch, two token buffers, one LN buffer, two row maps, two row-sum buffers
+    p->total = p->block_ws + 3 * p->act_bytes + 2 * p->map_bytes + 2 * p->stats_bytes;
     p->n_final = n;
     return true;
 }
@@ -612,6 +629,10 @@ rs_status rs_vit_fwd_taps(rs_ctx* ctx, const rs_vit_desc* d, const rs_block_weig
     void* act[2] = {base + p.block_ws, base + p.block_ws + p.act_bytes};
     void* ln_buf = base + p.block_ws + 2 * p.act_bytes;   // LN1 of the next block's input, from the pruning kernel
     int32_t* maps[2] = {(int32_t*)(base + p.block_ws + 3 * p.act_bytes), (int32_t*)(base + p.block_ws + 3 * p.act_bytes + p.map_bytes)};
+    float* stats[2] = {(float*)(base + p.block_ws + 3 * p.act_bytes + 2 * p.map_bytes),
+                       (float*)(base + p.block_ws + 3 * p.act_bytes + 2 * p.map_bytes + p.stats_bytes)};
+    const float* cur_stats = nullptr;    // row sums of the block input, when the previous block's FC2 left them
+    int cur_parts = 0;
     const float eps = d->ln_eps > 0.f ? d->ln_eps : 1e-6f;
     const void* cur = x;                 // the block input: dense [B, n, D], or, with cur_map, the previous
     const int32_t* cur_map = nullptr;    // block's un-pruned x^ read through the row map
@@ -629,8 +650,14 @@ rs_status rs_vit_fwd_taps(rs_ctx* ctx, const rs_vit_desc* d, const rs_block_weig
         // LN1 of block l+1 rides in this block's pruning kernel: one kernel less per block
         const rs::LnFuse next = {last ? nullptr : weights[l + 1].ln1_g, last ? nullptr : weights[l + 1].ln1_b, eps, ln_buf};
         bool ln_done = false;
+        // A block that drops nothing hands its output to the next block as it is: if that block's weights
+        // carry LN1 folded into QKV, this block's FC2 leaves the row sums and no LN1 kernel runs.
+        const bool fold_next = !last && drops[l] == 0 && d->dtype == RS_BF16 && weights[l + 1].w_qkv_ln &&
+                               weights[l + 1].c_qkv_ln && weights[l + 1].b_qkv_ln && rs_block_uses_tensor_cores(ctx, &bd);
+        int parts_out = 0;
         const LoopHooks hk = {cur_map, cur_ln, (last || !next.gamma || !next.beta) ? nullptr : &next,
-                              in_place ? maps[l & 1] : nullptr, !in_place, &ln_done, nullptr, nullptr, nullptr};
+                              in_place ? maps[l & 1] : nullptr, !in_place, &ln_done, nullptr, nullptr, nullptr,
+                              cur_stats, cur_parts, fold_next ? stats[l & 1] : nullptr, fold_next ? &parts_out : nullptr};
         rs_status st = block_fwd_impl(ctx, &bd, &weights[l], cur, out, taps->scores ? taps->scores[l] : nullptr,
                                       taps->keep_idx ? taps->keep_idx[l] : nullptr, in_place ? act[l & 1] : nullptr, base,
                                       p.block_ws, stream, &hk);
@@ -638,8 +665,23 @@ rs_status rs_vit_fwd_taps(rs_ctx* ctx, const rs_vit_desc* d, const rs_block_weig
         cur = in_place ? act[l & 1] : out;
         cur_map = in_place ? maps[l & 1] : nullptr;
         cur_ln = ln_done ? ln_buf : nullptr;
+        cur_stats = (fold_next && parts_out > 0) ? stats[l & 1] : nullptr;
+        cur_parts = parts_out;
         n -= drops[l];
     }
+    return RS_OK;
+}
+
+rs_status rs_prepare_ln1_fold(rs_ctx* ctx, rs_dtype dtype, int D, const void* w_qkv, const float* b_qkv,
+                              const float* ln1_g, const float* ln1_b, void* w_out, float* c_out, float* b_out,
+                              void* stream) {
+    if (!ctx) return RS_ERR_INVALID_ARG;
+    if (!w_qkv || !ln1_g || !ln1_b || !w_out || !c_out || !b_out) return fail(ctx, RS_ERR_INVALID_ARG, "rs_prepare_ln1_fold: null argument");
+    if (dtype != RS_BF16 || D < 128 || (D % 128)) return fail(ctx, RS_ERR_UNSUPPORTED, "rs_prepare_ln1_fold: bf16 and D a multiple of 128 only");
+    if (!aligned16(w_qkv) || !aligned16(w_out)) return fail(ctx, RS_ERR_INVALID_ARG, "rs_prepare_ln1_fold: misaligned pointer");
+    cudaError_t e = rs::launch_ln_fold_prep(w_qkv, b_qkv, ln1_g, ln1_b, 3 * D, D, w_out, c_out, b_out, (cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "rs_prepare_ln1_fold");
+    ctx->launches += 1;
     return RS_OK;
 }
 
@@ -672,7 +714,8 @@ rs_status rs_vit_fwd_ragged(rs_ctx* ctx, const rs_vit_desc* d, const rs_block_we
                             d->score_mode, d->dist};
         void* out = last ? x_out : act[l & 1];
         int32_t* next_lens = last ? lens_out : lens[l & 1];
-        const LoopHooks hk = {nullptr, nullptr, nullptr, nullptr, true, nullptr, cur_lens, sample_drops + (size_t)l * d->B, next_lens};
+        const LoopHooks hk = {nullptr, nullptr, nullptr, nullptr, true, nullptr, cur_lens, sample_drops + (size_t)l * d->B, next_lens,
+                              nullptr, 0, nullptr, nullptr};
         rs_status st = block_fwd_impl(ctx, &bd, &weights[l], cur, out, nullptr, last ? keep_last : nullptr, nullptr, base,
                                       p.block_ws, stream, &hk);
         if (st != RS_OK) return st;

@@ -208,4 +208,39 @@ cudaError_t launch_residual_score(const float* m, const float* x_prime, const vo
     return cudaGetLastError();
 }
 
+// LayerNorm folded into the projection that follows: one warp per output row n of W [n_out, K].
+namespace {
+__global__ void __launch_bounds__(256)
+ln_fold_prep_kernel(const __nv_bfloat16* __restrict__ W, const float* __restrict__ bias, const float* __restrict__ g,
+                    const float* __restrict__ beta, int n_out, int K, __nv_bfloat16* __restrict__ w_out,
+                    float* __restrict__ c_out, float* __restrict__ b_out) {
+    const int n = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    if (n >= n_out) return;
+    float c = 0.f, bb = 0.f;
+    for (int k = lane; k < K; k += 32) {
+        const float w = __bfloat162float(W[(size_t)n * K + k]);
+        const __nv_bfloat16 ws = __float2bfloat16_rn(w * g[k]);
+        w_out[(size_t)n * K + k] = ws;
+        c += __bfloat162float(ws);
+        bb = fmaf(w, beta[k], bb);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        c += __shfl_xor_sync(0xffffffffu, c, o);
+        bb += __shfl_xor_sync(0xffffffffu, bb, o);
+    }
+    if (lane == 0) {
+        c_out[n] = c;
+        b_out[n] = bb + (bias ? bias[n] : 0.f);
+    }
+}
+}  // namespace
+
+cudaError_t launch_ln_fold_prep(const void* W, const float* bias, const float* g, const float* beta, int n_out, int K,
+                                void* w_out, float* c_out, float* b_out, cudaStream_t st) {
+    ln_fold_prep_kernel<<<(n_out + 7) / 8, 256, 0, st>>>((const __nv_bfloat16*)W, bias, g, beta, n_out, K,
+                                                         (__nv_bfloat16*)w_out, c_out, b_out);
+    return cudaGetLastError();
+}
+
 }  // namespace rs

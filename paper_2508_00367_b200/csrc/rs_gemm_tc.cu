@@ -31,7 +31,12 @@ namespace {
 
 using namespace tc;
 
-enum { EPI_BIAS = 0, EPI_BIAS_GELU = 1, EPI_RESID = 2, EPI_SCORE = 3 };
+// EPI_SCORE_STATS: EPI_SCORE that also leaves, per row and column half of a tile, the sum and the sum of
+// squares of the (rounded) output values -- the row statistics of the next block's LayerNorm.
+// EPI_BIAS_LN: the LayerNorm of the A operand folded into the product: with W' = W * gamma (column-wise),
+// c_n = sum_k W'_nk and b'_n = b_n + sum_k W_nk beta_k,  LN(x) W^T + b = rstd (x W'^T - mu c) + b';  mu and
+// rstd of a row come from the statistics above, acc = x W'^T from the tensor cores.
+enum { EPI_BIAS = 0, EPI_BIAS_GELU = 1, EPI_RESID = 2, EPI_SCORE = 3, EPI_SCORE_STATS = 4, EPI_BIAS_LN = 5 };
 
 constexpr int BM = 128;                       // rows per CTA; the pair's tile has 2 * BM rows
 constexpr int BK = 64;
@@ -47,18 +52,20 @@ constexpr int RES_BOX_BYTES = 32 * 64;         // residual of one 32-column chun
 // for the room with one staging buffer per warp instead of two and one operand stage less.
 template <int BN, int EPI> struct Cfg {
     static constexpr bool RES_TMA = EPI == EPI_RESID;
+    static constexpr bool LN = EPI == EPI_BIAS_LN;                 // one staging buffer per warp, room for a second column vector
     static constexpr int B_BYTES = (BN / 2) * BK * 2;              // this CTA's half of the W tile
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
     static constexpr int STAGES = (BN == 128) ? 6 : RES_TMA ? 4 : 5;
     static constexpr int TMEM_COLS = (BN == 128) ? 256 : 512;      // two accumulators, a power of two
     static constexpr int SPLIT = (BN == 128) ? 64 : 128;           // epilogue warps 2-5 take columns [0, SPLIT)
-    static constexpr int STG_PER_WARP = RES_TMA ? 1 : 2;
+    static constexpr int STG_PER_WARP = (RES_TMA || LN) ? 1 : 2;
     static constexpr int RES_WARP_BYTES = RES_TMA ? (SPLIT / 32) * RES_BOX_BYTES : 0;   // the wider half's chunks
     static constexpr int OFF_STG = STAGES * STAGE_BYTES;
     static constexpr int OFF_RES = OFF_STG + kEpiWarps * STG_PER_WARP * STG_BYTES;
     static constexpr int OFF_BAR = OFF_RES + kEpiWarps * RES_WARP_BYTES;
     static constexpr int OFF_BIAS = OFF_BAR + 256;                 // float [2 tile parities][2 halves][128]: bias slices
-    static constexpr size_t SMEM = (size_t)OFF_BIAS + 2048;        // the window itself must be 1024-byte aligned
+    static constexpr int OFF_COLSUM = OFF_BIAS + 2048;             // EPI_BIAS_LN: float [2][2][128] like the bias slices
+    static constexpr size_t SMEM = (size_t)OFF_BIAS + (LN ? 4096 : 2048);   // the window itself must be 1024-byte aligned
     static_assert(SMEM <= 227 * 1024, "shared memory of one CTA");
 };
 
@@ -72,6 +79,11 @@ struct GemmArgs {
     float* partials;          // EPI_SCORE (and EPI_RESID when non-null): [M, 2 * N / BN] sums of squares
     int score_kind;           // EPI_SCORE: scored pair (u, v) = 0: (m, x'), 1: (x^, x'), 2: (x^, x)
     int dist;                 // rs_dist of the score: L2 / L1 sums of (u - v)^2 / |u - v|, cosine sums of u.v, u.u, v.v
+    float* stats_out;         // EPI_SCORE_STATS: [M, 2 * N / BN][2] = (sum, sum of squares) of the row's outputs in that half tile
+    const float* stats_in;    // EPI_BIAS_LN: such statistics of the A operand's rows, stats_parts pairs per row over ln_dim = K values
+    const float* colsum;      // EPI_BIAS_LN: c [N]
+    int stats_parts;
+    float ln_eps;
     int* status;
 };
 
@@ -262,18 +274,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             if (args.row_map) issue_res_mapped(pair);
             else if (lane == 0) issue_res(pair);
         }
-        constexpr int RES_VECS = EPI == EPI_RESID ? 4 : EPI == EPI_SCORE ? 8 : 1;   // 16-byte loads per 32 columns
+        constexpr bool SCORE = EPI == EPI_SCORE || EPI == EPI_SCORE_STATS;
+        constexpr int RES_VECS = EPI == EPI_RESID ? 4 : SCORE ? 8 : 1;   // 16-byte loads per 32 columns
         for (int tile = pair; tile < tiles; tile += npairs, ++tl) {
             const int m0 = (tile / num_n) * (2 * BM) + (int)rank * BM, nt = tile % num_n, n0 = nt * BN;
             const uint32_t a = tl & 1u, aph = (tl >> 1) & 1u;
             const int row = m0 + trow;
             const bool valid = row < args.M;
             // row of the block input x (EPI_SCORE, whole-block shift), possibly through the row map
-            const int xrow = (EPI == EPI_SCORE && args.score_kind == 2 && args.row_map && valid) ? __ldg(args.row_map + row) : row;
+            const int xrow = (SCORE && args.score_kind == 2 && args.row_map && valid) ? __ldg(args.row_map + row) : row;
             // Residual values of 32 columns of this thread's row (zeros for rows past M).  They are
             // fetched one chunk ahead, the first chunk before the accumulator is even complete.
             auto load_res = [&](int c, uint4* dst) {
-                if (EPI == EPI_SCORE) {
+                if (SCORE) {
                     const size_t off = (size_t)row * args.N + n0 + c;
                     const uint4* rp = reinterpret_cast<const uint4*>(reinterpret_cast<const float*>(args.residual) + off);
 #pragma unroll
@@ -282,6 +295,23 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             };
             uint4 res_next[RES_VECS];
             load_res(c_begin, res_next);
+            // EPI_BIAS_LN: mean and reciprocal standard deviation of this thread's row of A from the partial
+            // sums its producer left (fetched while the accumulator is still being computed)
+            float ln_mu = 0.f, ln_rstd = 0.f;
+            if (EPI == EPI_BIAS_LN) {
+                float s1 = 0.f, s2 = 0.f;
+                if (valid) {
+                    const float2* sp = reinterpret_cast<const float2*>(args.stats_in) + (size_t)row * args.stats_parts;
+                    for (int p = 0; p < args.stats_parts; ++p) {
+                        const float2 t = __ldg(sp + p);
+                        s1 += t.x; s2 += t.y;
+                    }
+                }
+                const float inv_d = 1.f / (float)args.K;
+                ln_mu = s1 * inv_d;
+                ln_rstd = rsqrtf(fmaxf(s2 * inv_d - ln_mu * ln_mu, 0.f) + args.ln_eps);
+            }
+            float st1 = 0.f, st2 = 0.f;                  // EPI_SCORE_STATS: sums over this thread's columns
             // The four warps of a column half decide together whether to go on: the named
             // barriers below have no time limit, so no warp may leave the loop alone.
             // this half's slice of the bias goes to shared memory while the accumulator is still being
@@ -289,6 +319,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             // Two copies, by tile parity: a warp may still be reading the last tile's slice.
             float* bias_s = reinterpret_cast<float*>(smem + C::OFF_BIAS) + (tl & 1u) * 256 + half * 128;
             if (c_begin + t128 < c_end) bias_s[t128] = args.bias ? __ldg(args.bias + n0 + c_begin + t128) : 0.f;
+            float* cs_s = reinterpret_cast<float*>(smem + C::OFF_COLSUM) + (tl & 1u) * 256 + half * 128;   // EPI_BIAS_LN only
+            if (EPI == EPI_BIAS_LN && c_begin + t128 < c_end) cs_s[t128] = __ldg(args.colsum + n0 + c_begin + t128);
             if (!__all_sync(0xffffffffu, mbar_wait(&tfull[a], aph, abort_flag))) half_fail[half] = 1;
             if (C::RES_TMA && !__all_sync(0xffffffffu, mbar_wait(&res_full[warp - 2], tl & 1u, abort_flag))) half_fail[half] = 1;
             named_barrier(1 + half, 128);
@@ -331,10 +363,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
                 for (int j = 0; j < 32; j += 4) {
                     const float4 b = *reinterpret_cast<const float4*>(bias_s + (c - c_begin) + j);
-                    v[j] = __uint_as_float(r[j]) + b.x;
-                    v[j + 1] = __uint_as_float(r[j + 1]) + b.y;
-                    v[j + 2] = __uint_as_float(r[j + 2]) + b.z;
-                    v[j + 3] = __uint_as_float(r[j + 3]) + b.w;
+                    if (EPI == EPI_BIAS_LN) {
+                        const float4 cc = *reinterpret_cast<const float4*>(cs_s + (c - c_begin) + j);
+                        v[j] = fmaf(ln_rstd, fmaf(-ln_mu, cc.x, __uint_as_float(r[j])), b.x);
+                        v[j + 1] = fmaf(ln_rstd, fmaf(-ln_mu, cc.y, __uint_as_float(r[j + 1])), b.y);
+                        v[j + 2] = fmaf(ln_rstd, fmaf(-ln_mu, cc.z, __uint_as_float(r[j + 2])), b.z);
+                        v[j + 3] = fmaf(ln_rstd, fmaf(-ln_mu, cc.w, __uint_as_float(r[j + 3])), b.w);
+                    } else {
+                        v[j] = __uint_as_float(r[j]) + b.x;
+                        v[j + 1] = __uint_as_float(r[j + 1]) + b.y;
+                        v[j + 2] = __uint_as_float(r[j + 2]) + b.z;
+                        v[j + 3] = __uint_as_float(r[j + 3]) + b.w;
+                    }
                 }
                 if (EPI == EPI_BIAS_GELU) {
 #pragma unroll
@@ -354,7 +394,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                             v[8 * j + 2 * e + 1] += x1;
                         }
                     }
-                } else if (EPI == EPI_SCORE) {
+                } else if (SCORE) {
                     if (args.score_kind == 2) {
                         // whole-block shift: x^ - x, with the block input x read here (rows past M: zeros)
                         const uint4* x0p = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(args.residual2) +
@@ -396,9 +436,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
                     for (int g = 0; g < 4; ++g) {
                         const int piece = cb * 4 + g;
-                        *reinterpret_cast<uint4*>(stg + stg_row + ((piece ^ r8) << 4)) =
-                            make_uint4(pack_bf16(v[8 * g], v[8 * g + 1]), pack_bf16(v[8 * g + 2], v[8 * g + 3]),
-                                       pack_bf16(v[8 * g + 4], v[8 * g + 5]), pack_bf16(v[8 * g + 6], v[8 * g + 7]));
+                        const uint4 pk = make_uint4(pack_bf16(v[8 * g], v[8 * g + 1]), pack_bf16(v[8 * g + 2], v[8 * g + 3]),
+                                                    pack_bf16(v[8 * g + 4], v[8 * g + 5]), pack_bf16(v[8 * g + 6], v[8 * g + 7]));
+                        *reinterpret_cast<uint4*>(stg + stg_row + ((piece ^ r8) << 4)) = pk;
+                        if (EPI == EPI_SCORE_STATS) {
+                            // the statistics are those of the values as stored: the next block reads these bf16 numbers
+                            const uint32_t w[4] = {pk.x, pk.y, pk.z, pk.w};
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const float y0 = __uint_as_float(w[e] << 16), y1 = __uint_as_float(w[e] & 0xffff0000u);
+                                st1 += y0 + y1;
+                                st2 = fmaf(y0, y0, fmaf(y1, y1, st2));
+                            }
+                        }
                     }
                 } else {
 #pragma unroll
@@ -425,7 +475,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     else if (lane == 0) issue_res(tile + npairs);
                 }
             }
-            if ((EPI == EPI_SCORE || (EPI == EPI_RESID && args.partials)) && valid) {
+            if (EPI == EPI_SCORE_STATS && valid) {
+                const size_t pi = (size_t)row * (2 * num_n) + 2 * nt + half;
+                reinterpret_cast<float2*>(args.stats_out)[pi] = make_float2(st1, st2);
+            }
+            if ((SCORE || (EPI == EPI_RESID && args.partials)) && valid) {
                 const size_t pi = (size_t)row * (2 * num_n) + 2 * nt + half;
                 if (args.dist == RS_DIST_COS) {
                     args.partials[3 * pi] = sq; args.partials[3 * pi + 1] = sq1; args.partials[3 * pi + 2] = sq2;
@@ -581,10 +635,14 @@ int gemm_tc_score_parts(const rs_ctx* ctx, long long M, int N) {
 
 cudaError_t launch_gemm_tc(rs_ctx* ctx, int epi, const void* A, const void* W, const float* bias,
                            const void* residual, const void* residual2, const int32_t* row_map, void* out, rs_dtype out_dtype,
-                           float* partials, int score_kind, int dist, long long M, int N, int K, cudaStream_t st) {
+                           float* partials, int score_kind, int dist, long long M, int N, int K, cudaStream_t st,
+                           const GemmLn* ln) {
     if (!ctx->encode_tiled) return cudaErrorNotSupported;
+    if (ln && epi == EPI_SCORE && ln->stats_out && out_dtype == RS_BF16) epi = EPI_SCORE_STATS;
+    if (ln && epi == EPI_BIAS && ln->stats_in) epi = EPI_BIAS_LN;
     const int bn = pick_bn(M, N, ctx->sm_count);
     const int out_bytes = (epi == EPI_RESID || (epi == EPI_SCORE && out_dtype == RS_F32)) ? 4 : 2;
+    if (epi == EPI_SCORE_STATS && ln->stats_parts_out) *ln->stats_parts_out = 2 * (N / bn);
     CUtensorMap tmA, tmB, tmOut, tmRes;
     if (epi == EPI_RESID && !row_map && !make_tmap_res(ctx, &tmRes, residual, (uint64_t)M, (uint64_t)N)) return cudaErrorInvalidValue;
     if (!make_tmap_2d(ctx, &tmA, A, 2, (uint64_t)M, (uint64_t)K, BM) ||
@@ -595,6 +653,11 @@ cudaError_t launch_gemm_tc(rs_ctx* ctx, int epi, const void* A, const void* W, c
     GemmArgs args;
     args.M = (int)M; args.N = N; args.K = K; args.bias = bias; args.residual = residual;
     args.residual2 = residual2; args.row_map = row_map; args.partials = partials; args.score_kind = score_kind; args.dist = dist; args.status = ctx->d_status;
+    args.stats_out = ln ? ln->stats_out : nullptr;
+    args.stats_in = ln ? ln->stats_in : nullptr;
+    args.colsum = ln ? ln->colsum : nullptr;
+    args.stats_parts = ln ? ln->stats_parts : 0;
+    args.ln_eps = ln ? ln->eps : 0.f;
     const int sms = ctx->sm_count;
 #define RS_GEMM_CASE(E, T)                                                                       \
     return bn == 256   ? launch_one<256, E, T>(tmA, tmB, tmOut, tmRes, args, sms, st)           \
@@ -607,6 +670,8 @@ cudaError_t launch_gemm_tc(rs_ctx* ctx, int epi, const void* A, const void* W, c
         case EPI_SCORE:
             if (out_dtype == RS_F32) RS_GEMM_CASE(EPI_SCORE, float);
             RS_GEMM_CASE(EPI_SCORE, __nv_bfloat16);
+        case EPI_SCORE_STATS: RS_GEMM_CASE(EPI_SCORE_STATS, __nv_bfloat16);
+        case EPI_BIAS_LN: RS_GEMM_CASE(EPI_BIAS_LN, __nv_bfloat16);
     }
 #undef RS_GEMM_CASE
     return cudaErrorInvalidValue;

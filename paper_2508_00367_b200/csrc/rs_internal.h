@@ -150,10 +150,24 @@ int gemm_tc_score_parts(const rs_ctx* ctx, long long M, int N);   // partial sum
 // out[M, N] = epilogue(A[M, K] . W[N, K]^T); see rs_gemm_tc.cu for the epilogues.
 // row_map (optional, [M] int32): row t of the block input (the bf16 residual of RS_EPI_RESID, residual2
 // of RS_EPI_SCORE) is row row_map[t] of the given matrix -- the un-pruned output of the previous block.
+cudaError_t launch_ln_fold_prep(const void* W, const float* bias, const float* g, const float* beta, int n_out, int K,
+                                void* w_out, float* c_out, float* b_out, cudaStream_t st);
+// LayerNorm folded across two products (the layer loop's non-pruning blocks): the FC2 launch of a block also
+// leaves per-row partial sums (stats_out, and how many per row in *stats_parts_out); the QKV launch of the
+// next block reads them (stats_in, stats_parts) and applies the normalisation in its epilogue, with the
+// prepared weights of rs_prepare_ln1_fold as W and bias and their column sums c.
+struct GemmLn {
+    float* stats_out;
+    int* stats_parts_out;
+    const float* stats_in;
+    int stats_parts;
+    const float* colsum;
+    float eps;
+};
 cudaError_t launch_gemm_tc(rs_ctx* ctx, int epi, const void* A, const void* W, const float* bias,
                            const void* residual, const void* residual2, const int32_t* row_map, void* out,
                            rs_dtype out_dtype, float* partials, int score_kind, int dist, long long M, int N, int K,
-                           cudaStream_t st);
+                           cudaStream_t st, const GemmLn* ln = nullptr);
 
 // ---- tcgen05 attention (rs_attn_tc.cu): bf16, head dimension 64 ----
 bool attn_tc_supported(const rs_attn_desc& d);

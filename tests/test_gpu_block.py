@@ -378,3 +378,43 @@ def test_tensor_maps_are_encoded_once_per_buffer():
         assert torch.equal(first[k], again[k]), k
     ctx.async_status()
     ctx.close()
+
+
+@pytest.mark.parametrize("B,N,D,H,drops", [(3, 197, 256, 4, [0, 0, 16]), (2, 300, 512, 8, [0, 40, 0, 0]),
+                                           (64, 197, 768, 12, [0, 0])])
+def test_layer_loop_with_ln1_folded_into_qkv(ctx, B, N, D, H, drops):
+    """rs_prepare_ln1_fold: a block whose predecessor drops nothing runs no LN1 kernel, its QKV product reads
+    the tokens themselves and normalises in its epilogue from the sums the previous FC2 left.  Every block
+    of the folded loop against the oracle fed that block's actual input (Eq. att, Eq. MLP, Sec. 3.2 / 3.1),
+    and one launch less per folded block."""
+    import paper_2508_00367_b200 as rs
+    L = len(drops)
+    x = synth.make_tokens(B, N, D, "bf16", seed=3 * N + D)
+    blocks = [synth.make_block_weights(D, 4 * D, "bf16", seed=50 + l) for l in range(L)]
+    plain = rs.PrunedViT(ctx, blocks, H, drops, torch.bfloat16)
+    folded = rs.PrunedViT(ctx, blocks, H, drops, torch.bfloat16, fold_ln1=True)
+    dx = x.to(torch.bfloat16).cuda()
+    n0 = ctx.launch_count()
+    outs_p = [{k: v.clone() for k, v in o.items()} for o in plain.forward(dx)]
+    n1 = ctx.launch_count()
+    outs = [{k: v.cpu() for k, v in o.items()} for o in folded.forward(dx)]
+    n2 = ctx.launch_count()
+    ctx.async_status()
+    n_folded = sum(1 for l in range(1, L) if drops[l - 1] == 0)
+    assert (n1 - n0) - (n2 - n1) == n_folded
+    cur = x.to(torch.bfloat16)
+    nsamp = min(B, 2)                       # the oracle on the first samples; the batch exercises the tiling
+    for l in range(L):
+        ref = orc.block_fwd(cur[:nsamp].double().numpy(), _np(blocks[l]), H, drops[l])
+        o = outs[l]
+        sc = o["scores"][:nsamp].double().numpy()
+        rel = np.abs(sc - ref["scores"]) / np.maximum(np.abs(ref["scores"]), 1e-30)
+        assert rel.max() < 5e-4, (l, rel.max())
+        parity.check_keep(ref["scores"], ref["keep_idx"], o["keep_idx"][:nsamp].numpy(), True)
+        for b in range(nsamp):
+            want = orc.round_to(ref["x_hat"][b][o["keep_idx"][b].long().numpy()], "bf16")
+            parity.check_float(o["x_out"][b].double().numpy()[None], want[None], "bf16", True)
+        # the folded loop stays within rounding of the plain one
+        torch.testing.assert_close(o["x_out"].float(), outs_p[l]["x_out"].cpu().float(), rtol=4e-2, atol=4e-2)
+        cur = o["x_out"]
+
