@@ -276,6 +276,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
         constexpr bool SCORE = EPI == EPI_SCORE || EPI == EPI_SCORE_STATS;
         constexpr int RES_VECS = EPI == EPI_RESID ? 4 : SCORE ? 8 : 1;   // 16-byte loads per 32 columns
+        // EPI_BIAS_LN: the partial row sums of this thread's row of the NEXT tile are fetched a tile ahead into
+        // registers (up to kLnPre pairs; more are read on the spot), so their way from L2 is never waited for
+        constexpr int kLnPre = EPI == EPI_BIAS_LN ? 16 : 1;
+        float2 ln_pre[kLnPre];
+        auto ln_fetch = [&](int tile) {
+            const int frow = (tile / num_n) * (2 * BM) + (int)rank * BM + trow;
+            const bool ok = tile < tiles && frow < args.M && args.stats_parts <= kLnPre;
+            const float2* sp = reinterpret_cast<const float2*>(args.stats_in) + (size_t)(ok ? frow : 0) * args.stats_parts;
+#pragma unroll
+            for (int p = 0; p < kLnPre; ++p) ln_pre[p] = (ok && p < args.stats_parts) ? __ldg(sp + p) : make_float2(0.f, 0.f);
+        };
+        if (EPI == EPI_BIAS_LN) ln_fetch(pair);
         for (int tile = pair; tile < tiles; tile += npairs, ++tl) {
             const int m0 = (tile / num_n) * (2 * BM) + (int)rank * BM, nt = tile % num_n, n0 = nt * BN;
             const uint32_t a = tl & 1u, aph = (tl >> 1) & 1u;
@@ -300,7 +312,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             float ln_mu = 0.f, ln_rstd = 0.f;
             if (EPI == EPI_BIAS_LN) {
                 float s1 = 0.f, s2 = 0.f;
-                if (valid) {
+                if (args.stats_parts <= kLnPre) {
+#pragma unroll
+                    for (int p = 0; p < kLnPre; ++p) { s1 += ln_pre[p].x; s2 += ln_pre[p].y; }
+                    ln_fetch(tile + npairs);
+                } else if (valid) {
                     const float2* sp = reinterpret_cast<const float2*>(args.stats_in) + (size_t)row * args.stats_parts;
                     for (int p = 0; p < args.stats_parts; ++p) {
                         const float2 t = __ldg(sp + p);
