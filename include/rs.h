@@ -188,8 +188,9 @@ typedef struct {           /* all dev pointers */
  * the [T, D] activations) disappears; mu and rstd come from sums that the previous block's last
  * product leaves behind.  This call writes W' (rounded to `dtype`), c (sums of the rounded W') and b'
  * into caller buffers; put them in rs_block_weights and the layer loop uses the folded form for every
- * block whose predecessor drops no token (after a pruning block the normalisation already rides in
- * the kernel that moves the kept rows).  RS_BF16 only; D a multiple of 128.  Results differ from
+ * block but the first: the sums come from the previous block's FC2 epilogue when that block drops no
+ * token, else from the kernel that moves the kept rows (which then copies them instead of normalising
+ * them, into a dense buffer).  RS_BF16 only; D a multiple of 128.  Results differ from
  * the unfolded loop by rounding (W g is rounded once more, LN(x) is not rounded to bf16). */
 RS_API rs_status rs_prepare_ln1_fold(rs_ctx* ctx, rs_dtype dtype, int D, const void* w_qkv, const float* b_qkv,
                                      const float* ln1_g, const float* ln1_b, void* w_out, float* c_out,

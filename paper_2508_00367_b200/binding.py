@@ -594,10 +594,9 @@ class PrunedViT:
         self.has_cls, self.score_mode, self.dist = has_cls, score_mode, dist
         self.weights: List[DeviceBlockWeights] = [DeviceBlockWeights(w, dtype, ctx.device) for w in blocks]
         if fold_ln1 and dtype == torch.bfloat16:
-            # LN1 of a block whose predecessor drops no token is applied inside its QKV product
+            # LN1 of every block but the first is applied inside its QKV product
             for l in range(1, L):
-                if self.drops[l - 1] == 0:
-                    self.weights[l].fold_ln1(ctx)
+                self.weights[l].fold_ln1(ctx)
         self._plan = None
 
     def plan(self, B: int, N: int, D: int):

@@ -472,8 +472,11 @@ static rs_status block_fwd_impl(rs_ctx* ctx, const rs_block_desc* d, const rs_bl
         float* fc2_parts = d->score_mode == RS_SCORE_ATTN ? m + (size_t)T * nparts * 3 : m;
         const int kind = d->score_mode == RS_SCORE_MLP_DELTA ? 1 : d->score_mode == RS_SCORE_BLOCK ? 2 : 0;
         RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_tc(ctx, rs::RS_EPI_BIAS_GELU, u, w->w_fc1, w->b_fc1, nullptr, nullptr, nullptr, h, RS_BF16, nullptr, 0, 0, T, Dm, D, st), "FC1");
-        const rs::GemmLn lnout = {hk ? hk->stats_out : nullptr, hk ? hk->parts_out : nullptr, nullptr, 0, nullptr, 0.f};
-        RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_tc(ctx, rs::RS_EPI_SCORE, h, w->w_fc2, w->b_fc2, x_prime, x, in_map, x_hat, d->out_dtype, fc2_parts, kind, (int)d->dist, T, D, Dm, st, (hk && hk->stats_out) ? &lnout : nullptr), "FC2+residual+score");
+        // row sums for a LayerNorm folded into the next block's QKV: from this epilogue when the block's output is
+        // the next block's input as it stands, else from the kernel that moves the kept rows (below)
+        const bool fc2_stats = hk && hk->stats_out && x_hat == x_out;
+        const rs::GemmLn lnout = {fc2_stats ? hk->stats_out : nullptr, fc2_stats ? hk->parts_out : nullptr, nullptr, 0, nullptr, 0.f};
+        RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_tc(ctx, rs::RS_EPI_SCORE, h, w->w_fc2, w->b_fc2, x_prime, x, in_map, x_hat, d->out_dtype, fc2_parts, kind, (int)d->dist, T, D, Dm, st, fc2_stats ? &lnout : nullptr), "FC2+residual+score");
     } else {
         RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_simt(d->dtype, u, w->w_fc1, w->b_fc1, 1, nullptr, RS_F32, h, d->dtype, T, Dm, D, st), "FC1");
         RS_CHECK_LAUNCH(ctx, RS_K_GEMM, st, rs::launch_gemm_simt(d->dtype, h, w->w_fc2, w->b_fc2, 0, nullptr, RS_F32, m, RS_F32, T, D, Dm, st), "FC2");
@@ -486,6 +489,13 @@ static rs_status block_fwd_impl(rs_ctx* ctx, const rs_block_desc* d, const rs_bl
     const bool moves = x_hat != x_out;      // something is dropped: the kept rows are moved (or normalised) here
     const rs::LnFuse* ln = (hk && hk->next_ln && moves && rs::ln_fusable(d->out_dtype, D)) ? hk->next_ln : nullptr;
     if (ln && hk->ln_done) *hk->ln_done = true;
+    // the kept rows' sums for a LayerNorm folded into the next block's QKV (one pair per row)
+    rs::LnFuse sums = {nullptr, nullptr, 0.f, nullptr, nullptr};
+    if (!ln && tc && moves && dense_out && hk && hk->stats_out && !ragged && d->out_dtype == RS_BF16) {
+        sums.stats = hk->stats_out;
+        ln = &sums;
+        if (hk->parts_out) *hk->parts_out = 1;
+    }
     int32_t* out_map = (hk && moves) ? hk->out_map : nullptr;
     void* dense = dense_out ? x_out : nullptr;
     const int cls = d->has_cls ? 1 : 0;
@@ -645,17 +655,19 @@ rs_status rs_vit_fwd_taps(rs_ctx* ctx, const rs_vit_desc* d, const rs_block_weig
         // A block that drops tokens and whose compacted output nobody asked for writes no dense copy:
         // its un-pruned x^ stays in a token buffer and the next block reads the kept rows in place
         // (LN1 in the pruning kernel or through the map, the projection's residual through the map).
-        const bool in_place = !last && drops[l] > 0 && !taps->x_out[l] && rs_block_uses_tensor_cores(ctx, &bd);
+        // the next block's LN1 folded into its QKV product (its weights carry that form): this block hands over
+        // its output tokens themselves with their row sums, whether it drops tokens or not
+        const bool fold_next = !last && d->dtype == RS_BF16 && weights[l + 1].w_qkv_ln && weights[l + 1].c_qkv_ln &&
+                               weights[l + 1].b_qkv_ln && rs_block_uses_tensor_cores(ctx, &bd);
+        const bool in_place = !last && drops[l] > 0 && !taps->x_out[l] && !fold_next && rs_block_uses_tensor_cores(ctx, &bd);
         void* out = in_place ? nullptr : (taps->x_out[l] ? taps->x_out[l] : act[l & 1]);
         // LN1 of block l+1 rides in this block's pruning kernel: one kernel less per block
         const rs::LnFuse next = {last ? nullptr : weights[l + 1].ln1_g, last ? nullptr : weights[l + 1].ln1_b, eps, ln_buf};
         bool ln_done = false;
         // A block that drops nothing hands its output to the next block as it is: if that block's weights
         // carry LN1 folded into QKV, this block's FC2 leaves the row sums and no LN1 kernel runs.
-        const bool fold_next = !last && drops[l] == 0 && d->dtype == RS_BF16 && weights[l + 1].w_qkv_ln &&
-                               weights[l + 1].c_qkv_ln && weights[l + 1].b_qkv_ln && rs_block_uses_tensor_cores(ctx, &bd);
         int parts_out = 0;
-        const LoopHooks hk = {cur_map, cur_ln, (last || !next.gamma || !next.beta) ? nullptr : &next,
+        const LoopHooks hk = {cur_map, cur_ln, (last || fold_next || !next.gamma || !next.beta) ? nullptr : &next,
                               in_place ? maps[l & 1] : nullptr, !in_place, &ln_done, nullptr, nullptr, nullptr,
                               cur_stats, cur_parts, fold_next ? stats[l & 1] : nullptr, fold_next ? &parts_out : nullptr};
         rs_status st = block_fwd_impl(ctx, &bd, &weights[l], cur, out, taps->scores ? taps->scores[l] : nullptr,

@@ -107,7 +107,9 @@ cudaError_t launch_select(const float* scores, int nparts, float* scores_out, in
                           int sm_count, cudaStream_t st, int* launches);
 // The compaction kernels can also write LN(x_out) for the block that follows (its LN1 of Eq. att):
 // the warp that copies a kept row has it in registers.  out: [B, K, D] of the rows' dtype.
-struct LnFuse { const float* gamma; const float* beta; float eps; void* out; };
+// gamma == null with stats set: no LayerNorm; the kept rows are copied and the sum and sum of squares of each
+// copied row's bf16 values go to stats[2 * row], stats[2 * row + 1] (for a LayerNorm folded into the next product).
+struct LnFuse { const float* gamma; const float* beta; float eps; void* out; float* stats; };
 bool ln_fusable(rs_dtype dtype, int D);   // the row fits the registers of one warp
 // x_out may be null when ln is given: only the normalised rows are written (no dense copy).
 cudaError_t launch_gather(rs_dtype dtype, const void* x, const int32_t* keep_idx, int B, int N, int K,

@@ -192,6 +192,7 @@ __device__ __forceinline__ void copy_row(const uint4* __restrict__ src, long lon
                                          uint4* __restrict__ x_out, const LnFuse& ln) {
     if constexpr (std::is_void<LT>::value) {
         uint4* dst = x_out + orow * row_vecs;
+        float s1 = 0.f, s2 = 0.f;
         for (int base = 0; base < row_vecs; base += 32 * MAXV) {
             uint4 v[MAXV];
 #pragma unroll
@@ -202,8 +203,27 @@ __device__ __forceinline__ void copy_row(const uint4* __restrict__ src, long lon
 #pragma unroll
             for (int j = 0; j < MAXV; ++j) {
                 const int iv = base + j * 32 + lane;
-                if (iv < row_vecs) dst[iv] = v[j];
+                if (iv < row_vecs) {
+                    dst[iv] = v[j];
+                    if (ln.stats) {                  // bf16 rows only (the caller's business)
+                        const uint32_t w[4] = {v[j].x, v[j].y, v[j].z, v[j].w};
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const float y0 = __uint_as_float(w[e] << 16), y1 = __uint_as_float(w[e] & 0xffff0000u);
+                            s1 += y0 + y1;
+                            s2 = fmaf(y0, y0, fmaf(y1, y1, s2));
+                        }
+                    }
+                }
             }
+        }
+        if (ln.stats) {
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                s1 += __shfl_xor_sync(0xffffffffu, s1, o);
+                s2 += __shfl_xor_sync(0xffffffffu, s2, o);
+            }
+            if (lane == 0) { ln.stats[2 * orow] = s1; ln.stats[2 * orow + 1] = s2; }
         }
     } else {
         uint4 v[MAXV];
@@ -565,7 +585,7 @@ linewise_kernel(const float* __restrict__ scores, int H, int W, int Hk, int Wk, 
     const int P = Hk * Wk, G = gridDim.x, per = (P + G - 1) / G;
     const int lo = blockIdx.x * per, hi = min(lo + per, P);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
-    const LnFuse none = {nullptr, nullptr, 0.f, nullptr};
+    const LnFuse none = {nullptr, nullptr, 0.f, nullptr, nullptr};
     auto src_of = [&](int p) {
         const int i = p / Wk, j = p - i * Wk;
         return x + (((long long)b * H + kept[i]) * W + kept[kLineMax + j]) * row_vecs;
@@ -649,12 +669,13 @@ cudaError_t launch_prune(const float* scores, int nparts, float* scores_out, int
     if (launches) *launches = 0;
     if (B == 0) return cudaSuccess;
     const size_t per_sample = prune_scratch_per_sample(N);
-    if (N > kPruneMaxN || (ln && !ln_fusable(dtype, D)) || (x && !x_out && !ln) || flags_bytes < per_sample ||
+    const bool norm = ln && ln->gamma;               // else ln, if given, only asks for the row sums of the copy
+    if (N > kPruneMaxN || (norm && !ln_fusable(dtype, D)) || (x && !x_out && !norm) || flags_bytes < per_sample ||
         (reinterpret_cast<uintptr_t>(flags) & 3u))
         return cudaErrorInvalidValue;
     const int row_vecs = x ? (int)((size_t)D * dtype_size(dtype) / 16) : 0;
     const size_t sz = dtype_size(dtype);
-    const LnFuse none = {nullptr, nullptr, 0.f, nullptr};
+    const LnFuse none = {nullptr, nullptr, 0.f, nullptr, nullptr};
     // samples per pass: as many as the scratch holds (all of them, unless the batch is huge)
     const int Bc = (int)((flags_bytes / per_sample) < (size_t)B ? flags_bytes / per_sample : (size_t)B);
     for (int b0 = 0; b0 < B; b0 += Bc) {
@@ -665,7 +686,8 @@ cudaError_t launch_prune(const float* scores, int nparts, float* scores_out, int
         const uint4* xs = x ? (const uint4*)((const char*)x + (size_t)t0 * D * sz) : nullptr;
         uint4* xo = x_out ? (uint4*)((char*)x_out + (size_t)k0 * D * sz) : nullptr;
         LnFuse lnc = ln ? *ln : none;
-        if (ln) lnc.out = (char*)ln->out + (size_t)k0 * D * sz;
+        if (norm) lnc.out = (char*)ln->out + (size_t)k0 * D * sz;
+        if (ln && ln->stats) lnc.stats = ln->stats + 2 * k0;
         cudaError_t e;
         {
             // ranking: 64 tokens per CTA (4 threads each) up to 1024 tokens, else 128 (8 threads each);
@@ -687,7 +709,7 @@ cudaError_t launch_prune(const float* scores, int nparts, float* scores_out, int
 #define RS_GR_CASE(LT)                                                                                                  \
     launch_pdl(gather_ranked_kernel<4, LT>, grid, block, 0, st, xs, (const uint8_t*)fl, (const int32_t*)counts, nsl, P, \
                rows, N, K, b0, row_vecs, keep_idx + k0, rm, xo, lnc, rg)
-            if (!ln) e = RS_GR_CASE(void);
+            if (!norm) e = RS_GR_CASE(void);
             else if (dtype == RS_BF16) e = RS_GR_CASE(__nv_bfloat16);
             else e = RS_GR_CASE(float);
 #undef RS_GR_CASE
@@ -704,12 +726,13 @@ cudaError_t launch_gather(rs_dtype dtype, const void* x, const int32_t* keep_idx
     if (rows == 0) return cudaSuccess;
     const int row_vecs = (int)((size_t)D * dtype_size(dtype) / 16);
     const unsigned grid = (unsigned)((rows + 7) / 8);
-    if ((ln && !ln_fusable(dtype, D)) || (!x_out && !ln)) return cudaErrorInvalidValue;
-    const LnFuse none = {nullptr, nullptr, 0.f, nullptr};
+    const bool norm = ln && ln->gamma;
+    if ((norm && !ln_fusable(dtype, D)) || (!x_out && !norm)) return cudaErrorInvalidValue;
+    const LnFuse none = {nullptr, nullptr, 0.f, nullptr, nullptr};
 #define RS_G_CASE(LT)                                                                                               \
     launch_pdl(gather_kernel<4, LT>, dim3(grid), dim3(256), 0, st, (const uint4*)x, keep_idx, rows, N, K, row_vecs, \
                (uint4*)x_out, ln ? *ln : none)
-    if (!ln) return RS_G_CASE(void);
+    if (!norm) return RS_G_CASE(void);
     return dtype == RS_BF16 ? RS_G_CASE(__nv_bfloat16) : RS_G_CASE(float);
 #undef RS_G_CASE
 }
