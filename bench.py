@@ -504,7 +504,9 @@ def run_gpu(args, wl):
     sz = 2 if wl.dtype == "bf16" else 4
     gather_bytes = sum(2 * wl.B * (n - r) * wl.D * sz for n, r in zip(Ns, wl.drops) if r > 0)
     # pruning blocks before the last write no dense copy of their kept tokens (read in place by the next block)
-    dense_copy_bytes_removed = sum(wl.B * (n - r) * wl.D * sz for n, r in list(zip(Ns, wl.drops))[:-1] if r > 0)
+    # (with the LayerNorm fold the kept rows are copied, un-normalised, instead of their LN1 being written: the same bytes)
+    dense_copy_bytes_removed = (sum(wl.B * (n - r) * wl.D * sz for n, r in list(zip(Ns, wl.drops))[:-1] if r > 0)
+                                if args.no_ln_fold or wl.dtype != "bf16" else 0)
     cls_ms = m["cls_ms"]
     other_cls = "attn" if dom == "gemm" else "gemm"
     parts = {
@@ -515,8 +517,10 @@ def run_gpu(args, wl):
         "gather": dict(ms_per_step=m["raw_ms"]["gather"], ms_per_step_overhead_corrected=cls_ms["gather"],
                        gbs=(gather_bytes / (m["raw_ms"]["gather"] * 1e-3) / 1e9 if m["raw_ms"]["gather"] else 0.0),
                        dense_copy_bytes_not_written_per_step=dense_copy_bytes_removed,
-                       note="selection, index lists and LN1 of the next block in one kernel for N <= 4608; the dense "
-                            "[B, K, D] copy is written for the last block only"),
+                       note=("selection, index lists and LN1 of the next block in one kernel for N <= 4608; the dense "
+                             "[B, K, D] copy is written for the last block only") if args.no_ln_fold else
+                            ("selection, index lists, the kept rows and their sums (LN1 of the next block is applied "
+                             "inside its QKV product)")),
         "select": dict(ms_per_step=m["raw_ms"]["select"]),
         "layernorm": dict(ms_per_step=m["raw_ms"]["layernorm"]),
         "note": "in-situ, event-timed; activations between kernels sit in the 126 MB L2 "
