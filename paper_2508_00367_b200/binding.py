@@ -593,7 +593,7 @@ class PrunedViT:
         self.tapped = set(range(L)) if tap_blocks is None else (set(int(b) for b in tap_blocks) | {L - 1})
         self.has_cls, self.score_mode, self.dist = has_cls, score_mode, dist
         self.weights: List[DeviceBlockWeights] = [DeviceBlockWeights(w, dtype, ctx.device) for w in blocks]
-        if fold_ln1 and dtype == torch.bfloat16:
+        if fold_ln1 and dtype == torch.bfloat16 and self.weights[0].t["w_qkv"].shape[1] % 128 == 0:
             # LN1 of every block but the first is applied inside its QKV product
             for l in range(1, L):
                 self.weights[l].fold_ln1(ctx)
