@@ -514,6 +514,8 @@ def run_gpu(args, wl):
         "attn_target_0p60_met": bool(cr["attn"]["frac"] >= 0.60),
         "attn_kernels": "attn_tc_kernel (two query tiles per CTA) or attn_tc3_kernel (three, 64-key tiles), "
                         "whichever the library's cost model expects to be faster for the block's B, N and H",
+        "attn_kernel_by_tokens": {str(n): rs.attn_kernel_choice(torch.cuda.get_device_properties(dev).multi_processor_count,
+                                                                 wl.B, wl.H, n) for n in sorted(set(Ns), reverse=True)},
         "gather": dict(ms_per_step=m["raw_ms"]["gather"], ms_per_step_overhead_corrected=cls_ms["gather"],
                        gbs=(gather_bytes / (m["raw_ms"]["gather"] * 1e-3) / 1e9 if m["raw_ms"]["gather"] else 0.0),
                        dense_copy_bytes_not_written_per_step=dense_copy_bytes_removed,

@@ -32,6 +32,11 @@ RS_API rs_status rs_timing_read(rs_ctx* ctx, void* stream, double* ms /*host[RS_
  * shape, box) and kept in a 128-slot cache of the context.  Hits and misses so far (host counters). */
 RS_API rs_status rs_tmap_cache_stats(const rs_ctx* ctx, long long* hits /*host*/, long long* misses /*host*/);
 
+/* Which of the two tensor-core attention kernels rs_attn_fwd picks for B samples, H heads and N tokens on a
+ * GPU of sm_count SMs: 2 (two query tiles per thread block; also every N <= 128) or 3 (three).  Host
+ * arithmetic only (the cost model of the choice); needs no context and no GPU. */
+RS_API int rs_attn_kernel_choice(int sm_count, int B, int H, int N);
+
 #ifdef __cplusplus
 }
 #endif

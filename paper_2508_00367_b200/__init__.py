@@ -5,4 +5,4 @@ the package needs neither a GPU nor the built library, so the input generator
 (`synth`) and the build script stay importable everywhere.
 """
 from .binding import (Context, block_fwd_static, static_async_status, DeviceBlockWeights, PrunedViT, RsError, load_library, LIB_PATH,  # noqa: F401
-                      EXPORTS)
+                      EXPORTS, attn_kernel_choice)

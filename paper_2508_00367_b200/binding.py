@@ -28,7 +28,7 @@ EXPORTS = ("rs_create", "rs_destroy", "rs_last_error", "rs_async_status", "rs_us
            "rs_block_workspace_bytes", "rs_block_fwd", "rs_timing_enable", "rs_timing_read",
            "rs_static_scratch_bytes", "rs_block_fwd_static", "rs_linear_fwd", "rs_vit_workspace_bytes", "rs_vit_fwd",
            "rs_vit_fwd_taps", "rs_linewise_compact", "rs_static_async_status", "rs_linear_uses_tensor_cores",
-           "rs_block_uses_tensor_cores", "rs_attn_fwd_ragged", "rs_topk_compact_ragged", "rs_block_fwd_ragged", "rs_vit_fwd_ragged", "rs_prepare_ln1_fold", "rs_tmap_cache_stats")
+           "rs_block_uses_tensor_cores", "rs_attn_fwd_ragged", "rs_topk_compact_ragged", "rs_block_fwd_ragged", "rs_vit_fwd_ragged", "rs_prepare_ln1_fold", "rs_attn_kernel_choice", "rs_tmap_cache_stats")
 LIN_EPILOGUE = {"bias": 0, "gelu": 1, "residual": 2}
 KERNEL_CLASSES = ("layernorm", "gemm", "attn", "score", "select", "gather")
 
@@ -153,8 +153,15 @@ def load_library() -> ctypes.CDLL:
     lib.rs_vit_fwd_ragged.restype = ci
     lib.rs_prepare_ln1_fold.argtypes = [vp, ci, ci, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.rs_prepare_ln1_fold.restype = ci
+    lib.rs_attn_kernel_choice.argtypes = [ci, ci, ci, ci]
+    lib.rs_attn_kernel_choice.restype = ci
     _lib = lib
     return lib
+
+
+def attn_kernel_choice(sm_count: int, B: int, H: int, N: int) -> int:
+    """rs_attn_kernel_choice: 2 or 3, the attention kernel rs_attn_fwd picks for the shape (host arithmetic only)."""
+    return int(load_library().rs_attn_kernel_choice(sm_count, B, H, N))
 
 
 def _dt(t: torch.Tensor) -> int:

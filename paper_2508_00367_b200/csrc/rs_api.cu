@@ -193,6 +193,12 @@ int rs_uses_tensor_cores(const rs_ctx* ctx, rs_dtype dtype) {
 
 long long rs_launch_count(const rs_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
+int rs_attn_kernel_choice(int sm_count, int B, int H, int N) {
+    if (sm_count < 1 || B < 1 || H < 1 || N < 1) return 0;
+    if (N <= 128) return 2;
+    return rs::attn_plan((long long)B * H, N, sm_count).three ? 3 : 2;
+}
+
 rs_status rs_tmap_cache_stats(const rs_ctx* ctx, long long* hits, long long* misses) {
     if (!ctx || !hits || !misses) return RS_ERR_INVALID_ARG;
     *hits = ctx->tmap_hits;

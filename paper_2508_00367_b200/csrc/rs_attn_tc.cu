@@ -488,6 +488,54 @@ bool attn_tc_supported(const rs_attn_desc& d) {
     return true;
 }
 
+// How a shape with more than one query tile per head is run (host side, remembered per shape).
+// Two query tiles per CTA (this file): items go to the CTAs round robin, and a pair of query tiles costs
+// twice a single one, so a last round with few pairs left keeps most SMs idle for a whole pair's time.
+// The tiles of the last few (sample, head)s are therefore handed out one by one where that shortens the
+// longest CTA: best_hs is the count with the smallest makespan under the cost model pair = 10, single = 7
+// (a query tile alone runs faster than next to another, but not twice as fast: measured).
+// This kernel or the one with three query tiles per CTA (rs_attn_tc3.cu)?  Both are paced by the longest
+// CTA: its items (in tenths) times the key tiles of an item, plus a cost per item; microseconds fitted to
+// CUDA-event times of thirteen shapes from N = 197 to 4097 (worst error 6 % and 9 %).
+AttnPlan attn_plan(long long BH, int N, int G) {
+    const int nt = (N + BQ - 1) / BQ, per = (N + 2 * BQ - 1) / (2 * BQ);
+    auto makespan = [&](long long hs) {
+        const long long pair_items = (BH - hs) * per, singles = hs * nt, all = pair_items + singles;
+        long long worst = 0;
+        for (int c = 0; c < G && c < all; ++c) {          // CTA c takes items c, c + G, ...
+            long long load = 0;
+            for (long long w = c; w < all; w += G)
+                load += w < pair_items ? (((w % per) == per - 1 && (nt & 1)) ? 7 : 10) : 7;
+            if (load > worst) worst = load;
+        }
+        return worst;
+    };
+    static std::mutex memo_mu;
+    static std::map<std::tuple<long long, int, int>, AttnPlan> memo;
+    AttnPlan plan = {0, 0, 0};
+    const auto key = std::make_tuple(BH, N, G);
+    std::lock_guard<std::mutex> lock(memo_mu);
+    const auto hit = memo.find(key);
+    if (hit != memo.end()) return hit->second;
+    long long hs_max = (2ll * G + nt - 1) / nt + 1;        // enough single tiles for two rounds
+    if (hs_max > BH) hs_max = BH;
+    long long best = -1;
+    if (N > BQ && BH * per <= 200000) {                   // (a host loop over the items for every candidate)
+        for (long long hs = 0; hs <= hs_max; ++hs) {
+            const long long m = makespan(hs);
+            if (best < 0 || m < best) { best = m; plan.best_hs = hs; }
+        }
+        int wrap3 = 0;
+        const long long u3 = attn_tc3_plan(BH, N, G, &wrap3);
+        const double t2 = best / 10.0 * (((N + BKV - 1) / BKV) * 1.505 + 2.51) + 2.32;
+        const double t3 = u3 / 10.0 * (((N + 63) / 64) * 1.136 + 1.00) + 6.71;
+        plan.three = t3 < t2;
+        plan.wrap3 = wrap3;
+    }
+    memo[key] = plan;
+    return plan;
+}
+
 cudaError_t launch_attn_tc(rs_ctx* ctx, const rs_attn_desc& d, const void* q, const void* k, const void* v,
                            void* out, const int32_t* seq_lens, cudaStream_t st) {
     if (!ctx->encode_tiled) return cudaErrorNotSupported;
@@ -517,58 +565,9 @@ cudaError_t launch_attn_tc(rs_ctx* ctx, const rs_attn_desc& d, const void* q, co
     if (items >= (1ll << 30)) return cudaErrorInvalidValue;
     args.n_pair_items = (int)items; args.first_single_bh = d.B * d.H; args.tile_count = (d.N + BQ - 1) / BQ;
     if (!args.dual) {
-        // Items go to the CTAs round robin, and a pair of query tiles costs twice a single one, so a
-        // last round with few pairs left keeps most SMs idle for a whole pair's time.  The tiles of the
-        // last few (sample, head)s are therefore handed out one by one where that shortens the longest
-        // CTA: the count is the one with the smallest makespan under the cost model pair = 10, single = 7
-        // (a query tile alone runs faster than next to another, but not twice as fast: measured).
         const long long BH = (long long)d.B * d.H;
-        const int G = ctx->sm_count, nt = args.tile_count, per = args.per;
-        auto makespan = [&](long long hs) {
-            const long long pair_items = (BH - hs) * per, singles = hs * nt, all = pair_items + singles;
-            long long worst = 0;
-            for (int c = 0; c < G && c < all; ++c) {          // CTA c takes items c, c + G, ...
-                long long load = 0;
-                for (long long w = c; w < all; w += G)
-                    load += w < pair_items ? (((w % per) == per - 1 && (nt & 1)) ? 7 : 10) : 7;
-                if (load > worst) worst = load;
-            }
-            return worst;
-        };
-        // (a host loop over the items for every candidate: the answer is remembered per shape)
-        static std::mutex memo_mu;
-        struct Plan { long long best_hs; int three, wrap3; };
-        static std::map<std::tuple<long long, int, int>, Plan> memo;
-        Plan plan = {0, 0, 0};
-        const auto key = std::make_tuple(BH, d.N, G);
-        std::unique_lock<std::mutex> lock(memo_mu);
-        const auto hit = memo.find(key);
-        if (hit != memo.end()) {
-            plan = hit->second;
-        } else {
-            long long hs_max = (2ll * G + nt - 1) / nt + 1;    // enough single tiles for two rounds
-            if (hs_max > BH) hs_max = BH;
-            long long best = -1;
-            if (BH * per <= 200000) {
-                for (long long hs = 0; hs <= hs_max; ++hs) {
-                    const long long m = makespan(hs);
-                    if (best < 0 || m < best) { best = m; plan.best_hs = hs; }
-                }
-                // This kernel or the one with three query tiles per CTA (rs_attn_tc3.cu)?  Both are
-                // paced by the longest CTA: its items (in tenths) times the key tiles of an item,
-                // plus a cost per item; microseconds fitted to CUDA-event times of thirteen shapes
-                // from N = 197 to 4097 (worst error 6 % and 9 %).  Sequences with lengths of their
-                // own stay here.
-                int wrap3 = 0;
-                const long long u3 = attn_tc3_plan(BH, d.N, G, &wrap3);
-                const double t2 = best / 10.0 * (((d.N + BKV - 1) / BKV) * 1.505 + 2.51) + 2.32;
-                const double t3 = u3 / 10.0 * (((d.N + 63) / 64) * 1.136 + 1.00) + 6.71;
-                plan.three = t3 < t2;
-                plan.wrap3 = wrap3;
-            }
-            memo[key] = plan;
-        }
-        lock.unlock();
+        const int nt = args.tile_count, per = args.per;
+        const AttnPlan plan = attn_plan(BH, d.N, ctx->sm_count);
         const int force = ctx->attn_kernel;                    // RS_ATTN_KERNEL=2 / 3: one kernel for every shape it takes
         if (!seq_lens && (force == 3 || (force != 2 && plan.three))) {
             CUtensorMap tmK3, tmV3;

@@ -173,6 +173,10 @@ cudaError_t launch_gemm_tc(rs_ctx* ctx, int epi, const void* A, const void* W, c
 
 // ---- tcgen05 attention (rs_attn_tc.cu): bf16, head dimension 64 ----
 bool attn_tc_supported(const rs_attn_desc& d);
+// Which attention kernel runs a shape of BH (sample, head)s and N > 128 tokens on G SMs, and how: best_hs heads handed
+// out tile by tile (two-tile kernel), three = the three-tile kernel is expected to be faster, wrap3 its tail placement.
+struct AttnPlan { long long best_hs; int three, wrap3; };
+AttnPlan attn_plan(long long BH, int N, int G);
 // Three query tiles per CTA (rs_attn_tc3.cu), N > 128: the longest CTA's load under its item list, and the launch.
 long long attn_tc3_plan(long long BH, int N, int G, int* wrap);
 cudaError_t launch_attn_tc3(rs_ctx* ctx, const rs_attn_desc& d, const CUtensorMap& tmQ, const CUtensorMap& tmK,

@@ -217,3 +217,21 @@ def test_gelu_polynomial_matches_exact_erf_gelu():
     consts = [float(m) for m in re.findall(r"(-?\d+\.\d+(?:e-?\d+)?)f", body)]
     in_kernel = np.array(consts[:6][::-1], dtype=np.float64)     # Horner order is highest degree first
     assert fg.max_error_fp32(in_kernel) < 1e-6
+
+
+def test_attention_kernel_choice_follows_the_measured_winners():
+    """The cost model that picks between the two attention kernels (two or three query tiles per thread
+    block) against the kernel that was the faster one when both were timed on a B200 of 148 SMs (CUDA
+    events over graph replays; the one shape the model gets wrong, B=4 H=16 N=2305, lost 3 %)."""
+    import paper_2508_00367_b200 as rs
+    measured = {  # (B, H, N): faster kernel
+        (4, 16, 4097): 3, (4, 16, 3073): 3, (4, 16, 1729): 2, (4, 16, 1297): 3, (16, 12, 1569): 3, (16, 12, 1099): 3,
+        (16, 12, 770): 3, (16, 12, 539): 2, (32, 16, 577): 3, (32, 16, 337): 3, (64, 12, 197): 2, (1, 16, 4097): 2,
+    }
+    for (B, H, N), want in measured.items():
+        assert rs.attn_kernel_choice(148, B, H, N) == want, (B, H, N)
+    assert rs.attn_kernel_choice(148, 4, 16, 2305) == 2          # measured 151.5 against 147.1 us: the known miss
+    for N in (1, 64, 128):
+        assert rs.attn_kernel_choice(148, 64, 12, N) == 2        # one query tile per head: two heads per item
+    assert rs.attn_kernel_choice(0, 1, 1, 1) == 0
+
